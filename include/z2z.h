@@ -1,0 +1,177 @@
+/*
+ * z2z.h — C ABI of the zip2zip dynamic-vocabulary hot path on NVIDIA B200 (sm_100a).
+ *
+ * The library implements the work the method adds to every prefill and decode step of an LLM
+ * (paper Section 2): the per-sequence LZW codebook (Section 2.1), the hyper-encoder that turns a
+ * new codebook entry into a hyper-embedding / hyper-unembedding row (Section 2.2), and logits
+ * over the static vocabulary joined with the sequence's own hypertokens with the reductions
+ * taken from them (Section 2.3, steps 7-10).
+ *
+ * Conventions for every entry point
+ *   - Returns an int32 status: Z2Z_OK or a negative Z2Z_ERR_* for errors the host can detect
+ *     (bad arguments, workspace too small, a CUDA launch error).  Never throws, never exits.
+ *   - Conditions only the device can see are OR-ed into a per-sequence status word
+ *     (Z2Z_ST_* bits), readable with z2z_status().
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller owns every
+ *     buffer; the library allocates no device memory.  The opaque handle is host memory that
+ *     stores the configuration and offsets into the caller's workspace.
+ *   - All work is enqueued on the given stream and returns without synchronising (except
+ *     z2z_status, which waits for the stream).
+ *   - Ids are int32.  Tables are row-major [rows, d] in the configured dtype.
+ *   - Hypertoken id = V + k where k is the creation order within the sequence.
+ *   - Limits: V + cap < 2^24 - 1, cap <= 65535, 1 <= M <= 8, d % 8 == 0, B <= 1024.
+ */
+#ifndef Z2Z_H_
+#define Z2Z_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* z2z_stream;          /* a cudaStream_t */
+typedef struct z2z_codebook z2z_codebook;        /* opaque, host memory */
+
+enum {
+  Z2Z_OK = 0,
+  Z2Z_ERR_INVALID_ARG = -1,
+  Z2Z_ERR_WORKSPACE_TOO_SMALL = -2,
+  Z2Z_ERR_CUDA = -3,
+  Z2Z_ERR_UNSUPPORTED = -4
+};
+
+/* bits of the per-sequence device status word */
+enum {
+  Z2Z_ST_CAP_FROZEN = 1,     /* codebook reached cap: matching continues, inserting stopped  */
+  Z2Z_ST_BAD_TOKEN = 2,      /* a code named a hypertoken that does not exist; state unchanged */
+  Z2Z_ST_TABLE_FULL = 4,     /* hash probe ran through the whole table (cannot happen at load <= 1/2) */
+  Z2Z_ST_WAIT_TIMEOUT = 8    /* a bounded wait inside a kernel gave up                          */
+};
+
+enum { Z2Z_DTYPE_FP32 = 0, Z2Z_DTYPE_BF16 = 1 };
+enum { Z2Z_SELECT_ARGMAX = 0, Z2Z_SELECT_GUMBEL = 1 };
+enum { Z2Z_CACHE_EMBED = 0, Z2Z_CACHE_UNEMBED = 1 };
+
+typedef struct {
+  int32_t V;            /* static vocabulary size                                   */
+  int32_t d;            /* embedding dimension                                      */
+  int32_t M;            /* maximum merge size (Section 2.1)                         */
+  int32_t cap;          /* maximum hypertokens per sequence; at cap the book freezes */
+  int32_t B;            /* sequences in the session                                 */
+  int32_t dtype;        /* Z2Z_DTYPE_*: tables, encoder tensors, hidden states, caches */
+  int32_t enc_layers;   /* hyper-encoder layers; 0 = the parameter-free averaging variant */
+  int32_t enc_heads;    /* attention heads (d % enc_heads == 0)                     */
+  int32_t enc_dff;      /* feed-forward width                                       */
+  int32_t tied;         /* 1: the caller passes the same cache for both sides       */
+} z2z_config;
+
+/* Hyper-encoder parameters (Section 2.2; Section 3.1: transformer encoder layers), all in the
+ * configured dtype, as a HOST array of DEVICE pointers in this order:
+ *   pos[M,d], then for each layer:
+ *   ln1_w[d] ln1_b[d] Wqkv[3d,d] bqkv[3d] Wo[d,d] bo[d] ln2_w[d] ln2_b[d] W1[dff,d] b1[dff] W2[d,dff] b2[d]
+ * n_tensors must be 1 + 12 * enc_layers.                                                      */
+typedef struct {
+  const void* const* tensors;
+  int32_t n_tensors;
+} z2z_encoder_weights;
+
+/* Bytes of device workspace the session needs (codebooks, counters, kernel scratch). */
+int32_t z2z_workspace_bytes(const z2z_config* cfg, size_t* out_bytes);
+
+/* Section 2.2 "At the beginning of each inference session V_h is initialized as an empty set".
+ * Creates the handle on first use (*cb == NULL) and clears every sequence's codebook, counters
+ * and status.  d_ws must be 256-byte aligned and stay valid for the life of the handle.  May be
+ * called again on an existing handle to start a new session.                                   */
+int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, size_t ws_bytes,
+                          z2z_stream stream);
+
+/* Section 2.1 / Section 2.3 step 2: compress each prompt with LZW (greedy longest match against
+ * the growing codebook; new entry = emitted phrase + next base token, only if shorter than M
+ * tokens before the append and the book is not full).
+ *   d_tokens [B, T_max] int32 base tokens in [0, V); d_lens [B] valid length of each row.
+ *   d_codes  [B, T_max] int32 out; d_code_lens [B] out.
+ *   d_entries_after [B, T_max] int32 out or NULL: hypertokens that exist once code i is emitted.
+ * Leaves every sequence ready for z2z_lzw_step (previous code = its last code).               */
+int32_t z2z_lzw_encode(z2z_codebook* cb, const int32_t* d_tokens, const int32_t* d_lens,
+                       int32_t T_max, int32_t* d_codes, int32_t* d_code_lens,
+                       int32_t* d_entries_after, z2z_stream stream);
+
+/* Figure 1 / Section 2.3 step 10: online update with one newly selected code per sequence.
+ * Candidate entry = phrase(previous code) ++ first base token of phrase(new code); created if
+ * the previous phrase is shorter than M, the book is not full and the phrase is not there yet.
+ *   d_new_codes [B]; d_active [B] (0 = skip this sequence) or NULL;
+ *   d_new_entry [B] out: entry number created, or -1.
+ * A code >= V + n that is not the one this very step creates sets Z2Z_ST_BAD_TOKEN and leaves
+ * that sequence untouched (Section 2.3, "Consistent Vocabulary Updates").                     */
+int32_t z2z_lzw_step(z2z_codebook* cb, const int32_t* d_new_codes, const uint8_t* d_active,
+                     int32_t* d_new_entry, z2z_stream stream);
+
+/* Section 2.2 + Section 2.3 "Hyper-Embedding Cache": run the hyper-encoder over entries
+ * [first_b, first_b + count_b) of every sequence and store one d-vector per entry.
+ *   which    Z2Z_CACHE_EMBED (rows of W_E in, E_h out) or Z2Z_CACHE_UNEMBED (W_U in, U_h out);
+ *            only selects which "embedded so far" counter is used when d_first/d_count are NULL.
+ *   d_table  [V, d]; enc: that side's encoder.
+ *   d_first / d_count [B] or both NULL = every entry created since the last such call.
+ *   max_entries  host upper bound on sum_b count_b (<= 0: B * cap); bounds the launch count.
+ *   d_cache  [B, cap, d] in the configured dtype (row k of sequence b = hypertoken V + k).
+ *   d_cache_f32 [B, cap, d] fp32 or NULL: the same rows before rounding to the cache dtype.    */
+int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
+                        const z2z_encoder_weights* enc, const int32_t* d_first,
+                        const int32_t* d_count, int32_t max_entries, void* d_cache,
+                        float* d_cache_f32, z2z_stream stream);
+
+/* Section 2.3 steps 7-9: for each of N hidden rows, logits over W_U joined with the first
+ * n_vis rows of the owning sequence's U_h; log-sum-exp, argmax (lowest index on ties) and
+ * optionally a Gumbel-max sample at the given temperature.  The logit matrix is not stored.
+ *   d_hidden [N, d]; d_row_seq [N] owning sequence of each row (NULL: row r belongs to r);
+ *   d_row_nvis [N] visible hypertokens per row or NULL = all n_b of the sequence;
+ *   d_WU [V, d]; d_Uh [B, cap, d];
+ *   select/temperature/seed/step: sampling (Philox4x32-10 keyed by seed, counter
+ *            (column/4, row, step), u = ((x >> 9) + 0.5) * 2^-23, g = -log(-log u));
+ *   d_targets [N] or NULL -> d_target_logit [N] = logit of that column (NaN if not visible);
+ *   d_lse [N], d_argmax [N], d_max_logit [N]; d_sample [N] (required iff select == GUMBEL);
+ *   d_logits_debug [N, V + cap] fp32 or NULL: every logit, for tests.                         */
+int32_t z2z_dynamic_logits(z2z_codebook* cb, const void* d_hidden, int32_t N,
+                           const int32_t* d_row_seq, const int32_t* d_row_nvis, const void* d_WU,
+                           const void* d_Uh, int32_t select, float temperature, uint64_t seed,
+                           uint64_t step, const int32_t* d_targets, float* d_lse,
+                           int32_t* d_argmax, float* d_max_logit, int32_t* d_sample,
+                           float* d_target_logit, float* d_logits_debug, z2z_stream stream);
+
+/* One whole decode step (Section 2.3 steps 7-10 and the cache update): logits and selection for
+ * hidden row b of sequence b, LZW update with the selected code, hyper-encoder on the at most
+ * one new entry per sequence for both caches.
+ *   d_forced [B] or NULL: codes to feed the update instead of the selection (teacher forcing;
+ *            the selection is still computed and returned in d_selected).
+ *   d_next_codes [B] out: the code that was applied; d_selected [B] out or NULL: argmax/sample;
+ *   d_lse [B] out; d_new_entry [B] out or NULL.
+ *   d_Eh_f32 / d_Uh_f32: optional fp32 copies of the new rows, as in z2z_hyper_embed.          */
+int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE,
+                        const void* d_WU, const z2z_encoder_weights* enc_E,
+                        const z2z_encoder_weights* enc_U, void* d_Eh, void* d_Uh,
+                        int32_t select, float temperature, uint64_t seed, uint64_t step,
+                        const int32_t* d_forced, int32_t* d_next_codes, int32_t* d_selected,
+                        float* d_lse, int32_t* d_new_entry, float* d_Eh_f32, float* d_Uh_f32,
+                        z2z_stream stream);
+
+/* Waits for the stream, then copies per-sequence status bits and hypertoken counts to the host.
+ * Either output may be NULL.                                                                  */
+int32_t z2z_status(z2z_codebook* cb, int32_t* h_status, int32_t* h_n, z2z_stream stream);
+
+/* Copies the codebook of one sequence to the host for inspection: constituents
+ * h_cons [cap, M] (-1 padded) and lengths h_len [cap]; waits for the stream.                  */
+int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t* h_len,
+                          z2z_stream stream);
+
+/* Frees the host handle (never the workspace). */
+int32_t z2z_codebook_destroy(z2z_codebook* cb);
+
+/* Text of the last host-side error on this thread (static storage). */
+const char* z2z_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* Z2Z_H_ */

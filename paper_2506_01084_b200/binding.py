@@ -1,0 +1,193 @@
+"""ctypes binding of the C ABI in include/z2z.h: same names, argument marshalling only.
+
+Every call takes torch tensors (device memory owned by the caller) and forwards raw pointers and
+the current CUDA stream.  Nothing is computed here; if the shared library has not been built the
+import of the library fails loudly (there is no fallback path).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libz2z.so")
+
+OK = 0
+ST_CAP_FROZEN, ST_BAD_TOKEN, ST_TABLE_FULL, ST_WAIT_TIMEOUT = 1, 2, 4, 8
+DTYPE_FP32, DTYPE_BF16 = 0, 1
+SELECT_ARGMAX, SELECT_GUMBEL = 0, 1
+CACHE_EMBED, CACHE_UNEMBED = 0, 1
+
+EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lzw_step",
+           "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
+           "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error"]
+
+
+class Config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("V", "d", "M", "cap", "B", "dtype", "enc_layers",
+                                         "enc_heads", "enc_dff", "tied")]
+
+
+class EncoderWeights(C.Structure):
+    _fields_ = [("tensors", C.POINTER(C.c_void_p)), ("n_tensors", C.c_int32)]
+
+
+class Z2ZError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the shared library (once).  Raises if it is missing: build it first with
+    ``python -m paper_2506_01084_b200.build``."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise Z2ZError(f"{LIB_PATH} not found: run `python -m paper_2506_01084_b200.build`")
+        _lib = C.CDLL(LIB_PATH)
+        _lib.z2z_last_error.restype = C.c_char_p
+        for name in EXPORTS:
+            if name != "z2z_last_error":
+                getattr(_lib, name).restype = C.c_int32
+    return _lib
+
+
+def _check(rc: int):
+    if rc != OK:
+        raise Z2ZError(f"z2z error {rc}: {lib().z2z_last_error().decode()}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return C.c_void_p(0)
+    assert t.is_contiguous(), "tensors passed to the ABI must be contiguous"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_config(V, d, M, cap, B, dtype, enc_layers, enc_heads, enc_dff, tied=0) -> Config:
+    if dtype in ("fp32", torch.float32):
+        dt = DTYPE_FP32
+    elif dtype in ("bf16", torch.bfloat16):
+        dt = DTYPE_BF16
+    else:
+        dt = int(dtype)
+    return Config(V, d, M, cap, B, dt, enc_layers, enc_heads, enc_dff, tied)
+
+
+def encoder_weights(tensors: Sequence[torch.Tensor]) -> EncoderWeights:
+    """HOST array of DEVICE pointers in ABI order.  The returned struct keeps the array alive."""
+    arr = (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+    ew = EncoderWeights(C.cast(arr, C.POINTER(C.c_void_p)), len(tensors))
+    ew._keep = (arr, list(tensors))
+    return ew
+
+
+def z2z_workspace_bytes(cfg: Config) -> int:
+    out = C.c_size_t(0)
+    _check(lib().z2z_workspace_bytes(C.byref(cfg), C.byref(out)))
+    return out.value
+
+
+class Codebook:
+    """Owns the opaque handle; the workspace tensor is allocated by the caller side (torch)."""
+
+    def __init__(self, cfg: Config, device="cuda:0"):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        nbytes = z2z_workspace_bytes(cfg)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        off = (-self.workspace.data_ptr()) % 256
+        self._ws_ptr = self.workspace.data_ptr() + off
+        self._ws_bytes = nbytes
+        self.handle = C.c_void_p(0)
+        z2z_codebook_init(self)
+
+    def __del__(self):
+        try:
+            if self.handle and _lib is not None:
+                _lib.z2z_codebook_destroy(self.handle)
+                self.handle = C.c_void_p(0)
+        except Exception:
+            pass
+
+
+def z2z_codebook_init(cb: Codebook):
+    _check(lib().z2z_codebook_init(C.byref(cb.handle), C.byref(cb.cfg), C.c_void_p(cb._ws_ptr),
+                                   C.c_size_t(cb._ws_bytes), _stream()))
+
+
+def z2z_lzw_encode(cb: Codebook, tokens: torch.Tensor, lens: Optional[torch.Tensor],
+                   codes: torch.Tensor, code_lens: torch.Tensor,
+                   entries_after: Optional[torch.Tensor] = None):
+    T_max = tokens.shape[1] if tokens.dim() == 2 else 0
+    _check(lib().z2z_lzw_encode(cb.handle, _ptr(tokens), _ptr(lens), C.c_int32(T_max), _ptr(codes),
+                                _ptr(code_lens), _ptr(entries_after), _stream()))
+
+
+def z2z_lzw_step(cb: Codebook, new_codes: torch.Tensor, active: Optional[torch.Tensor],
+                 new_entry: Optional[torch.Tensor]):
+    _check(lib().z2z_lzw_step(cb.handle, _ptr(new_codes), _ptr(active), _ptr(new_entry), _stream()))
+
+
+def z2z_hyper_embed(cb: Codebook, which: int, table: torch.Tensor, enc: EncoderWeights,
+                    first: Optional[torch.Tensor], count: Optional[torch.Tensor], max_entries: int,
+                    cache: torch.Tensor, cache_f32: Optional[torch.Tensor] = None):
+    _check(lib().z2z_hyper_embed(cb.handle, C.c_int32(which), _ptr(table), C.byref(enc),
+                                 _ptr(first), _ptr(count), C.c_int32(max_entries), _ptr(cache),
+                                 _ptr(cache_f32), _stream()))
+
+
+def z2z_dynamic_logits(cb: Codebook, hidden: torch.Tensor, row_seq: Optional[torch.Tensor],
+                       row_nvis: Optional[torch.Tensor], W_U: torch.Tensor, U_h: torch.Tensor,
+                       select: int, temperature: float, seed: int, step: int,
+                       targets: Optional[torch.Tensor], lse: Optional[torch.Tensor],
+                       argmax: Optional[torch.Tensor], max_logit: Optional[torch.Tensor],
+                       sample: Optional[torch.Tensor] = None,
+                       target_logit: Optional[torch.Tensor] = None,
+                       logits_debug: Optional[torch.Tensor] = None):
+    N = hidden.shape[0]
+    _check(lib().z2z_dynamic_logits(cb.handle, _ptr(hidden), C.c_int32(N), _ptr(row_seq),
+                                    _ptr(row_nvis), _ptr(W_U), _ptr(U_h), C.c_int32(select),
+                                    C.c_float(temperature), C.c_uint64(seed), C.c_uint64(step),
+                                    _ptr(targets), _ptr(lse), _ptr(argmax), _ptr(max_logit),
+                                    _ptr(sample), _ptr(target_logit), _ptr(logits_debug), _stream()))
+
+
+def z2z_decode_step(cb: Codebook, hidden: torch.Tensor, W_E: torch.Tensor, W_U: torch.Tensor,
+                    enc_E: EncoderWeights, enc_U: EncoderWeights, E_h: torch.Tensor,
+                    U_h: torch.Tensor, select: int, temperature: float, seed: int, step: int,
+                    forced: Optional[torch.Tensor], next_codes: torch.Tensor,
+                    selected: Optional[torch.Tensor], lse: Optional[torch.Tensor],
+                    new_entry: Optional[torch.Tensor] = None,
+                    E_h_f32: Optional[torch.Tensor] = None, U_h_f32: Optional[torch.Tensor] = None):
+    _check(lib().z2z_decode_step(cb.handle, _ptr(hidden), _ptr(W_E), _ptr(W_U), C.byref(enc_E),
+                                 C.byref(enc_U), _ptr(E_h), _ptr(U_h), C.c_int32(select),
+                                 C.c_float(temperature), C.c_uint64(seed), C.c_uint64(step),
+                                 _ptr(forced), _ptr(next_codes), _ptr(selected), _ptr(lse),
+                                 _ptr(new_entry), _ptr(E_h_f32), _ptr(U_h_f32), _stream()))
+
+
+def z2z_status(cb: Codebook):
+    """(status bits [B], hypertoken counts [B]) as host int32 tensors; waits for the stream."""
+    B = cb.cfg.B
+    st = torch.empty(B, dtype=torch.int32)
+    n = torch.empty(B, dtype=torch.int32)
+    _check(lib().z2z_status(cb.handle, _ptr(st), _ptr(n), _stream()))
+    return st, n
+
+
+def z2z_codebook_read(cb: Codebook, b: int):
+    """Codebook of sequence b on the host: (constituents [cap, M] int32, lengths [cap] int32)."""
+    cons = torch.empty(cb.cfg.cap, cb.cfg.M, dtype=torch.int32)
+    ln = torch.empty(cb.cfg.cap, dtype=torch.int32)
+    _check(lib().z2z_codebook_read(cb.handle, C.c_int32(b), _ptr(cons), _ptr(ln), _stream()))
+    return cons, ln

@@ -1,0 +1,73 @@
+// Internal launch wrappers shared between the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "z2z_common.cuh"
+
+namespace z2z {
+
+// ---- z2z_lzw.cu ------------------------------------------------------------------------------
+cudaError_t launch_codebook_clear(const CbView& cb, cudaStream_t s);
+cudaError_t launch_lzw_encode(const CbView& cb, const int32_t* tokens, const int32_t* lens,
+                              int T_max, int32_t* codes, int32_t* code_lens,
+                              int32_t* entries_after, cudaStream_t s);
+cudaError_t launch_lzw_step(const CbView& cb, const int32_t* new_codes, const uint8_t* active,
+                            int32_t* new_entry, cudaStream_t s);
+
+// ---- z2z_encoder.cu --------------------------------------------------------------------------
+// Work list of one encoder pass: up to `chunk` entries, entry e -> (sequence, entry number).
+struct EntryList {
+  int32_t* seq;       // [chunk]  sequence of entry e, -1 = unused slot
+  int32_t* idx;       // [chunk]  entry number within the sequence
+  int32_t* off;       // [B + 2]  exclusive prefix sum of per-sequence counts, then the total
+  int chunk;
+};
+struct EncoderArgs {
+  int d, dff, heads, layers, M;
+  int dtype;
+  const void* table;            // [V, d]
+  const void* const* w;         // host array of device pointers, ABI order
+  void* cache;                  // [B, cap, d] dtype
+  float* cache_f32;             // optional
+  float *X, *A, *QKV, *H;       // fp32 scratch, rows = chunk * M
+  __nv_bfloat16 *Ahl, *Hhl;     // bf16 hi/lo scratch for the tensor-core path
+  float* part;                  // split-K partial tiles
+  size_t part_bytes;
+};
+// Per-sequence ranges from (first, count) arrays, or "everything since the last call" when NULL.
+cudaError_t launch_entry_offsets(const CbView& cb, int which, const int32_t* first,
+                                 const int32_t* count, const EntryList& el, cudaStream_t s);
+// Ranges of the decode step: the entry created by this step's LZW update, if any.
+cudaError_t launch_entry_offsets_from_new(const CbView& cb, const int32_t* new_entry,
+                                          const EntryList& el, cudaStream_t s);
+cudaError_t launch_entry_fill(const CbView& cb, int which, const int32_t* first,
+                              const int32_t* new_entry, const EntryList& el, int chunk_index,
+                              cudaStream_t s);
+cudaError_t launch_mark_embedded(const CbView& cb, int which, cudaStream_t s);
+cudaError_t run_encoder_pass(const CbView& cb, const EncoderArgs& a, const EntryList& el,
+                             bool use_tensor_cores, cudaStream_t s);
+
+// ---- z2z_logits.cu ---------------------------------------------------------------------------
+struct LogitsArgs {
+  int d, dtype, N;
+  const void* hidden;           // [N, d]
+  const int32_t* row_seq;       // [N] or NULL
+  const int32_t* row_nvis;      // [N] or NULL
+  const void* WU;               // [V, d]
+  const void* Uh;               // [B, cap, d]
+  int select; float inv_temperature; uint64_t seed, step;
+  const int32_t* targets;
+  float* lse; int32_t* argmax; float* max_logit; int32_t* sample; float* target_logit;
+  float* logits_debug;
+  void* lpart; size_t lpart_bytes;
+  int row_base;                 // global index of row 0 of this launch (sampling counter)
+};
+cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, cudaStream_t s);
+
+// Selected code of the decode step: sample or argmax, overridden by `forced` when given.
+cudaError_t launch_pick_codes(int B, const int32_t* argmax, const int32_t* sample,
+                              const int32_t* forced, int32_t* next_codes, int32_t* selected,
+                              cudaStream_t s);
+
+}  // namespace z2z

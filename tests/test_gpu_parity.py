@@ -1,0 +1,378 @@
+"""GPU parity: the CUDA path (through the C ABI binding) against the CPU oracle, element by
+element, on the same seeded inputs.  Integer results are bit-exact; floats within the stated
+tolerance; selections follow the oracle except inside its top-2 gap."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lzw as olzw, logits as olg
+from paper_2506_01084_b200 import binding as zb
+from paper_2506_01084_b200 import synth_inputs as si
+from tests._harness import GAP, TOL, Pair, f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+# ------------------------------------------------------------------------------------------------
+# LZW: bit-exact
+# ------------------------------------------------------------------------------------------------
+class LzwOnly:
+    def __init__(self, V, M, cap, B):
+        self.V, self.M, self.cap, self.B = V, M, cap, B
+        self.cfg = zb.make_config(V, 8, M, cap, B, "fp32", 0, 1, 8)
+        self.cb = zb.Codebook(self.cfg, DEV)
+
+    def encode(self, tokens, lens=None):
+        B, T = tokens.shape
+        g_tok = torch.from_numpy(np.ascontiguousarray(tokens.astype(np.int32))).to(DEV)
+        g_lens = None if lens is None else torch.tensor(lens, dtype=torch.int32, device=DEV)
+        codes = torch.full((B, max(T, 1)), -7, dtype=torch.int32, device=DEV)
+        after = torch.full((B, max(T, 1)), -7, dtype=torch.int32, device=DEV)
+        clen = torch.zeros(B, dtype=torch.int32, device=DEV)
+        zb.z2z_lzw_encode(self.cb, g_tok, g_lens, codes, clen, after)
+        return codes.cpu().numpy(), clen.cpu().numpy(), after.cpu().numpy()
+
+    def entries(self, b):
+        cons, ln = zb.z2z_codebook_read(self.cb, b)
+        st, n = zb.z2z_status(self.cb)
+        return [tuple(int(x) for x in cons[k, :int(ln[k])]) for k in range(int(n[b]))], int(st[b])
+
+
+def _compare_encode(V, M, cap, tokens, lens=None):
+    B, T = tokens.shape
+    g = LzwOnly(V, M, cap, B)
+    codes, clen, after = g.encode(tokens, lens)
+    for b in range(B):
+        L = T if lens is None else lens[b]
+        want, waft, ob = olzw.encode(tokens[b, :L].tolist(), V, M, cap)
+        assert clen[b] == len(want)
+        assert codes[b, :clen[b]].tolist() == want
+        assert after[b, :clen[b]].tolist() == waft
+        ents, st = g.entries(b)
+        assert ents == ob.entries
+        assert st & ~zb.ST_CAP_FROZEN == 0
+        assert bool(st & zb.ST_CAP_FROZEN) == (len(ents) >= cap)
+    return g
+
+
+def test_lzw_worked_example():
+    path = os.path.join(os.path.dirname(__file__), "golden", "fig1_to_be_or_not_to_be.txt")
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, toks, codes, ents = [p.strip() for p in line.split("|")]
+        V, M, cap = map(int, head.split())
+        x = np.array([[int(t) for t in toks.split()]], dtype=np.int32)
+        g = LzwOnly(V, M, cap, 1)
+        got, clen, _ = g.encode(x)
+        assert got[0, :clen[0]].tolist() == [int(c) for c in codes.split()]
+        want_entries = [tuple(int(t) for t in e.split(":")[1].split(",")) for e in ents.split()]
+        assert g.entries(0)[0] == want_entries
+
+
+@pytest.mark.parametrize("name,T", [("tiny", None), ("phi3_mini_head", None),
+                                    ("llama3_8b_head", None), ("prefill_heavy", None),
+                                    ("long_context", None)])
+def test_lzw_encode_full_configs(name, T):
+    w = si.WORKLOADS[name]
+    tokens = si.make_tokens(w, 17)
+    _compare_encode(w.V, w.M, w.cap, tokens)
+
+
+def test_lzw_encode_ragged_empty_and_freeze():
+    w = si.WORKLOADS["tiny"].scaled(B=7, T=300)
+    tokens = si.make_tokens(w, 3)
+    lens = [0, 1, 2, 31, 32, 33, 300]
+    _compare_encode(w.V, 3, 256, tokens, lens)
+    _compare_encode(w.V, 3, 5, tokens, lens)          # freezes early
+    _compare_encode(w.V, 1, 256, tokens, lens)        # M = 1: identity coding
+    _compare_encode(w.V, 8, 256, tokens, lens)        # largest supported merge size
+    _compare_encode(w.V, 3, 0, tokens, lens)          # no hypertokens at all
+    rep = np.zeros((2, 500), dtype=np.int32); rep[1] = np.arange(500) % 3
+    _compare_encode(5, 8, 1000, rep)                  # heavy self-overlap (special-case ids)
+
+
+def test_lzw_brute_force_against_oracle():
+    for V, Tmax in ((2, 10), (3, 7)):
+        for T in range(1, Tmax + 1):
+            allx = np.array(list(itertools.product(range(V), repeat=T)), dtype=np.int32)
+            for s in range(0, len(allx), 1024):
+                chunk = allx[s:s + 1024]
+                for M in (2, 3):
+                    for cap in (1, 4, 64):
+                        _compare_encode(V, M, cap, chunk)
+
+
+def test_lzw_step_replay_equals_encode_and_rejects_bad_ids():
+    w = si.WORKLOADS["tiny"].scaled(B=5, T=200)
+    tokens = si.make_tokens(w, 9)
+    enc = [olzw.encode(tokens[b].tolist(), w.V, w.M, w.cap) for b in range(w.B)]
+    g = LzwOnly(w.V, w.M, w.cap, w.B)
+    steps = max(len(e[0]) for e in enc)
+    new_entry = torch.zeros(w.B, dtype=torch.int32, device=DEV)
+    replay = [olzw.Codebook(w.V, w.M, w.cap) for _ in range(w.B)]
+    for t in range(steps):
+        act = [1 if t < len(enc[b][0]) else 0 for b in range(w.B)]
+        z = [enc[b][0][t] if act[b] else 0 for b in range(w.B)]
+        zb.z2z_lzw_step(g.cb, torch.tensor(z, dtype=torch.int32, device=DEV),
+                        torch.tensor(act, dtype=torch.uint8, device=DEV), new_entry)
+        got = new_entry.cpu().tolist()
+        for b in range(w.B):
+            want = replay[b].step(z[b]) if act[b] else -1
+            assert got[b] == want
+    for b in range(w.B):
+        ents, st = g.entries(b)
+        assert ents == enc[b][2].entries and st == 0
+    # ids that name nothing: state untouched, BAD_TOKEN raised (consistent vocabulary updates)
+    st0, n0 = zb.z2z_status(g.cb)
+    bad = [w.V + int(n0[b]) + 1 for b in range(w.B)]
+    bad[1] = -3
+    zb.z2z_lzw_step(g.cb, torch.tensor(bad, dtype=torch.int32, device=DEV), None, new_entry)
+    st1, n1 = zb.z2z_status(g.cb)
+    assert torch.equal(n0, n1) and all(int(s) & zb.ST_BAD_TOKEN for s in st1)
+    assert new_entry.cpu().tolist() == [-1] * w.B
+    for b in range(w.B):
+        assert g.entries(b)[0] == enc[b][2].entries
+    # and the next legal code behaves as if the bad one had never been sent
+    z = [int(tokens[b, 0]) for b in range(w.B)]
+    zb.z2z_lzw_step(g.cb, torch.tensor(z, dtype=torch.int32, device=DEV), None, new_entry)
+    for b in range(w.B):
+        assert new_entry.cpu().tolist()[b] == replay[b].step(z[b])
+
+
+def test_lzw_step_special_case_id():
+    g = LzwOnly(2, 3, 16, 1)
+    ne = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ob = olzw.Codebook(2, 3, 16)
+    for z in [0, 2, 3, 0, 4]:      # 2 and 3 are created by the step that receives them
+        zb.z2z_lzw_step(g.cb, torch.tensor([z], dtype=torch.int32, device=DEV), None, ne)
+        assert ne.item() == ob.step(z)
+        ents, st = g.entries(0)
+        assert ents == ob.entries and st == ob.status
+
+
+# ------------------------------------------------------------------------------------------------
+# Hyper-encoder
+# ------------------------------------------------------------------------------------------------
+SMALL_BF16 = si.Workload("small_bf16", V=1000, d=256, dtype="bf16", B=3, T=160, M=4, cap=96,
+                         zipf_s=1.1, copy_p=0.4, seg_min=3, seg_max=12, steps=12, enc_layers=2,
+                         enc_heads=2, enc_dff=512)
+SMALL_FP32 = SMALL_BF16.scaled(name="small_fp32", dtype="fp32", d=72, enc_heads=3, enc_dff=200,
+                               M=5)
+
+
+def _prefill_both(p: Pair):
+    w = p.w
+    codes, clen, after = p.gpu_encode()
+    ocodes, oafter = p.oracle.prefill([p.tokens[b].tolist() for b in range(w.B)])
+    for b in range(w.B):
+        assert codes[b, :clen[b]].tolist() == ocodes[b]
+        assert after[b, :clen[b]].tolist() == oafter[b]
+    p.check_codebooks()
+    total = sum(bk.n() for bk in p.oracle.books)
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, total, p.E_h, p.E_f32)
+    if not w.tied:
+        zb.z2z_hyper_embed(p.cb, zb.CACHE_UNEMBED, p.g_WU, p.g_encU, None, None, total, p.U_h,
+                           p.U_f32)
+    worst = 0.0
+    for b in range(w.B):
+        worst = max(worst, p.check_cache_rows(b, 0, p.oracle.books[b].n()))
+    return ocodes, worst
+
+
+@pytest.mark.parametrize("w", [si.WORKLOADS["tiny"], SMALL_BF16, SMALL_FP32,
+                               SMALL_BF16.scaled(name="avg", enc_layers=0),
+                               SMALL_BF16.scaled(name="one_layer", enc_layers=1),
+                               SMALL_BF16.scaled(name="tied", tied=1)],
+                         ids=lambda w: w.name)
+def test_hyper_embed_all_prefill_entries(w):
+    p = Pair(w, seed=5)
+    _, worst = _prefill_both(p)
+    print(f"{w.name}: max |hyper-embedding error| = {worst:.3e}")
+    # rows beyond n_b were not touched
+    for b in range(w.B):
+        n = p.oracle.books[b].n()
+        assert float(p.E_h[b, n:].abs().max().item() if n < w.cap else 0.0) == 0.0
+    if w.dtype == "fp32":
+        for b in range(w.B):
+            assert p.check_cache_rows(b, 0, p.oracle.books[b].n(), tol=2e-5) <= 2e-5
+
+
+def test_hyper_embed_explicit_ranges_and_incremental():
+    w = SMALL_BF16
+    p = Pair(w, seed=6)
+    p.gpu_encode()
+    p.oracle.prefill([p.tokens[b].tolist() for b in range(w.B)])
+    n = [bk.n() for bk in p.oracle.books]
+    first = [0, min(5, n[1]), n[2]]
+    count = [min(3, n[0]), max(0, n[1] - 5), 0]
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE,
+                       torch.tensor(first, dtype=torch.int32, device=DEV),
+                       torch.tensor(count, dtype=torch.int32, device=DEV), sum(count), p.E_h, p.E_f32)
+    got = p.E_f32.cpu().double().numpy()
+    for b in range(w.B):
+        lo, hi = first[b], first[b] + count[b]
+        if hi > lo:
+            assert np.abs(got[b, lo:hi] - p.oracle.E_exact[b][lo:hi]).max() <= TOL
+        assert np.all(got[b, :lo] == 0) and np.all(got[b, hi:] == 0)
+    # NULL ranges after that: "everything since the last NULL call" = all entries
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, 0, p.E_h, p.E_f32)
+    got = p.E_f32.cpu().double().numpy()
+    for b in range(w.B):
+        assert np.abs(got[b, :n[b]] - p.oracle.E_exact[b]).max() <= TOL
+
+
+# ------------------------------------------------------------------------------------------------
+# Joint logits and reductions
+# ------------------------------------------------------------------------------------------------
+def _logits_case(w, seed, rows_per_seq, causal, select, temperature=0.8):
+    p = Pair(w, seed=seed, generic_encoder=False)
+    codes, clen, after = p.gpu_encode()
+    ocodes, oafter = p.oracle.prefill([p.tokens[b].tolist() for b in range(w.B)])
+    n = [bk.n() for bk in p.oracle.books]
+    # synthetic hyper-unembedding rows straight from the generator (same values on both sides)
+    U = si.normal_tensor((w.B, max(w.cap, 1), w.d), 0.05, seed + 100, w.torch_dtype)
+    p.U_h.copy_(U.to(p.dev))
+    U64 = f64(U)
+    rng = np.random.default_rng(seed)
+    row_seq, row_nvis = [], []
+    for b in range(w.B):
+        for _ in range(rows_per_seq[b]):
+            row_seq.append(b)
+            row_nvis.append(int(rng.integers(0, n[b] + 1)) if causal else n[b])
+    N = len(row_seq)
+    hid = si.make_hidden(w, N, seed)
+    targets = [int(rng.integers(0, w.V + w.cap)) for _ in range(N)]
+    g_hid = hid.to(p.dev)
+    out = {k: torch.zeros(N, dtype=torch.float32, device=p.dev) for k in ("lse", "max", "tl")}
+    am = torch.zeros(N, dtype=torch.int32, device=p.dev)
+    smp = torch.zeros(N, dtype=torch.int32, device=p.dev)
+    dbg = torch.full((N, w.V + w.cap), float("nan"), dtype=torch.float32, device=p.dev)
+    zb.z2z_dynamic_logits(p.cb, g_hid, torch.tensor(row_seq, dtype=torch.int32, device=p.dev),
+                          torch.tensor(row_nvis, dtype=torch.int32, device=p.dev) if causal else None,
+                          p.g_WU, p.U_h, select, temperature, 0xABCDEF12345, 77,
+                          torch.tensor(targets, dtype=torch.int32, device=p.dev),
+                          out["lse"], am, out["max"], smp if select else None, out["tl"], dbg)
+    dbg = dbg.cpu().double().numpy()
+    lse, mx, tl = (out[k].cpu().double().numpy() for k in ("lse", "max", "tl"))
+    am, smp = am.cpu().numpy(), smp.cpu().numpy()
+    H = f64(hid)
+    worst = 0.0
+    for r in range(N):
+        b, nv = row_seq[r], row_nvis[r]
+        l = olg.joint_logits(H[r], p.oracle.W_U, U64[b, :nv])
+        got = dbg[r, :w.V + nv]
+        err = np.abs(got - l).max()
+        worst = max(worst, err)
+        assert err <= TOL
+        assert np.all(np.isnan(dbg[r, w.V + nv:]))            # invisible columns never computed
+        assert abs(lse[r] - olg.lse(l)) <= TOL
+        a, best, gap = olg.top2(l)
+        assert abs(mx[r] - best) <= TOL
+        if am[r] != a:
+            assert gap < GAP and l[am[r]] >= best - GAP
+        if targets[r] < w.V + nv:
+            assert abs(tl[r] - l[targets[r]]) <= TOL
+        else:
+            assert np.isnan(tl[r])
+        if select:
+            ch, scores, sgap = olg.select(l, 1, temperature, 0xABCDEF12345, 77, r)
+            if smp[r] != ch:
+                assert sgap < GAP and scores[smp[r]] >= scores[ch] - GAP
+    return worst
+
+
+@pytest.mark.parametrize("w", [si.WORKLOADS["tiny"].scaled(B=2), SMALL_BF16, SMALL_FP32],
+                         ids=lambda w: w.name)
+@pytest.mark.parametrize("causal,select", [(False, 0), (True, 1)])
+def test_dynamic_logits_elementwise(w, causal, select):
+    rows = [1] * w.B if not causal else [70, 0, 5][:w.B] + [3] * max(0, w.B - 3)
+    worst = _logits_case(w, 11, rows, causal, select)
+    print(f"{w.name}: max |logit error| = {worst:.3e}")
+
+
+def test_dynamic_logits_no_hypertokens_is_plain_lm_head():
+    w = SMALL_BF16.scaled(cap=0, name="nocap")
+    worst = _logits_case(w, 12, [2, 1, 1], False, 0)
+    assert worst <= TOL
+
+
+# ------------------------------------------------------------------------------------------------
+# Whole decode step, following the GPU's selections inside the oracle's top-2 gap
+# ------------------------------------------------------------------------------------------------
+def _decode_follow(w, seed, select, steps=None, forced_every=0):
+    p = Pair(w, seed=seed)
+    _prefill_both(p)
+    for b in range(w.B):
+        p.force_caches_from_oracle(b, 0, p.oracle.books[b].n())
+    steps = w.steps if steps is None else steps
+    hid = si.make_hidden(w, steps * w.B, seed + 1).view(steps, w.B, w.d)
+    H = f64(hid)
+    g_hid = hid.to(p.dev)
+    nxt = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    sel = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    lse = torch.zeros(w.B, dtype=torch.float32, device=p.dev)
+    new = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    followed = 0
+    worst_lse = 0.0
+    rng = np.random.default_rng(seed)
+    for t in range(steps):
+        n0 = [bk.n() for bk in p.oracle.books]
+        forced = None
+        if forced_every and t % forced_every == forced_every - 1:
+            forced = [int(rng.integers(0, w.V + n0[b] + 1)) if p.oracle.books[b].prev is not None
+                      else int(rng.integers(0, w.V)) for b in range(w.B)]
+            # an id equal to V + n is legal only in the special case; keep forced ids existing
+            forced = [min(z, w.V + n0[b] - 1) if n0[b] else min(z, w.V - 1)
+                      for b, z in enumerate(forced)]
+        zb.z2z_decode_step(p.cb, g_hid[t], p.g_WE, p.g_WU, p.g_encE, p.g_encU, p.E_h, p.U_h,
+                           select, 0.9, 4242, t,
+                           None if forced is None else torch.tensor(forced, dtype=torch.int32,
+                                                                    device=p.dev),
+                           nxt, sel, lse, new, p.E_f32, p.U_f32)
+        g_sel, g_nxt, g_lse, g_new = (x.cpu().numpy() for x in (sel, nxt, lse, new))
+        sc = p.oracle.score(H[t], select, 0.9, 4242, t)
+        apply = []
+        for b in range(w.B):
+            assert abs(g_lse[b] - sc[b]["lse"]) <= TOL, (t, b, g_lse[b], sc[b]["lse"])
+            worst_lse = max(worst_lse, abs(g_lse[b] - sc[b]["lse"]))
+            assert 0 <= g_sel[b] < w.V + n0[b]
+            if g_sel[b] != sc[b]["choice"]:
+                s = sc[b]["scores"]
+                assert sc[b]["gap"] < GAP and s[g_sel[b]] >= s[sc[b]["choice"]] - GAP, \
+                    (t, b, g_sel[b], sc[b]["choice"], sc[b]["gap"])
+                followed += 1
+            want_next = forced[b] if forced is not None else int(g_sel[b])
+            assert g_nxt[b] == want_next
+            apply.append(want_next)
+        onew = p.oracle.advance(apply)
+        assert g_new.tolist() == onew, (t, g_new.tolist(), onew)
+        for b in range(w.B):
+            if onew[b] >= 0:
+                p.check_cache_rows(b, onew[b], onew[b] + 1)
+                p.force_caches_from_oracle(b, onew[b], onew[b] + 1)
+        st, n = zb.z2z_status(p.cb)
+        assert n.tolist() == [bk.n() for bk in p.oracle.books]
+    p.check_codebooks()
+    return followed, worst_lse
+
+
+def test_decode_step_tiny_config_argmax():
+    followed, worst = _decode_follow(si.WORKLOADS["tiny"], 21, zb.SELECT_ARGMAX)
+    print(f"tiny: followed {followed} near-ties, worst |LSE error| {worst:.2e}")
+
+
+def test_decode_step_tiny_config_sampling_and_forcing():
+    _decode_follow(si.WORKLOADS["tiny"], 22, zb.SELECT_GUMBEL, forced_every=3)
+
+
+@pytest.mark.parametrize("w", [SMALL_BF16, SMALL_FP32, SMALL_BF16.scaled(name="tied", tied=1)],
+                         ids=lambda w: w.name)
+def test_decode_step_small(w):
+    _decode_follow(w, 23, zb.SELECT_ARGMAX, steps=w.steps)
+    _decode_follow(w, 24, zb.SELECT_GUMBEL, steps=6, forced_every=2)

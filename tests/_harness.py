@@ -76,7 +76,7 @@ class Pair:
             for k in range(n):
                 assert np.all(cons[k, int(ln[k]):] == -1)
             assert (st & ~zb.ST_CAP_FROZEN) == (ob.status & ~1), (b, st, ob.status)
-            assert bool(st & zb.ST_CAP_FROZEN) == (n >= self.w.cap)
+            assert bool(st & zb.ST_CAP_FROZEN) == (n >= self.w.cap > 0)
 
     def force_caches_from_oracle(self, b, lo, hi):
         """Overwrite GPU cache rows [lo, hi) of sequence b with the oracle's stored rows."""

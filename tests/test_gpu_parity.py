@@ -55,7 +55,7 @@ def _compare_encode(V, M, cap, tokens, lens=None):
         ents, st = g.entries(b)
         assert ents == ob.entries
         assert st & ~zb.ST_CAP_FROZEN == 0
-        assert bool(st & zb.ST_CAP_FROZEN) == (len(ents) >= cap)
+        assert bool(st & zb.ST_CAP_FROZEN) == (len(ents) >= cap > 0)
     return g
 
 

@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the dynamic-vocabulary decode step (LZW update + hyper-encoder + joint logits).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one z2z_decode_step over a batch of B sequences of the workload (default: the
+Phi-3-mini-shaped head, the configuration the headline metric is quoted on): joint logits and
+selection, online LZW update with the selected code, hyper-encoder on the new entry of each
+sequence for both caches.  The prompts are compressed and their entries embedded before the timed
+region (session set-up).  Prints ONE JSON line.
+
+`--impl reference` times the CPU oracle (oracle/) as it stands on the host cores, on a bounded
+sample of the same workload.  With N > 1 ranks each rank runs an independent replica of the
+workload (the path has no exchange step); the value is the sum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2506_01084_b200 import synth_inputs as si  # noqa: E402
+
+METRIC = "base-token-equiv decode tok/s (LZW+hyper-embed+logits)"
+UNIT = "base tokens/s"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return {"hbm_gbs": float(j["hbm_gbs"]), "bf16_tflops": float(j["bf16_tflops"]),
+                "bf16_tflops_sustained": float(j.get("bf16_tflops_sustained", j["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [s for s in sm if s > 0]
+        return {"sm_mhz": float(np.median(busy)) if busy else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------------
+# algorithmic bytes of one decode step (what the kernels must move at minimum)
+# --------------------------------------------------------------------------------------------------
+def logits_bytes(w: si.Workload, n_hyper_total: int) -> float:
+    """W_U once + every visible hyper-unembedding row once + hidden rows (bf16 = 2 B)."""
+    es = 2 if w.dtype == "bf16" else 4
+    return es * (w.V * w.d + n_hyper_total * w.d + w.B * w.d)
+
+
+def encoder_gemm_bytes(w: si.Workload) -> float:
+    """Linear-layer weights of both hyper-encoders, each streamed once per step."""
+    es = 2 if w.dtype == "bf16" else 4
+    per_layer = 4 * w.d * w.d + 2 * w.d * w.dff
+    return es * per_layer * w.enc_layers * (1 if w.tied else 2)
+
+
+# --------------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------------
+def run_ours(args, rank: int, world: int):
+    from paper_2506_01084_b200 import binding as zb
+    zb.lib()                                  # fail loudly if the CUDA library is missing
+    dev = torch.device(f"cuda:{int(os.environ.get('LOCAL_RANK', 0))}")
+    torch.cuda.set_device(dev)
+    w = si.WORKLOADS[args.workload]
+    if w.steps == 0:
+        raise SystemExit("this workload has no decode steps; use tests for the prefill path")
+    K, Wm = args.steps, args.warmup
+    seed = 1000 + rank
+    tokens = si.make_tokens(w, seed)
+    W_E, W_U = si.make_tables(w, seed)
+    encE_t = [t.to(dev) for t in si.make_encoder(w, seed * 3 + 1)]
+    encU_t = encE_t if w.tied else [t.to(dev) for t in si.make_encoder(w, seed * 3 + 2)]
+    g_WE = W_E.to(dev)
+    g_WU = g_WE if w.tied else W_U.to(dev)
+    cfg = zb.make_config(w.V, w.d, w.M, w.cap, w.B, w.dtype, w.enc_layers, w.heads, w.dff, w.tied)
+    cb = zb.Codebook(cfg, dev)
+    encE, encU = zb.encoder_weights(encE_t), zb.encoder_weights(encU_t)
+    E_h = torch.zeros(w.B, w.cap, w.d, dtype=w.torch_dtype, device=dev)
+    U_h = E_h if w.tied else torch.zeros_like(E_h)
+    n_steps_total = Wm + 3 * K                # warm-up, device-timed, per-kernel-timed, end-to-end
+    hidden_host = si.make_hidden(w, n_steps_total * w.B, seed).view(n_steps_total, w.B, w.d).pin_memory()
+    hidden = hidden_host.to(dev)
+
+    # ---- session set-up (not timed as steps; reported separately) ----
+    g_tok = torch.from_numpy(tokens).to(dev)
+    codes = torch.zeros(w.B, w.T, dtype=torch.int32, device=dev)
+    clen = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    zb.z2z_lzw_encode(cb, g_tok, None, codes, clen, None)
+    ev[1].record()
+    zb.z2z_hyper_embed(cb, zb.CACHE_EMBED, g_WE, encE, None, None, w.B * w.T, E_h, None)
+    if not w.tied:
+        zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, w.B * w.T, U_h, None)
+    ev[2].record()
+    torch.cuda.synchronize()
+    st, n0 = zb.z2z_status(cb)
+    prefill = {"lzw_encode_ms": ev[0].elapsed_time(ev[1]), "hyper_embed_all_ms": ev[1].elapsed_time(ev[2]),
+               "prompt_tokens": int(w.B * w.T), "compressed_tokens": int(clen.sum().item()),
+               "hypertokens": int(n0.sum().item())}
+
+    nxt_all = torch.zeros(n_steps_total, w.B, dtype=torch.int32, device=dev)
+    lse = torch.zeros(w.B, dtype=torch.float32, device=dev)
+
+    def step(t, hid):
+        zb.z2z_decode_step(cb, hid, g_WE, g_WU, encE, encU, E_h, U_h, zb.SELECT_ARGMAX, 1.0, 0, t,
+                           None, nxt_all[t], None, lse)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(Wm):
+        step(t, hidden[t])
+    zb.z2z_profile_read(cb)                    # reset launch counters
+
+    # ---- device-timed region: inputs resident in HBM ----
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    barrier()
+    n_before = zb.z2z_status(cb)[1].sum().item()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for t in range(Wm, Wm + K):
+        step(t, hidden[t])
+    e1.record()
+    barrier()
+    dev_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    _, launches = zb.z2z_profile_read(cb)
+    n_after = zb.z2z_status(cb)[1].sum().item()
+
+    # ---- same K steps again with per-kernel-class events (for the roofline numbers) ----
+    zb.z2z_profile(cb, True)
+    for t in range(Wm + K, Wm + 2 * K):
+        step(t, hidden[t])
+    zb.z2z_profile(cb, False)
+    cls_ms, cls_launches = zb.z2z_profile_read(cb)
+    n_after2 = zb.z2z_status(cb)[1].sum().item()
+
+    # ---- end to end: host buffers, H2D of the hidden rows and D2H of the results every step ----
+    out_host = torch.zeros(w.B, dtype=torch.int32).pin_memory()
+    lse_host = torch.zeros(w.B, dtype=torch.float32).pin_memory()
+    hid_dev = torch.empty(w.B, w.d, dtype=w.torch_dtype, device=dev)
+    barrier()
+    t0 = time.perf_counter()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for t in range(Wm + 2 * K, Wm + 3 * K):
+        hid_dev.copy_(hidden_host[t], non_blocking=True)
+        step(t, hid_dev)
+        out_host.copy_(nxt_all[t], non_blocking=True)
+        lse_host.copy_(lse, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller needs the token to go on
+    e3.record()
+    barrier()
+    e2e_ms = max(e2.elapsed_time(e3), (time.perf_counter() - t0) * 1e3)
+
+    # ---- base-token equivalents of what was emitted ----
+    stt, n_fin = zb.z2z_status(cb)
+    lens = []
+    for b in range(w.B):
+        _, ln = zb.z2z_codebook_read(cb, b)
+        lens.append(ln.numpy())
+    nx = nxt_all.cpu().numpy()
+
+    def base_tokens(lo, hi):
+        tot = 0
+        for b in range(w.B):
+            z = nx[lo:hi, b]
+            tot += int(np.where(z < w.V, 1, lens[b][np.clip(z - w.V, 0, w.cap - 1)]).sum())
+        return tot
+
+    bt_dev = base_tokens(Wm, Wm + K)
+    bt_e2e = base_tokens(Wm + 2 * K, Wm + 3 * K)
+    bad = int(sum(1 for s in stt.tolist() if s & (zb.ST_BAD_TOKEN | zb.ST_TABLE_FULL | zb.ST_WAIT_TIMEOUT)))
+
+    # ---- reduce over ranks: max time, summed tokens ----
+    if world > 1:
+        tt = torch.tensor([dev_ms, e2e_ms], device=dev)
+        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
+        dev_ms, e2e_ms = tt.tolist()
+        cc = torch.tensor([bt_dev, bt_e2e], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(cc)
+        bt_dev, bt_e2e = cc.tolist()
+
+    pk = peaks()
+    # dominant kernel class by measured time
+    mean_hyper = 0.5 * (n_after + n_after2)     # hyper rows visible during the profiled pass
+    classes = {"logits": logits_bytes(w, mean_hyper), "encoder_gemm": encoder_gemm_bytes(w)}
+    dom = max(classes, key=lambda k: cls_ms.get(k, 0.0))
+    per_launch_group_ms = cls_ms[dom] / K       # time of that class per step
+    achieved = classes[dom] / (per_launch_group_ms * 1e-3) / 1e9 if per_launch_group_ms > 0 else 0.0
+    roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": pk["hbm_gbs"],
+            "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "traffic": None,
+            "peak_source": pk["source"],
+            "algorithmic_bytes_per_step": classes[dom], "ms_per_step": per_launch_group_ms,
+            "launches_per_step": cls_launches[dom] / K,
+            "timing": "CUDA events around each launch of the class, second pass of K steps",
+            "per_class_ms_per_step": {k: v / K for k, v in cls_ms.items()},
+            "logits": {"bytes": classes["logits"], "ms": cls_ms["logits"] / K,
+                       "gbs": classes["logits"] / max(cls_ms["logits"] / K, 1e-9) / 1e6,
+                       "frac": classes["logits"] / max(cls_ms["logits"] / K, 1e-9) / 1e6 / pk["hbm_gbs"]},
+            "encoder_gemm": {"bytes": classes["encoder_gemm"], "ms": cls_ms["encoder_gemm"] / K,
+                             "gbs": classes["encoder_gemm"] / max(cls_ms["encoder_gemm"] / K, 1e-9) / 1e6,
+                             "frac": classes["encoder_gemm"] / max(cls_ms["encoder_gemm"] / K, 1e-9) / 1e6 / pk["hbm_gbs"]}}
+    es = 2 if w.dtype == "bf16" else 4
+    line = {
+        "metric": METRIC, "value": bt_dev / (dev_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": Wm, "ms_per_step": dev_ms / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "prompt_tokens": w.T,
+                   "M": w.M, "cap": w.cap, "enc_layers": w.enc_layers, "enc_dff": w.dff,
+                   "select": "argmax, free-running", "replicas": world,
+                   "l2": "per-step inputs (W_U and both encoders' weights) exceed the 126 MB L2"},
+        "steps_per_s": K / (dev_ms * 1e-3),
+        "mean_phrase_len": bt_dev / (K * w.B * world),
+        "new_entries_in_timed_region": int(n_after - n_before),
+        "status_errors": bad,
+        "prefill": prefill,
+        "e2e": {"value": bt_e2e / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / K,
+                "h2d_bytes_per_step": int(w.B * w.d * es), "d2h_bytes_per_step": int(w.B * 8)},
+        "gpu_launches": int(sum(launches.values())),
+        "gpu_launches_by_class": launches,
+        "clocks": clocks,
+        "roofline": roof,
+    }
+    return line, w
+
+
+# --------------------------------------------------------------------------------------------------
+# oracle on the host cores (cpu_baseline of our arm, and the whole `--impl reference` arm)
+# --------------------------------------------------------------------------------------------------
+def oracle_sample(w: si.Workload, n_steps: int, seed: int = 1000, prompt_tokens: int = 256):
+    """Times `n_steps` decode steps of the oracle session on the workload's shapes.
+
+    Bounded sample: prompts are cut to `prompt_tokens` tokens so that embedding their entries in
+    fp64 stays within seconds; V, d, B, M, the encoder and the per-step work (joint logits over
+    V + n_b columns, LZW update, both encoders on the new entries) are the workload's own.
+    """
+    from oracle import decode_step as ods
+    torch.set_num_threads(os.cpu_count() or 1)
+    T = min(w.T, prompt_tokens)
+    tokens = si.make_tokens(w, seed, T=T)
+    W_E, W_U = si.make_tables(w, seed)
+    f = lambda t: t.double().numpy()
+    encE = [f(t) for t in si.make_encoder(w, seed * 3 + 1)]
+    encU = encE if w.tied else [f(t) for t in si.make_encoder(w, seed * 3 + 2)]
+    s = ods.Session(w.V, w.M, w.cap, w.B, w.heads, w.dtype, f(W_E), f(W_E) if w.tied else f(W_U),
+                    encE, encU)
+    t0 = time.perf_counter()
+    s.prefill([tokens[b].tolist() for b in range(w.B)])
+    t_prefill = time.perf_counter() - t0
+    hid = si.make_hidden(w, n_steps * w.B, seed).double().numpy().reshape(n_steps, w.B, w.d)
+    base = 0
+    t0 = time.perf_counter()
+    for t in range(n_steps):
+        sc, _ = s.step(hid[t], 0, 1.0, 0, t)
+        base += sum(len(s.books[b].phrase(sc[b]["choice"])) for b in range(w.B))
+    dt = time.perf_counter() - t0
+    return {"value": base / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+            "threads": torch.get_num_threads(),
+            "sample": f"{n_steps} decode steps of the full-shape workload (V, d, B, M, encoder as "
+                      f"configured) after prompts cut to {T} tokens; oracle prefill took "
+                      f"{t_prefill:.1f} s",
+            "seconds": dt, "ms_per_step": dt / n_steps * 1e3}
+
+
+def run_reference(args):
+    w = si.WORKLOADS[args.workload]
+    K = max(1, args.steps)
+    per_step = 1 if w.d >= 2048 else 4
+    res = oracle_sample(w, n_steps=max(1, min(K, 6)) * per_step)
+    line = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT,
+            "n_gpus": args.gpus, "steps": K, "warmup": args.warmup,
+            "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "M": w.M, "cap": w.cap},
+            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="phi3_mini_head", choices=list(si.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args)
+        return
+    if world > 1:
+        torch.distributed.init_process_group("nccl")
+    line, w = run_ours(args, rank, world)
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            res = oracle_sample(w, n_steps=2 if w.d >= 2048 else 16)
+            line["cpu_baseline"] = {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

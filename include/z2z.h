@@ -165,6 +165,18 @@ int32_t z2z_status(z2z_codebook* cb, int32_t* h_status, int32_t* h_n, z2z_stream
 int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t* h_len,
                           z2z_stream stream);
 
+/* Launch accounting and per-kernel-class timing (no counterpart in the paper; measurement aid).
+ * The library always counts the kernels it launches, per class:
+ *   0 joint-logits main kernel, 1 logits merge / selection, 2 LZW kernels,
+ *   3 hyper-encoder linear layers, 4 other hyper-encoder kernels and work lists.
+ * z2z_profile(cb, 1) additionally brackets every launch group with CUDA events on the caller's
+ * stream until z2z_profile(cb, 0).  z2z_profile_read waits for the stream, returns the summed
+ * event time in milliseconds (h_ms, may be NULL) and the launch counts (h_launches, may be NULL)
+ * for the first n_classes classes, and resets both.                                           */
+int32_t z2z_profile(z2z_codebook* cb, int32_t enable);
+int32_t z2z_profile_read(z2z_codebook* cb, int32_t n_classes, double* h_ms, int64_t* h_launches,
+                         z2z_stream stream);
+
 /* Frees the host handle (never the workspace). */
 int32_t z2z_codebook_destroy(z2z_codebook* cb);
 

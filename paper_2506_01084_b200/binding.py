@@ -23,7 +23,8 @@ CACHE_EMBED, CACHE_UNEMBED = 0, 1
 
 EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lzw_step",
            "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
-           "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error"]
+           "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error", "z2z_profile",
+           "z2z_profile_read"]
 
 
 class Config(C.Structure):
@@ -191,3 +192,20 @@ def z2z_codebook_read(cb: Codebook, b: int):
     ln = torch.empty(cb.cfg.cap, dtype=torch.int32)
     _check(lib().z2z_codebook_read(cb.handle, C.c_int32(b), _ptr(cons), _ptr(ln), _stream()))
     return cons, ln
+
+
+PROFILE_CLASSES = ["logits", "logits_merge", "lzw", "encoder_gemm", "encoder_other"]
+
+
+def z2z_profile(cb: Codebook, enable: bool):
+    _check(lib().z2z_profile(cb.handle, C.c_int32(1 if enable else 0)))
+
+
+def z2z_profile_read(cb: Codebook):
+    """({class: milliseconds}, {class: launches}) since the last read; waits for the stream."""
+    n = len(PROFILE_CLASSES)
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    _check(lib().z2z_profile_read(cb.handle, C.c_int32(n), ms, cnt, _stream()))
+    return ({k: ms[i] for i, k in enumerate(PROFILE_CLASSES)},
+            {k: int(cnt[i]) for i, k in enumerate(PROFILE_CLASSES)})

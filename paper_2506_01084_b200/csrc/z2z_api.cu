@@ -15,6 +15,7 @@ struct z2z_codebook {
   z2z::CbView view;
   int dff, heads;
   int use_tensor_cores;
+  z2z::Prof prof;
 };
 
 namespace {
@@ -105,7 +106,7 @@ int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s) {
     if (a.target_logit) c.target_logit = a.target_logit + r0;
     if (a.logits_debug) c.logits_debug = a.logits_debug + (size_t)r0 * ldbg;
     if (a.row_seq == nullptr && r0 > 0) return fail(Z2Z_ERR_INVALID_ARG, "d_row_seq is required when N > B");
-    Z2Z_CUDA(z2z::run_logits_simt(cb->view, c, s), "logits");
+    Z2Z_CUDA(z2z::run_logits_simt(cb->view, c, &cb->prof, s), "logits");
   }
   return Z2Z_OK;
 }
@@ -154,6 +155,7 @@ int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, 
   v.status = reinterpret_cast<int32_t*>(h->ws + plan.off_status);
   v.n_emb = reinterpret_cast<int32_t*>(h->ws + plan.off_n_emb);
   *cb = h;
+  z2z::ProfScope ps(&h->prof, z2z::kProfLzw, 1, reinterpret_cast<cudaStream_t>(stream));
   Z2Z_CUDA(z2z::launch_codebook_clear(v, reinterpret_cast<cudaStream_t>(stream)), "codebook_init");
   return Z2Z_OK;
 }
@@ -165,6 +167,7 @@ int32_t z2z_lzw_encode(z2z_codebook* cb, const int32_t* d_tokens, const int32_t*
   if (T_max < 0) return fail(Z2Z_ERR_INVALID_ARG, "T_max < 0");
   if (!d_code_lens) return fail(Z2Z_ERR_INVALID_ARG, "d_code_lens is NULL");
   if (T_max > 0 && (!d_tokens || !d_codes)) return fail(Z2Z_ERR_INVALID_ARG, "d_tokens / d_codes is NULL");
+  z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, reinterpret_cast<cudaStream_t>(stream));
   Z2Z_CUDA(z2z::launch_lzw_encode(cb->view, d_tokens, d_lens, T_max, d_codes, d_code_lens,
                                   d_entries_after, reinterpret_cast<cudaStream_t>(stream)),
            "lzw_encode");
@@ -175,6 +178,7 @@ int32_t z2z_lzw_step(z2z_codebook* cb, const int32_t* d_new_codes, const uint8_t
                      int32_t* d_new_entry, z2z_stream stream) {
   if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
   if (!d_new_codes) return fail(Z2Z_ERR_INVALID_ARG, "d_new_codes is NULL");
+  z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, reinterpret_cast<cudaStream_t>(stream));
   Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_new_codes, d_active, d_new_entry,
                                 reinterpret_cast<cudaStream_t>(stream)), "lzw_step");
   return Z2Z_OK;
@@ -197,12 +201,21 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
   long long bound = (long long)cb->cfg.B * cb->cfg.cap;
   if (max_entries > 0 && max_entries < bound) bound = max_entries;
   const int n_chunks = (int)((bound + el.chunk - 1) / el.chunk);
-  Z2Z_CUDA(z2z::launch_entry_offsets(cb->view, which, d_first, d_count, el, s), "hyper_embed");
-  for (int c = 0; c < n_chunks; ++c) {
-    Z2Z_CUDA(z2z::launch_entry_fill(cb->view, which, d_first, nullptr, el, c, s), "hyper_embed");
-    Z2Z_CUDA(z2z::run_encoder_pass(cb->view, a, el, cb->use_tensor_cores != 0, s), "hyper_embed");
+  {
+    z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
+    Z2Z_CUDA(z2z::launch_entry_offsets(cb->view, which, d_first, d_count, el, s), "hyper_embed");
   }
-  if (!d_first) Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, which, s), "hyper_embed");
+  for (int c = 0; c < n_chunks; ++c) {
+    {
+      z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
+      Z2Z_CUDA(z2z::launch_entry_fill(cb->view, which, d_first, nullptr, el, c, s), "hyper_embed");
+    }
+    Z2Z_CUDA(z2z::run_encoder_pass(cb->view, a, el, cb->use_tensor_cores != 0, &cb->prof, s), "hyper_embed");
+  }
+  if (!d_first) {
+    z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
+    Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, which, s), "hyper_embed");
+  }
   return Z2Z_OK;
 }
 
@@ -270,20 +283,30 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
   a.lpart = cb->ws + cb->plan.off_lpart; a.lpart_bytes = cb->plan.lpart_bytes;
   rc = logits_call(cb, a, s);
   if (rc) return rc;
-  Z2Z_CUDA(z2z::launch_pick_codes(B, w_argmax, a.sample, d_forced, d_next_codes, d_selected, s), "decode_step");
+  {
+    z2z::ProfScope ps(&cb->prof, z2z::kProfLogitsMerge, 1, s);
+    Z2Z_CUDA(z2z::launch_pick_codes(B, w_argmax, a.sample, d_forced, d_next_codes, d_selected, s), "decode_step");
+  }
   // step 10: online LZW update
-  Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_next_codes, nullptr, w_new, s), "decode_step");
+  {
+    z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, s);
+    Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_next_codes, nullptr, w_new, s), "decode_step");
+  }
   // cache update: the at most one new entry per sequence, on both sides
   if (cb->cfg.cap > 0) {
     z2z::EntryList el = entry_list(cb);
-    Z2Z_CUDA(z2z::launch_entry_offsets_from_new(cb->view, w_new, el, s), "decode_step");
-    Z2Z_CUDA(z2z::launch_entry_fill(cb->view, 0, nullptr, w_new, el, 0, s), "decode_step");
+    {
+      z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 2, s);
+      Z2Z_CUDA(z2z::launch_entry_offsets_from_new(cb->view, w_new, el, s), "decode_step");
+      Z2Z_CUDA(z2z::launch_entry_fill(cb->view, 0, nullptr, w_new, el, 0, s), "decode_step");
+    }
     z2z::EncoderArgs e = encoder_args(cb, d_WE, enc_E, d_Eh, d_Eh_f32);
-    Z2Z_CUDA(z2z::run_encoder_pass(cb->view, e, el, cb->use_tensor_cores != 0, s), "decode_step");
+    Z2Z_CUDA(z2z::run_encoder_pass(cb->view, e, el, cb->use_tensor_cores != 0, &cb->prof, s), "decode_step");
     if (!tied) {
       z2z::EncoderArgs u = encoder_args(cb, d_WU, enc_U, d_Uh, d_Uh_f32);
-      Z2Z_CUDA(z2z::run_encoder_pass(cb->view, u, el, cb->use_tensor_cores != 0, s), "decode_step");
+      Z2Z_CUDA(z2z::run_encoder_pass(cb->view, u, el, cb->use_tensor_cores != 0, &cb->prof, s), "decode_step");
     }
+    z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 2, s);
     Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 0, s), "decode_step");
     Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 1, s), "decode_step");
   }
@@ -319,6 +342,31 @@ int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t*
     delete[] tmp;
     if (e != cudaSuccess) return fail_cuda(e, "codebook_read");
   }
+  return Z2Z_OK;
+}
+
+int32_t z2z_profile(z2z_codebook* cb, int32_t enable) {
+  if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
+  cb->prof.timing = enable != 0;
+  return Z2Z_OK;
+}
+
+int32_t z2z_profile_read(z2z_codebook* cb, int32_t n_classes, double* h_ms, int64_t* h_launches,
+                         z2z_stream stream) {
+  if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
+  if (n_classes < 0 || n_classes > z2z::kProfClasses) n_classes = z2z::kProfClasses;
+  Z2Z_CUDA(cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)), "profile_read");
+  double ms[z2z::kProfClasses] = {0, 0, 0, 0, 0};
+  for (auto& r : cb->prof.recs) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) ms[r.cls] += t;
+  }
+  for (int i = 0; i < n_classes; ++i) {
+    if (h_ms) h_ms[i] = ms[i];
+    if (h_launches) h_launches[i] = cb->prof.launches[i];
+  }
+  cb->prof.release_all();
+  for (int i = 0; i < z2z::kProfClasses; ++i) cb->prof.launches[i] = 0;
   return Z2Z_OK;
 }
 

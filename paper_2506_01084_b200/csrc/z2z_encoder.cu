@@ -288,37 +288,54 @@ cudaError_t launch_mark_embedded(const CbView& cb, int which, cudaStream_t s) {
 
 template <typename T>
 static cudaError_t encoder_pass_simt(const CbView& cb, const EncoderArgs& a, const EntryList& el,
-                                     cudaStream_t s) {
+                                     Prof* prof, cudaStream_t s) {
   const int d = a.d, dff = a.dff, M = cb.M;
   const int E = el.chunk, R = E * M;
   const int32_t* n_live = el.off + cb.B + 1;
   auto W = [&](int i) { return reinterpret_cast<const T*>(a.w[i]); };
-  k_enc_gather<T><<<R, 128, 0, s>>>(cb, el, reinterpret_cast<const T*>(a.table), W(0), a.X, d);
+  { ProfScope ps(prof, kProfEncOther, 1, s);
+    k_enc_gather<T><<<R, 128, 0, s>>>(cb, el, reinterpret_cast<const T*>(a.table), W(0), a.X, d); }
   const dim3 blk(256);
   const int rt = (R + kTR - 1) / kTR;
   for (int l = 0; l < a.layers; ++l) {
     const int o = 1 + 12 * l;
-    k_enc_layernorm<T><<<R, 256, 0, s>>>(cb, el, a.X, W(o + 0), W(o + 1), a.A, d);
-    k_enc_linear<T, 0><<<dim3((3 * d + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.A, d, W(o + 2), 3 * d,
-                                                                        W(o + 3), a.QKV, R, n_live, M);
-    k_enc_attention<<<dim3(E, a.heads), dim3(32, M), 0, s>>>(cb, el, a.QKV, a.A, d, a.heads);
-    k_enc_linear<T, 2><<<dim3((d + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.A, d, W(o + 4), d, W(o + 5),
-                                                                    a.X, R, n_live, M);
-    k_enc_layernorm<T><<<R, 256, 0, s>>>(cb, el, a.X, W(o + 6), W(o + 7), a.A, d);
-    k_enc_linear<T, 1><<<dim3((dff + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.A, d, W(o + 8), dff,
-                                                                      W(o + 9), a.H, R, n_live, M);
-    k_enc_linear<T, 2><<<dim3((d + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.H, dff, W(o + 10), d,
-                                                                    W(o + 11), a.X, R, n_live, M);
+{ ProfScope ps(prof, kProfEncOther, 1, s);
+        k_enc_layernorm<T><<<R, 256, 0, s>>>(cb, el, a.X, W(o + 0), W(o + 1), a.A, d);
+      }
+{ ProfScope ps(prof, kProfEncGemm, 1, s);
+        k_enc_linear<T, 0><<<dim3((3 * d + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.A, d, W(o + 2), 3 * d,
+                                                                          W(o + 3), a.QKV, R, n_live, M);
+      }
+{ ProfScope ps(prof, kProfEncOther, 1, s);
+        k_enc_attention<<<dim3(E, a.heads), dim3(32, M), 0, s>>>(cb, el, a.QKV, a.A, d, a.heads);
+      }
+{ ProfScope ps(prof, kProfEncGemm, 1, s);
+        k_enc_linear<T, 2><<<dim3((d + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.A, d, W(o + 4), d, W(o + 5),
+                                                                      a.X, R, n_live, M);
+      }
+{ ProfScope ps(prof, kProfEncOther, 1, s);
+        k_enc_layernorm<T><<<R, 256, 0, s>>>(cb, el, a.X, W(o + 6), W(o + 7), a.A, d);
+      }
+{ ProfScope ps(prof, kProfEncGemm, 1, s);
+        k_enc_linear<T, 1><<<dim3((dff + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.A, d, W(o + 8), dff,
+                                                                        W(o + 9), a.H, R, n_live, M);
+      }
+{ ProfScope ps(prof, kProfEncGemm, 1, s);
+        k_enc_linear<T, 2><<<dim3((d + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.H, dff, W(o + 10), d,
+                                                                      W(o + 11), a.X, R, n_live, M);
+      }
   }
-  k_enc_pool<T><<<E, 256, 0, s>>>(cb, el, a.X, reinterpret_cast<T*>(a.cache), a.cache_f32, d);
+{ ProfScope ps(prof, kProfEncOther, 1, s);
+      k_enc_pool<T><<<E, 256, 0, s>>>(cb, el, a.X, reinterpret_cast<T*>(a.cache), a.cache_f32, d);
+      }
   return cudaGetLastError();
 }
 
 cudaError_t run_encoder_pass(const CbView& cb, const EncoderArgs& a, const EntryList& el,
-                             bool use_tensor_cores, cudaStream_t s) {
+                             bool use_tensor_cores, Prof* prof, cudaStream_t s) {
   (void)use_tensor_cores;
-  if (a.dtype == Z2Z_DTYPE_FP32) return encoder_pass_simt<float>(cb, a, el, s);
-  return encoder_pass_simt<__nv_bfloat16>(cb, a, el, s);
+  if (a.dtype == Z2Z_DTYPE_FP32) return encoder_pass_simt<float>(cb, a, el, prof, s);
+  return encoder_pass_simt<__nv_bfloat16>(cb, a, el, prof, s);
 }
 
 }  // namespace z2z

@@ -4,6 +4,7 @@
 #include <stdint.h>
 
 #include "z2z_common.cuh"
+#include "z2z_prof.h"
 
 namespace z2z {
 
@@ -46,7 +47,7 @@ cudaError_t launch_entry_fill(const CbView& cb, int which, const int32_t* first,
                               cudaStream_t s);
 cudaError_t launch_mark_embedded(const CbView& cb, int which, cudaStream_t s);
 cudaError_t run_encoder_pass(const CbView& cb, const EncoderArgs& a, const EntryList& el,
-                             bool use_tensor_cores, cudaStream_t s);
+                             bool use_tensor_cores, Prof* prof, cudaStream_t s);
 
 // ---- z2z_logits.cu ---------------------------------------------------------------------------
 struct LogitsArgs {
@@ -63,7 +64,7 @@ struct LogitsArgs {
   void* lpart; size_t lpart_bytes;
   int row_base;                 // global index of row 0 of this launch (sampling counter)
 };
-cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, cudaStream_t s);
+cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, Prof* prof, cudaStream_t s);
 
 // Selected code of the decode step: sample or argmax, overridden by `forced` when given.
 cudaError_t launch_pick_codes(int B, const int32_t* argmax, const int32_t* sample,

@@ -158,7 +158,7 @@ __global__ void k_fill_nan(float* p, int n) {
   if (i < n) p[i] = __int_as_float(0x7fc00000);
 }
 
-cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, cudaStream_t s) {
+cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, Prof* prof, cudaStream_t s) {
   const int n_static = (cb.V + kTJ - 1) / kTJ;
   const int tiles_per_seq = (cb.cap + kTJ - 1) / kTJ;
   const int n_tiles = n_static + cb.B * tiles_per_seq;
@@ -167,11 +167,18 @@ cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, cudaStream_t 
   if (G > n_tiles) G = n_tiles;
   while (G > 1 && (size_t)a.N * G * sizeof(LogitPartial) > a.lpart_bytes) --G;
   if ((size_t)a.N * G * sizeof(LogitPartial) > a.lpart_bytes) return cudaErrorInvalidValue;
-  if (a.target_logit) k_fill_nan<<<(a.N + 255) / 256, 256, 0, s>>>(a.target_logit, a.N);
-  if (a.dtype == Z2Z_DTYPE_FP32)
-    k_logits_simt<float><<<dim3(G, row_tiles), 256, 0, s>>>(cb, a, n_static, tiles_per_seq, n_tiles);
-  else
-    k_logits_simt<__nv_bfloat16><<<dim3(G, row_tiles), 256, 0, s>>>(cb, a, n_static, tiles_per_seq, n_tiles);
+  if (a.target_logit) {
+    ProfScope ps(prof, kProfLogitsMerge, 1, s);
+    k_fill_nan<<<(a.N + 255) / 256, 256, 0, s>>>(a.target_logit, a.N);
+  }
+  {
+    ProfScope ps(prof, kProfLogits, 1, s);
+    if (a.dtype == Z2Z_DTYPE_FP32)
+      k_logits_simt<float><<<dim3(G, row_tiles), 256, 0, s>>>(cb, a, n_static, tiles_per_seq, n_tiles);
+    else
+      k_logits_simt<__nv_bfloat16><<<dim3(G, row_tiles), 256, 0, s>>>(cb, a, n_static, tiles_per_seq, n_tiles);
+  }
+  ProfScope ps(prof, kProfLogitsMerge, 1, s);
   k_logits_merge<<<(a.N + 3) / 4, 128, 0, s>>>(a, G);
   return cudaGetLastError();
 }

@@ -165,6 +165,12 @@ int32_t z2z_status(z2z_codebook* cb, int32_t* h_status, int32_t* h_n, z2z_stream
 int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t* h_len,
                           z2z_stream stream);
 
+/* Kernel family used for bf16 sessions (no counterpart in the paper; cross-checking aid).
+ * enable = 1 (default): tcgen05 tensor-core kernels wherever the shapes allow (d and enc_dff
+ * multiples of 128).  enable = 0: the CUDA-core kernels, which keep activations in fp32 and are
+ * the path fp32 sessions always take.  Both produce results within the stated tolerance.        */
+int32_t z2z_set_tensor_cores(z2z_codebook* cb, int32_t enable);
+
 /* Launch accounting and per-kernel-class timing (no counterpart in the paper; measurement aid).
  * The library always counts the kernels it launches, per class:
  *   0 joint-logits main kernel, 1 logits merge / selection, 2 LZW kernels,

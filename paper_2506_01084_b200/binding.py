@@ -24,7 +24,7 @@ CACHE_EMBED, CACHE_UNEMBED = 0, 1
 EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lzw_step",
            "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
            "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error", "z2z_profile",
-           "z2z_profile_read"]
+           "z2z_profile_read", "z2z_set_tensor_cores"]
 
 
 class Config(C.Structure):
@@ -209,3 +209,7 @@ def z2z_profile_read(cb: Codebook):
     _check(lib().z2z_profile_read(cb.handle, C.c_int32(n), ms, cnt, _stream()))
     return ({k: ms[i] for i, k in enumerate(PROFILE_CLASSES)},
             {k: int(cnt[i]) for i, k in enumerate(PROFILE_CLASSES)})
+
+
+def z2z_set_tensor_cores(cb: Codebook, enable: bool):
+    _check(lib().z2z_set_tensor_cores(cb.handle, C.c_int32(1 if enable else 0)))

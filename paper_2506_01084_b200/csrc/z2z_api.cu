@@ -62,7 +62,7 @@ z2z::EntryList entry_list(z2z_codebook* cb) {
 }
 
 z2z::EncoderArgs encoder_args(z2z_codebook* cb, const void* table, const z2z_encoder_weights* enc,
-                              void* cache, float* cache_f32) {
+                              void* cache, float* cache_f32, int entries, int group = 0) {
   z2z::EncoderArgs a{};
   a.d = cb->cfg.d; a.dff = cb->dff; a.heads = cb->heads; a.layers = cb->cfg.enc_layers;
   a.M = cb->cfg.M; a.dtype = cb->cfg.dtype;
@@ -73,8 +73,16 @@ z2z::EncoderArgs encoder_args(z2z_codebook* cb, const void* table, const z2z_enc
   a.H = reinterpret_cast<float*>(cb->ws + cb->plan.off_H);
   a.Ahl = reinterpret_cast<__nv_bfloat16*>(cb->ws + cb->plan.off_Ahl);
   a.Hhl = reinterpret_cast<__nv_bfloat16*>(cb->ws + cb->plan.off_Hhl);
+  if (group == 1) {
+    a.X = reinterpret_cast<float*>(cb->ws + cb->plan.off_g1_X);
+    a.QKV = reinterpret_cast<float*>(cb->ws + cb->plan.off_g1_QKV);
+    a.Ahl = reinterpret_cast<__nv_bfloat16*>(cb->ws + cb->plan.off_g1_Ahl);
+    a.Hhl = reinterpret_cast<__nv_bfloat16*>(cb->ws + cb->plan.off_g1_Hhl);
+  }
   a.part = reinterpret_cast<float*>(cb->ws + cb->plan.off_part);
   a.part_bytes = cb->plan.part_bytes;
+  a.entries = entries;
+  a.err = reinterpret_cast<int*>(cb->ws + cb->plan.off_words);
   return a;
 }
 
@@ -106,7 +114,12 @@ int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s) {
     if (a.target_logit) c.target_logit = a.target_logit + r0;
     if (a.logits_debug) c.logits_debug = a.logits_debug + (size_t)r0 * ldbg;
     if (a.row_seq == nullptr && r0 > 0) return fail(Z2Z_ERR_INVALID_ARG, "d_row_seq is required when N > B");
-    Z2Z_CUDA(z2z::run_logits_simt(cb->view, c, &cb->prof, s), "logits");
+    if (cb->use_tensor_cores && z2z::logits_tc_supported(cb->cfg.d, cb->cfg.dtype)) {
+      int* words = reinterpret_cast<int*>(cb->ws + cb->plan.off_words);
+      Z2Z_CUDA(z2z::run_logits_tc(cb->view, c, words + 1, words, &cb->prof, s), "logits (tensor cores)");
+    } else {
+      Z2Z_CUDA(z2z::run_logits_simt(cb->view, c, &cb->prof, s), "logits");
+    }
   }
   return Z2Z_OK;
 }
@@ -144,7 +157,7 @@ int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, 
   }
   h->cfg = c; h->plan = plan; h->ws = reinterpret_cast<char*>(d_ws); h->ws_bytes = ws_bytes;
   h->dff = c.enc_dff; h->heads = c.enc_heads;
-  h->use_tensor_cores = 0;
+  h->use_tensor_cores = 1;
   z2z::CbView& v = h->view;
   v.V = c.V; v.M = c.M; v.cap = c.cap; v.B = c.B; v.n_slots = plan.n_slots;
   v.hash = reinterpret_cast<unsigned long long*>(h->ws + plan.off_hash);
@@ -155,6 +168,7 @@ int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, 
   v.status = reinterpret_cast<int32_t*>(h->ws + plan.off_status);
   v.n_emb = reinterpret_cast<int32_t*>(h->ws + plan.off_n_emb);
   *cb = h;
+  Z2Z_CUDA(cudaMemsetAsync(h->ws + plan.off_words, 0, 256, reinterpret_cast<cudaStream_t>(stream)), "codebook_init");
   z2z::ProfScope ps(&h->prof, z2z::kProfLzw, 1, reinterpret_cast<cudaStream_t>(stream));
   Z2Z_CUDA(z2z::launch_codebook_clear(v, reinterpret_cast<cudaStream_t>(stream)), "codebook_init");
   return Z2Z_OK;
@@ -197,7 +211,9 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
   if (cb->cfg.cap == 0) return Z2Z_OK;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   z2z::EntryList el = entry_list(cb);
-  z2z::EncoderArgs a = encoder_args(cb, d_table, enc, d_cache, d_cache_f32);
+  z2z::EncoderArgs a = encoder_args(cb, d_table, enc, d_cache, d_cache_f32, el.chunk);
+  const bool tc = cb->use_tensor_cores && cb->cfg.enc_layers >= 0 &&
+                  z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype);
   long long bound = (long long)cb->cfg.B * cb->cfg.cap;
   if (max_entries > 0 && max_entries < bound) bound = max_entries;
   const int n_chunks = (int)((bound + el.chunk - 1) / el.chunk);
@@ -210,7 +226,8 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
       z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
       Z2Z_CUDA(z2z::launch_entry_fill(cb->view, which, d_first, nullptr, el, c, s), "hyper_embed");
     }
-    Z2Z_CUDA(z2z::run_encoder_pass(cb->view, a, el, cb->use_tensor_cores != 0, &cb->prof, s), "hyper_embed");
+    if (tc) Z2Z_CUDA(z2z::run_encoder_pass_tc(cb->view, &a, 1, el, &cb->prof, s), "hyper_embed (tensor cores)");
+    else Z2Z_CUDA(z2z::run_encoder_pass(cb->view, a, el, false, &cb->prof, s), "hyper_embed");
   }
   if (!d_first) {
     z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
@@ -300,11 +317,18 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
       Z2Z_CUDA(z2z::launch_entry_offsets_from_new(cb->view, w_new, el, s), "decode_step");
       Z2Z_CUDA(z2z::launch_entry_fill(cb->view, 0, nullptr, w_new, el, 0, s), "decode_step");
     }
-    z2z::EncoderArgs e = encoder_args(cb, d_WE, enc_E, d_Eh, d_Eh_f32);
-    Z2Z_CUDA(z2z::run_encoder_pass(cb->view, e, el, cb->use_tensor_cores != 0, &cb->prof, s), "decode_step");
-    if (!tied) {
-      z2z::EncoderArgs u = encoder_args(cb, d_WU, enc_U, d_Uh, d_Uh_f32);
-      Z2Z_CUDA(z2z::run_encoder_pass(cb->view, u, el, cb->use_tensor_cores != 0, &cb->prof, s), "decode_step");
+    const bool tc = cb->use_tensor_cores && z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype);
+    z2z::EncoderArgs g[2];
+    g[0] = encoder_args(cb, d_WE, enc_E, d_Eh, d_Eh_f32, B, 0);
+    if (!tied) g[1] = encoder_args(cb, d_WU, enc_U, d_Uh, d_Uh_f32, B, 1);
+    if (tc) {
+      Z2Z_CUDA(z2z::run_encoder_pass_tc(cb->view, g, tied ? 1 : 2, el, &cb->prof, s), "decode_step (tensor cores)");
+    } else {
+      Z2Z_CUDA(z2z::run_encoder_pass(cb->view, g[0], el, false, &cb->prof, s), "decode_step");
+      if (!tied) {
+        g[1] = encoder_args(cb, d_WU, enc_U, d_Uh, d_Uh_f32, B, 0);
+        Z2Z_CUDA(z2z::run_encoder_pass(cb->view, g[1], el, false, &cb->prof, s), "decode_step");
+      }
     }
     z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 2, s);
     Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 0, s), "decode_step");
@@ -319,7 +343,11 @@ int32_t z2z_status(z2z_codebook* cb, int32_t* h_status, int32_t* h_n, z2z_stream
   const size_t bytes = (size_t)cb->cfg.B * 4;
   if (h_status) Z2Z_CUDA(cudaMemcpyAsync(h_status, cb->view.status, bytes, cudaMemcpyDeviceToHost, s), "status");
   if (h_n) Z2Z_CUDA(cudaMemcpyAsync(h_n, cb->view.n, bytes, cudaMemcpyDeviceToHost, s), "status");
+  int kernel_err = 0;
+  Z2Z_CUDA(cudaMemcpyAsync(&kernel_err, cb->ws + cb->plan.off_words, 4, cudaMemcpyDeviceToHost, s), "status");
   Z2Z_CUDA(cudaStreamSynchronize(s), "status");
+  if (kernel_err && h_status)
+    for (int b = 0; b < cb->cfg.B; ++b) h_status[b] |= Z2Z_ST_WAIT_TIMEOUT;
   return Z2Z_OK;
 }
 
@@ -342,6 +370,12 @@ int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t*
     delete[] tmp;
     if (e != cudaSuccess) return fail_cuda(e, "codebook_read");
   }
+  return Z2Z_OK;
+}
+
+int32_t z2z_set_tensor_cores(z2z_codebook* cb, int32_t enable) {
+  if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
+  cb->use_tensor_cores = enable != 0;
   return Z2Z_OK;
 }
 

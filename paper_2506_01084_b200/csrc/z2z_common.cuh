@@ -52,6 +52,11 @@ __host__ __device__ inline uint32_t hash_pair(uint32_t prefix, uint32_t token) {
   return h;
 }
 
+// CTA that owns unit u when U units are dealt to G CTAs as [floor(c U / G), floor((c+1) U / G)).
+__host__ __device__ inline long long owner_of(long long u, long long U, long long G) {
+  return ((u + 1) * G - 1) / U;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Workspace plan: byte offsets of every region inside the caller's workspace.
 // ---------------------------------------------------------------------------------------------
@@ -63,6 +68,8 @@ struct WsPlan {
   size_t off_entry_seq, off_entry_idx, off_entry_off, off_new_entry, off_sel;
   size_t off_X, off_A, off_QKV, off_H;            // fp32 encoder activations
   size_t off_Ahl, off_Hhl;                        // bf16 hi/lo activations (tensor-core path)
+  size_t off_g1_X, off_g1_QKV, off_g1_Ahl, off_g1_Hhl;   // second encoder of the decode step
+  size_t off_words;                               // device words: [0] kernel error, [1] logits tiles
   size_t off_part, part_bytes;                    // GEMM split-K partial tiles
   size_t off_lpart, lpart_bytes;                  // logits partial reductions
   size_t off_step_out;                            // small per-step outputs
@@ -103,14 +110,23 @@ inline WsPlan plan_workspace(const z2z_config& c) {
   size_t R = (size_t)p.enc_rows;
   size_t dff = (size_t)(c.enc_dff > 0 ? c.enc_dff : 4 * c.d);
   size_t wide = dff > (size_t)3 * c.d ? dff : (size_t)3 * c.d;
-  p.off_X = take(R * c.d * 4);
-  p.off_A = take(R * c.d * 4);
-  p.off_QKV = take(R * 3 * c.d * 4);
-  p.off_H = take(R * dff * 4);
-  p.off_Ahl = take(2 * R * c.d * 2);
-  p.off_Hhl = take(2 * R * dff * 2);
-  p.part_bytes = (size_t)4 * 1024 * 1024 + R * wide * 4 * 2;
+  // encoder scratch: one full set for prefill passes (group 0) and a decode-sized set (B entries)
+  // for the second encoder of the decode step (group 1)
+  size_t Rp = (R + 127) / 128 * 128 + 128;
+  size_t R1 = ((size_t)c.B * c.M + 127) / 128 * 128 + 128;
+  p.off_X = take(Rp * c.d * 4);
+  p.off_A = take(Rp * c.d * 4);
+  p.off_QKV = take(Rp * 3 * c.d * 4);
+  p.off_H = take(Rp * dff * 4);
+  p.off_Ahl = take(2 * Rp * c.d * 2);
+  p.off_Hhl = take(2 * Rp * dff * 2);
+  p.off_g1_X = take(R1 * c.d * 4);
+  p.off_g1_QKV = take(R1 * 3 * c.d * 4);
+  p.off_g1_Ahl = take(2 * R1 * c.d * 2);
+  p.off_g1_Hhl = take(2 * R1 * dff * 2);
+  p.part_bytes = ((Rp / 128) * 2 * ((wide + 127) / 128) + 256) * (size_t)65536;
   p.off_part = take(p.part_bytes);
+  p.off_words = take(256);
   p.lpart_bytes = (size_t)kLogitPartRows * 32;
   p.off_lpart = take(p.lpart_bytes);
   p.off_step_out = take((size_t)c.B * 64);

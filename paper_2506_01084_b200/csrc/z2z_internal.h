@@ -35,7 +35,14 @@ struct EncoderArgs {
   __nv_bfloat16 *Ahl, *Hhl;     // bf16 hi/lo scratch for the tensor-core path
   float* part;                  // split-K partial tiles
   size_t part_bytes;
+  int entries;                  // host bound on the entries of this pass (<= chunk)
+  int* err;                     // device error word of the tensor-core kernels
 };
+bool encoder_tc_supported(int d, int dff, int dtype);
+bool logits_tc_supported(int d, int dtype);
+// Two encoders (embedding side, unembedding side) run through the same launches.
+cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* groups, int n_groups,
+                                const EntryList& el, Prof* prof, cudaStream_t s);
 // Per-sequence ranges from (first, count) arrays, or "everything since the last call" when NULL.
 cudaError_t launch_entry_offsets(const CbView& cb, int which, const int32_t* first,
                                  const int32_t* count, const EntryList& el, cudaStream_t s);
@@ -65,6 +72,11 @@ struct LogitsArgs {
   int row_base;                 // global index of row 0 of this launch (sampling counter)
 };
 cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, Prof* prof, cudaStream_t s);
+// Partial reduction of one hidden row over a subset of the columns.
+struct __align__(32) LogitPartial { float m, s; int idx; float gm; int gidx; int pad[3]; };
+// Tensor-core (tcgen05) version for bf16; returns cudaErrorNotSupported when the shapes do not fit.
+cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word, Prof* prof,
+                          cudaStream_t s);
 
 // Selected code of the decode step: sample or argmax, overridden by `forced` when given.
 cudaError_t launch_pick_codes(int B, const int32_t* argmax, const int32_t* sample,

@@ -12,8 +12,6 @@
 
 namespace z2z {
 
-struct __align__(32) LogitPartial { float m, s; int idx; float gm; int gidx; int pad[3]; };
-
 struct TileDesc { const void* base; int col0; int nvalid; int owner; int k0; };
 
 __device__ __forceinline__ TileDesc logits_tile(const CbView& cb, int t, int n_static,

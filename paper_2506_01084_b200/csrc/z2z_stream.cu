@@ -1,0 +1,567 @@
+// Weight-streaming skinny GEMM on tcgen05 tensor cores, for the HBM-bound decode regime.
+//
+//   D[r, j] = sum_k A[r, k] * W[j, k]      A: <=128 activation rows (bf16, K-major)
+//                                          W: weight rows streamed once from HBM (bf16, K-major)
+//
+// One persistent CTA per SM.  Warp 0 issues TMA loads into a ring of shared-memory stages, warp 1
+// issues tcgen05.mma (activations as the 128-row M operand, a tile of NT weight rows as the N
+// operand, fp32 accumulator in tensor memory, double buffered), warps 2-5 drain accumulators.
+// Two uses share the pipeline:
+//   * hyper-encoder linear layers: work is cut stream-K style, every CTA gets the same number of
+//     (tile, k-step) units, and each CTA stores fp32 partial tiles that the next (element-wise)
+//     kernel sums in a fixed order, so results are deterministic;
+//   * joint logits (paper Section 2.3 steps 7-9): tiles run over W_U and then over the visible
+//     rows of each sequence's U_h; the epilogue keeps max / sum-exp / argmax / best perturbed
+//     score per hidden row in registers, so the logits are never written.
+// Only the rows of A that exist are loaded: the MMA also reads the shared memory behind them,
+// which only feeds accumulator rows nobody reads (rows of D depend on the same rows of A only).
+#include "z2z_common.cuh"
+#include "z2z_internal.h"
+#include "z2z_sm100.cuh"
+#include "z2z_stream.h"
+
+namespace z2z {
+using namespace sm100;
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kTailPad = 16384;          // readable shared memory behind the last A tile
+
+struct Ctrl {
+  unsigned long long full[kMaxStages], empty[kMaxStages], acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  int abort;
+  int vt;                                // logits: number of virtual column tiles
+};
+
+__host__ __device__ constexpr int tmem_cols(int nt) {
+  return 2 * nt <= 32 ? 32 : (2 * nt <= 64 ? 64 : (2 * nt <= 128 ? 128 : (2 * nt <= 256 ? 256 : 512)));
+}
+
+struct Job {
+  int amap, wmap;        // tensor map indices
+  int arow, wrow;        // first row in A / W tensors
+  int kb0, kb1;          // k-step range
+  long long slot;        // GEMM: partial slot
+  int col0, nvalid, owner, k0;   // logits: first column id, valid rows, owning sequence, first entry
+  int rt;                // logits: hidden-row tile
+};
+
+// ---- GEMM schedule ------------------------------------------------------------------------------
+struct GemmSched {
+  const StreamGemmParams& p;
+  long long u, u1, c;
+  __device__ GemmSched(const StreamGemmParams& pp, int NT) : p(pp) {
+    const long long U = (long long)p.row_tiles * p.groups * p.tiles_per_group * p.ksteps, G = gridDim.x;
+    c = blockIdx.x;
+    u = c * U / G;
+    u1 = (c + 1) * U / G;
+    (void)NT;
+  }
+  __device__ bool next(Job& j, int NT) {
+    if (u >= u1) return false;
+    const long long tile = u / p.ksteps;
+    j.kb0 = (int)(u - tile * p.ksteps);
+    long long left = u1 - u;
+    j.kb1 = (int)((p.ksteps - j.kb0) < left ? p.ksteps : j.kb0 + left);
+    const int per_rt = p.groups * p.tiles_per_group;
+    j.rt = (int)(tile / per_rt);
+    const int rem = (int)(tile - (long long)j.rt * per_rt);
+    const int g = rem / p.tiles_per_group;
+    j.amap = g; j.wmap = g; j.arow = j.rt * 128;
+    j.wrow = (rem - g * p.tiles_per_group) * NT;
+    j.slot = tile + c;
+    u += j.kb1 - j.kb0;
+    return true;
+  }
+};
+
+// ---- logits schedule ----------------------------------------------------------------------------
+struct LogitSched {
+  const StreamLogitsParams& p;
+  const int* pref;       // shared: prefix of ragged tile counts, [B + 1]
+  long long u, u1;
+  int n_static, vt, ksteps;
+  __device__ LogitSched(const StreamLogitsParams& pp, const int* s_pref, int vt_, int NT) : p(pp), pref(s_pref) {
+    n_static = (p.cb.V + NT - 1) / NT;
+    vt = vt_;
+    ksteps = p.ksteps;
+    const long long U = (long long)p.row_tiles * vt, G = gridDim.x, c = blockIdx.x;
+    u = c * U / G;
+    u1 = (c + 1) * U / G;
+  }
+  __device__ bool next(Job& j, int NT) {
+    if (u >= u1) return false;
+    j.rt = (int)(u / vt);
+    const int v = (int)(u - (long long)j.rt * vt);
+    j.amap = 0; j.arow = j.rt * 128; j.kb0 = 0; j.kb1 = ksteps; j.slot = 0;
+    if (v < n_static) {
+      j.wmap = 0; j.wrow = v * NT; j.col0 = v * NT; j.owner = -1; j.k0 = 0;
+      j.nvalid = p.cb.V - j.col0 < NT ? p.cb.V - j.col0 : NT;
+    } else {
+      const int x = v - n_static;
+      int lo = 0, hi = p.cb.B - 1;                 // last b with pref[b] <= x
+      while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (pref[mid] <= x) lo = mid; else hi = mid - 1; }
+      j.owner = lo;
+      j.k0 = (x - pref[lo]) * NT;
+      j.wmap = 1; j.wrow = lo * p.cb.cap + j.k0; j.col0 = p.cb.V + j.k0;
+      const int n = p.cb.n[lo];
+      j.nvalid = n - j.k0 < NT ? n - j.k0 : NT;
+    }
+    ++u;
+    return true;
+  }
+};
+
+// ---- roles shared by both kernels -----------------------------------------------------------------
+template <int NT, int KSB, int STAGES, class Sched>
+__device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t stage_base,
+                                              int a_parts, int a_box_rows, int a_part_row,
+                                              const CUtensorMap* const* amaps,
+                                              const CUtensorMap* const* wmaps) {
+  const uint32_t a_part_bytes = (uint32_t)KSB * a_box_rows * 128;
+  const uint32_t stage_bytes = a_parts * a_part_bytes + (uint32_t)KSB * NT * 128;
+  const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
+  int stage = 0; uint32_t phase = 0;
+  Job j;
+  while (sched.next(j, NT)) {
+    for (int ks = j.kb0; ks < j.kb1; ++ks) {
+      if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) return;
+      const uint32_t full = smem_u32(&ctrl->full[stage]);
+      mbar_expect_tx(full, stage_bytes);
+      const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
+      for (int part = 0; part < a_parts; ++part)
+#pragma unroll
+        for (int i = 0; i < KSB; ++i)
+          tma_load_2d(sb + part * a_part_bytes + i * a_box_rows * 128, amaps[j.amap],
+                      (ks * KSB + i) * 64, j.arow + part * a_part_row, full, pol_a);
+#pragma unroll
+      for (int i = 0; i < KSB; ++i)
+        tma_load_2d(sb + a_parts * a_part_bytes + i * NT * 128, wmaps[j.wmap], (ks * KSB + i) * 64,
+                    j.wrow, full, pol_w);
+      if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+    }
+  }
+}
+
+template <int NT, int KSB, int STAGES, class Sched>
+__device__ __forceinline__ void mma_role(Sched& sched, Ctrl* ctrl, uint32_t stage_base, int a_parts,
+                                         int a_box_rows, uint32_t tmem_base) {
+  const uint32_t a_part_bytes = (uint32_t)KSB * a_box_rows * 128;
+  const uint32_t stage_bytes = a_parts * a_part_bytes + (uint32_t)KSB * NT * 128;
+  constexpr uint32_t idesc = idesc_bf16_f32(128, NT);
+  int stage = 0; uint32_t phase = 0;
+  uint32_t job_i = 0;
+  Job j;
+  while (sched.next(j, NT)) {
+    const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
+    if (!mbar_wait(smem_u32(&ctrl->acc_empty[buf]), aph ^ 1u, &ctrl->abort)) return;
+    tc_fence_after();
+    const uint32_t d = tmem_base + buf * NT;
+    uint32_t acc = 0;
+    for (int ks = j.kb0; ks < j.kb1; ++ks) {
+      if (!mbar_wait(smem_u32(&ctrl->full[stage]), phase, &ctrl->abort)) return;
+      tc_fence_after();
+      const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
+#pragma unroll
+      for (int i = 0; i < KSB; ++i) {
+        const uint32_t wb = sb + a_parts * a_part_bytes + i * NT * 128;
+        for (int part = 0; part < a_parts; ++part) {
+          const uint32_t ab = sb + part * a_part_bytes + i * a_box_rows * 128;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            umma_bf16(d, smem_desc_sw128(ab + k * 32), smem_desc_sw128(wb + k * 32), idesc, acc);
+            acc = 1;
+          }
+        }
+      }
+      umma_commit(smem_u32(&ctrl->empty[stage]));          // frees the stage when the MMAs are done
+      if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+    }
+    umma_commit(smem_u32(&ctrl->acc_full[buf]));
+    ++job_i;
+  }
+}
+
+template <int STAGES>
+__device__ __forceinline__ void setup_barriers(Ctrl* ctrl) {
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      mbar_init(smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&ctrl->acc_full[b]), 1);
+      mbar_init(smem_u32(&ctrl->acc_empty[b]), 4);
+    }
+    ctrl->abort = 0;
+    mbar_init_fence();
+  }
+}
+
+// =================================================================================================
+// GEMM kernel: partial tiles out
+// =================================================================================================
+template <int NT, int KSB, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0,
+              const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmW0,
+              const __grid_constant__ CUtensorMap tmW1) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm);
+  const uint32_t stage_base = smem_u32(sm + 1024);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  setup_barriers<STAGES>(ctrl);
+  if (warp == 0 && lane == 0) { prefetch_tmap(&tmA0); prefetch_tmap(&tmW0); if (p.groups > 1) { prefetch_tmap(&tmA1); prefetch_tmap(&tmW1); } }
+  __syncthreads();
+  if (warp == 2) { tmem_alloc(smem_u32(&ctrl->tmem_base), tmem_cols(NT)); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctrl->tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const CUtensorMap* amaps[2] = {&tmA0, &tmA1};
+      const CUtensorMap* wmaps[2] = {&tmW0, &tmW1};
+      GemmSched sched(p, NT);
+      producer_role<NT, KSB, STAGES>(sched, ctrl, stage_base, p.a_parts, p.a_box_rows, p.a_part_row, amaps, wmaps);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      GemmSched sched(p, NT);
+      mma_role<NT, KSB, STAGES>(sched, ctrl, stage_base, p.a_parts, p.a_box_rows, tmem_base);
+    }
+  } else {
+    const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    const int row = q * 32 + lane;
+    GemmSched sched(p, NT);
+    uint32_t job_i = 0;
+    Job j;
+    while (sched.next(j, NT)) {
+      const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
+      if (!mbar_wait(smem_u32(&ctrl->acc_full[buf]), aph, &ctrl->abort)) break;
+      tc_fence_after();
+      if (q * 32 < p.out_rows) {
+        float* dst = p.part + j.slot * p.slot_stride + (long long)row * NT;
+#pragma unroll 1
+        for (int c0 = 0; c0 < NT; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * NT + c0, v);
+          tmem_ld_wait();
+          if (row < p.out_rows) {
+#pragma unroll
+            for (int x = 0; x < 32; x += 4)
+              *reinterpret_cast<uint4*>(dst + c0 + x) = make_uint4(v[x], v[x + 1], v[x + 2], v[x + 3]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty[buf]));
+      ++job_i;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.err, 1);
+  if (warp == 2) tmem_dealloc(tmem_base, tmem_cols(NT));
+}
+
+// =================================================================================================
+// Logits kernel: fused reductions
+// =================================================================================================
+template <int NT, int KSB, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+k_stream_logits(const StreamLogitsParams p, const __grid_constant__ CUtensorMap tmH,
+                const __grid_constant__ CUtensorMap tmWU, const __grid_constant__ CUtensorMap tmUh) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm);
+  int* s_pref = reinterpret_cast<int*>(sm + 1024);              // [B + 1] <= 4100 bytes
+  const uint32_t stage_base = smem_u32(sm + 1024 + 5120);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  setup_barriers<STAGES>(ctrl);
+  for (int b = threadIdx.x; b < p.cb.B; b += kThreads) s_pref[b + 1] = (p.cb.n[b] + NT - 1) / NT;
+  if (warp == 0 && lane == 0) { prefetch_tmap(&tmH); prefetch_tmap(&tmWU); prefetch_tmap(&tmUh); }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s_pref[0] = 0;
+    for (int b = 0; b < p.cb.B; ++b) s_pref[b + 1] += s_pref[b];
+    ctrl->vt = (p.cb.V + NT - 1) / NT + s_pref[p.cb.B];
+    if (blockIdx.x == 0) *p.vt_out = ctrl->vt;
+  }
+  if (warp == 2) { tmem_alloc(smem_u32(&ctrl->tmem_base), tmem_cols(NT)); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctrl->tmem_base;
+  const int vt = ctrl->vt;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const CUtensorMap* amaps[1] = {&tmH};
+      const CUtensorMap* wmaps[2] = {&tmWU, &tmUh};
+      LogitSched sched(p, s_pref, vt, NT);
+      producer_role<NT, KSB, STAGES>(sched, ctrl, stage_base, 1, p.a_box_rows, 0, amaps, wmaps);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      LogitSched sched(p, s_pref, vt, NT);
+      mma_role<NT, KSB, STAGES>(sched, ctrl, stage_base, 1, p.a_box_rows, tmem_base);
+    }
+  } else {
+    const int q = warp & 3;
+    const LogitsArgs& a = p.la;
+    LogitSched sched(p, s_pref, vt, NT);
+    const long long U = (long long)p.row_tiles * vt, G = gridDim.x;
+    const uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
+    const uint32_t c2 = (uint32_t)a.step, c3 = (uint32_t)(a.step >> 32);
+    const size_t ldbg = (size_t)p.cb.V + p.cb.cap;
+    RowRed red; red.init();
+    int cur_rt = -1, r = -1, my_seq = -1, my_nvis = 0, my_tgt = -1;
+    uint32_t job_i = 0;
+    Job j;
+    auto flush = [&]() {
+      if (cur_rt >= 0 && r < a.N) {
+        const long long first = owner_of((long long)cur_rt * vt, U, G);
+        LogitPartial* lp = reinterpret_cast<LogitPartial*>(a.lpart) + (size_t)r * p.part_stride + (blockIdx.x - first);
+        lp->m = red.m; lp->s = red.s; lp->idx = red.idx; lp->gm = red.gm; lp->gidx = red.gidx;
+      }
+    };
+    while (sched.next(j, NT)) {
+      if (j.rt != cur_rt) {
+        flush();
+        cur_rt = j.rt; red.init();
+        r = cur_rt * 128 + q * 32 + lane;
+        my_seq = -1; my_nvis = 0; my_tgt = -1;
+        if (r < a.N) {
+          my_seq = a.row_seq ? a.row_seq[r] : r;
+          if (my_seq < 0 || my_seq >= p.cb.B) my_seq = -1;
+          if (my_seq >= 0) {
+            my_nvis = p.cb.n[my_seq];
+            if (a.row_nvis) { const int x = a.row_nvis[r]; my_nvis = x < my_nvis ? (x < 0 ? 0 : x) : my_nvis; }
+          }
+          if (a.targets) my_tgt = a.targets[r];
+        }
+      }
+      const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
+      if (!mbar_wait(smem_u32(&ctrl->acc_full[buf]), aph, &ctrl->abort)) break;
+      tc_fence_after();
+      int limit = 0;
+      if (my_seq >= 0) limit = j.owner < 0 ? j.nvalid : (my_seq == j.owner ? min(j.nvalid, my_nvis - j.k0) : 0);
+      const int rows_here = a.N - cur_rt * 128;
+      if (q * 32 < rows_here && __any_sync(0xffffffffu, limit > 0)) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < NT; c0 += 32) {
+          if (!__any_sync(0xffffffffu, limit > c0)) break;
+          uint32_t v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * NT + c0, v);
+          tmem_ld_wait();
+          Philox4 px{0, 0, 0, 0};
+          int px_blk = -1;
+#pragma unroll
+          for (int x = 0; x < 32; ++x) {
+            if (c0 + x < limit) {
+              const float l = __uint_as_float(v[x]);
+              const int col = j.col0 + c0 + x;
+              red.add(l, col);
+              if (a.select == Z2Z_SELECT_GUMBEL) {
+                if ((col >> 2) != px_blk) {
+                  px_blk = col >> 2;
+                  px = philox4x32_10((uint32_t)px_blk, (uint32_t)(a.row_base + r), c2, c3, k0, k1);
+                }
+                red.add_score(fmaf(l, a.inv_temperature, gumbel_from_word(philox_word(px, col & 3))), col);
+              }
+              if (a.logits_debug) a.logits_debug[(size_t)r * ldbg + col] = l;
+              if (col == my_tgt && a.target_logit) a.target_logit[r] = l;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty[buf]));
+      ++job_i;
+    }
+    flush();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.err, 1);
+  if (warp == 2) tmem_dealloc(tmem_base, tmem_cols(NT));
+}
+
+// One warp per row: merge the partial reductions of the CTAs that touched the row's tile.
+__global__ void __launch_bounds__(128) k_stream_logits_merge(StreamLogitsParams p, int G) {
+  const LogitsArgs& a = p.la;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= a.N) return;
+  const long long vt = *p.vt_out, U = (long long)p.row_tiles * vt;
+  const int rt = r >> 7;
+  const long long first = owner_of((long long)rt * vt, U, G), last = owner_of((long long)(rt + 1) * vt - 1, U, G);
+  const LogitPartial* lp = reinterpret_cast<const LogitPartial*>(a.lpart) + (size_t)r * p.part_stride;
+  RowRed red; red.init();
+  for (int g = lane; g <= (int)(last - first); g += 32) {
+    RowRed o; o.m = lp[g].m; o.s = lp[g].s; o.idx = lp[g].idx; o.gm = lp[g].gm; o.gidx = lp[g].gidx;
+    red.merge(o);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    RowRed o;
+    o.m = __shfl_xor_sync(0xffffffffu, red.m, off);
+    o.s = __shfl_xor_sync(0xffffffffu, red.s, off);
+    o.idx = __shfl_xor_sync(0xffffffffu, red.idx, off);
+    o.gm = __shfl_xor_sync(0xffffffffu, red.gm, off);
+    o.gidx = __shfl_xor_sync(0xffffffffu, red.gidx, off);
+    red.merge(o);
+  }
+  if (lane == 0) {
+    if (a.lse) a.lse[r] = red.m + logf(red.s);
+    if (a.argmax) a.argmax[r] = red.idx == 0x7fffffff ? -1 : red.idx;
+    if (a.max_logit) a.max_logit[r] = red.m;
+    if (a.sample) a.sample[r] = red.gidx == 0x7fffffff ? -1 : red.gidx;
+  }
+}
+
+__global__ void k_fill_nan_f32(float* p, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = __int_as_float(0x7fc00000);
+}
+
+// ---- host helpers ---------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+  }
+  return fn;
+}
+
+}  // namespace
+
+// Tensor map over a row-major bf16 matrix [rows, cols]; box = 64 columns x box_rows rows,
+// 128-byte swizzle, out-of-range elements read as zero.
+bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols % 8) || box_rows < 1 || box_rows > 256 || rows < 1) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  cuuint32_t es[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NT, int KSB>
+static int pick_stages(int a_parts, int a_box_rows, int extra) {
+  const int stage = a_parts * KSB * a_box_rows * 128 + KSB * NT * 128;
+  int s = (227 * 1024 - 2048 - extra - kTailPad) / stage;
+  return s > kMaxStages ? kMaxStages : s;
+}
+
+template <int NT, int KSB, int STAGES>
+static cudaError_t launch_gemm_t(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
+  const size_t stage = (size_t)p.a_parts * KSB * p.a_box_rows * 128 + (size_t)KSB * NT * 128;
+  const size_t smem = 1024 + 1024 + STAGES * stage + kTailPad;
+  auto kern = k_stream_gemm<NT, KSB, STAGES>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, kThreads, smem, s>>>(p, maps[0], maps[1], maps[2], maps[3]);
+  return cudaGetLastError();
+}
+
+// Launches the stream-K GEMM.  maps = {A group 0, A group 1, W group 0, W group 1}.
+cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
+  constexpr int NT = kGemmNT, KSB = kGemmKSB;
+  const int st = pick_stages<NT, KSB>(p.a_parts, p.a_box_rows, 0);
+  if (st >= 8) return launch_gemm_t<NT, KSB, 8>(p, maps, grid, s);
+  if (st >= 6) return launch_gemm_t<NT, KSB, 6>(p, maps, grid, s);
+  if (st >= 4) return launch_gemm_t<NT, KSB, 4>(p, maps, grid, s);
+  if (st >= 3) return launch_gemm_t<NT, KSB, 3>(p, maps, grid, s);
+  return cudaErrorInvalidConfiguration;
+}
+
+template <int NT, int KSB, int STAGES>
+static cudaError_t launch_logits_t(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
+  const size_t stage = (size_t)KSB * p.a_box_rows * 128 + (size_t)KSB * NT * 128;
+  const size_t smem = 1024 + 1024 + 5120 + STAGES * stage + kTailPad;
+  auto kern = k_stream_logits<NT, KSB, STAGES>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, kThreads, smem, s>>>(p, maps[0], maps[1], maps[2]);
+  return cudaGetLastError();
+}
+
+bool logits_tc_supported(int d, int dtype) { return dtype == Z2Z_DTYPE_BF16 && d % 64 == 0; }
+
+cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word, Prof* prof,
+                          cudaStream_t s) {
+  static int n_sm = 0;
+  if (!n_sm) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (n_sm <= 0) n_sm = 148;
+  }
+  StreamLogitsParams p{};
+  p.cb = cb; p.la = a;
+  p.ksteps = (a.d / 64 + kLogitKSB - 1) / kLogitKSB;
+  p.row_tiles = (a.N + 127) / 128;
+  p.a_box_rows = a.N >= 128 ? 128 : (a.N + 7) / 8 * 8;
+  p.part_stride = (n_sm + p.row_tiles - 1) / p.row_tiles + 2;
+  p.vt_out = vt_word; p.err = err_word;
+  if ((size_t)a.N * p.part_stride * sizeof(LogitPartial) > a.lpart_bytes) return cudaErrorMemoryAllocation;
+  CUtensorMap maps[3];
+  if (!make_tmap_bf16(&maps[0], a.hidden, a.N, a.d, p.a_box_rows)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&maps[1], a.WU, cb.V, a.d, kLogitNT)) return cudaErrorInvalidValue;
+  if (cb.cap > 0) {
+    if (!make_tmap_bf16(&maps[2], a.Uh, (long long)cb.B * cb.cap, a.d, kLogitNT)) return cudaErrorInvalidValue;
+  } else {
+    maps[2] = maps[1];
+  }
+  // every CTA must own at least one unit: the static tiles alone give a lower bound on the units
+  long long units_lb = (long long)p.row_tiles * ((cb.V + kLogitNT - 1) / kLogitNT);
+  const int grid = units_lb < n_sm ? (int)units_lb : n_sm;
+  p.part_stride = (grid + p.row_tiles - 1) / p.row_tiles + 2;
+  return launch_stream_logits(p, maps, grid, prof, s);
+}
+
+cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, Prof* prof,
+                                 cudaStream_t s) {
+  constexpr int NT = kLogitNT, KSB = kLogitKSB;
+  const LogitsArgs& a = p.la;
+  if (a.target_logit) {
+    ProfScope ps(prof, kProfLogitsMerge, 1, s);
+    k_fill_nan_f32<<<(a.N + 255) / 256, 256, 0, s>>>(a.target_logit, a.N);
+  }
+  cudaError_t e;
+  {
+    ProfScope ps(prof, kProfLogits, 1, s);
+    const int st = pick_stages<NT, KSB>(1, p.a_box_rows, 5120);
+    if (st >= 8) e = launch_logits_t<NT, KSB, 8>(p, maps, grid, s);
+    else if (st >= 6) e = launch_logits_t<NT, KSB, 6>(p, maps, grid, s);
+    else if (st >= 4) e = launch_logits_t<NT, KSB, 4>(p, maps, grid, s);
+    else e = cudaErrorInvalidConfiguration;
+  }
+  if (e != cudaSuccess) return e;
+  ProfScope ps(prof, kProfLogitsMerge, 1, s);
+  k_stream_logits_merge<<<(a.N + 3) / 4, 128, 0, s>>>(p, grid);
+  return cudaGetLastError();
+}
+
+}  // namespace z2z

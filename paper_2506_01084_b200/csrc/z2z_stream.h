@@ -1,0 +1,47 @@
+// Parameters of the tcgen05 weight-streaming kernels (z2z_stream.cu).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "z2z_common.cuh"
+#include "z2z_internal.h"
+
+namespace z2z {
+
+constexpr int kMaxStages = 8;
+constexpr int kGemmNT = 128, kGemmKSB = 1;      // weight rows per tile, 64-wide k blocks per stage
+constexpr int kLogitNT = 128, kLogitKSB = 1;
+
+// Stream-K GEMM over `groups` independent problems of identical shape (the two hyper-encoders).
+// The unit space is (group, tile, k-step); CTA c of G owns units [floor(cU/G), floor((c+1)U/G)).
+// Every maximal run of units inside one tile and one CTA produces one fp32 partial tile of
+// out_rows x NT values in slot (global tile index + c).
+struct StreamGemmParams {
+  int row_tiles;         // 128-row tiles of A (outermost dimension of the unit space)
+  int groups, tiles_per_group, ksteps;
+  int a_box_rows;        // rows per TMA box of A (multiple of 8, <= 128)
+  int a_parts;           // MMA row groups per k16: 1, or 2 when hi and lo rows do not fit 128 rows
+  int a_part_row;        // first global row of part 1
+  int out_rows;          // accumulator rows stored
+  float* part;
+  long long slot_stride; // floats per slot
+  int* err;
+};
+
+struct StreamLogitsParams {
+  CbView cb;
+  LogitsArgs la;
+  int ksteps;
+  int a_box_rows;
+  int row_tiles;         // ceil(N / 128)
+  int part_stride;       // partial slots per row
+  int* vt_out;           // device word: number of virtual column tiles
+  int* err;
+};
+
+bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows);
+cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s);
+cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, Prof* prof,
+                                 cudaStream_t s);
+
+}  // namespace z2z

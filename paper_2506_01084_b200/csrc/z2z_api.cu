@@ -94,7 +94,7 @@ int check_encoder(z2z_codebook* cb, const z2z_encoder_weights* enc) {
   return Z2Z_OK;
 }
 
-int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s) {
+int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s, z2z::LogitsPartInfo* info = nullptr) {
   // rows are processed in blocks so that the partial-reduction scratch stays bounded
   const int N = a.N;
   const size_t esz = cb->cfg.dtype == Z2Z_DTYPE_FP32 ? 4 : 2;
@@ -116,9 +116,9 @@ int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s) {
     if (a.row_seq == nullptr && r0 > 0) return fail(Z2Z_ERR_INVALID_ARG, "d_row_seq is required when N > B");
     if (cb->use_tensor_cores && z2z::logits_tc_supported(cb->cfg.d, cb->cfg.dtype)) {
       int* words = reinterpret_cast<int*>(cb->ws + cb->plan.off_words);
-      Z2Z_CUDA(z2z::run_logits_tc(cb->view, c, words + 1, words, &cb->prof, s), "logits (tensor cores)");
+      Z2Z_CUDA(z2z::run_logits_tc(cb->view, c, words + 1, words, info, &cb->prof, s), "logits (tensor cores)");
     } else {
-      Z2Z_CUDA(z2z::run_logits_simt(cb->view, c, &cb->prof, s), "logits");
+      Z2Z_CUDA(z2z::run_logits_simt(cb->view, c, info, &cb->prof, s), "logits");
     }
   }
   return Z2Z_OK;
@@ -213,7 +213,7 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
   z2z::EntryList el = entry_list(cb);
   z2z::EncoderArgs a = encoder_args(cb, d_table, enc, d_cache, d_cache_f32, el.chunk);
   const bool tc = cb->use_tensor_cores && cb->cfg.enc_layers >= 0 &&
-                  z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype);
+                  z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype, cb->heads, cb->cfg.M);
   long long bound = (long long)cb->cfg.B * cb->cfg.cap;
   if (max_entries > 0 && max_entries < bound) bound = max_entries;
   const int n_chunks = (int)((bound + el.chunk - 1) / el.chunk);
@@ -298,26 +298,41 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
   a.lse = d_lse ? d_lse : w_lse; a.argmax = w_argmax; a.max_logit = w_max;
   a.sample = select == Z2Z_SELECT_GUMBEL ? w_sample : nullptr;
   a.lpart = cb->ws + cb->plan.off_lpart; a.lpart_bytes = cb->plan.lpart_bytes;
-  rc = logits_call(cb, a, s);
-  if (rc) return rc;
-  {
-    z2z::ProfScope ps(&cb->prof, z2z::kProfLogitsMerge, 1, s);
-    Z2Z_CUDA(z2z::launch_pick_codes(B, w_argmax, a.sample, d_forced, d_next_codes, d_selected, s), "decode_step");
-  }
-  // step 10: online LZW update
-  {
+  const bool fused = B <= 128;                 // one launch for merge + select + LZW update + work list
+  z2z::EntryList el = entry_list(cb);
+  if (fused) {
+    z2z::LogitsPartInfo info{0, 0};
+    rc = logits_call(cb, a, s, &info);
+    if (rc) return rc;
+    z2z::DecodeUpdateArgs u{};
+    u.lpart = reinterpret_cast<const z2z::LogitPartial*>(a.lpart);
+    u.part_stride = info.stride; u.part_count = info.count; u.select = select; u.forced = d_forced;
+    u.next_codes = d_next_codes; u.selected = d_selected; u.lse = a.lse; u.new_entry = w_new;
     z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, s);
-    Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_next_codes, nullptr, w_new, s), "decode_step");
+    Z2Z_CUDA(z2z::launch_decode_update(cb->view, u, el, s), "decode_step");
+  } else {
+    rc = logits_call(cb, a, s);
+    if (rc) return rc;
+    {
+      z2z::ProfScope ps(&cb->prof, z2z::kProfLogitsMerge, 1, s);
+      Z2Z_CUDA(z2z::launch_pick_codes(B, w_argmax, a.sample, d_forced, d_next_codes, d_selected, s), "decode_step");
+    }
+    // step 10: online LZW update
+    {
+      z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, s);
+      Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_next_codes, nullptr, w_new, s), "decode_step");
+    }
+    if (cb->cfg.cap > 0) {
+      z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 4, s);
+      Z2Z_CUDA(z2z::launch_entry_offsets_from_new(cb->view, w_new, el, s), "decode_step");
+      Z2Z_CUDA(z2z::launch_entry_fill(cb->view, 0, nullptr, w_new, el, 0, s), "decode_step");
+      Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 0, s), "decode_step");
+      Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 1, s), "decode_step");
+    }
   }
   // cache update: the at most one new entry per sequence, on both sides
   if (cb->cfg.cap > 0) {
-    z2z::EntryList el = entry_list(cb);
-    {
-      z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 2, s);
-      Z2Z_CUDA(z2z::launch_entry_offsets_from_new(cb->view, w_new, el, s), "decode_step");
-      Z2Z_CUDA(z2z::launch_entry_fill(cb->view, 0, nullptr, w_new, el, 0, s), "decode_step");
-    }
-    const bool tc = cb->use_tensor_cores && z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype);
+    const bool tc = cb->use_tensor_cores && z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype, cb->heads, cb->cfg.M);
     z2z::EncoderArgs g[2];
     g[0] = encoder_args(cb, d_WE, enc_E, d_Eh, d_Eh_f32, B, 0);
     if (!tied) g[1] = encoder_args(cb, d_WU, enc_U, d_Uh, d_Uh_f32, B, 1);
@@ -330,9 +345,6 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
         Z2Z_CUDA(z2z::run_encoder_pass(cb->view, g[1], el, false, &cb->prof, s), "decode_step");
       }
     }
-    z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 2, s);
-    Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 0, s), "decode_step");
-    Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 1, s), "decode_step");
   }
   return Z2Z_OK;
 }

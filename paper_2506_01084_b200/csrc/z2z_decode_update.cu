@@ -1,0 +1,91 @@
+// Middle of the decode step in ONE launch (paper Section 2.3, steps 8-10): finish the joint
+// softmax reductions of every sequence from the per-CTA partials of the logits kernel, select the
+// token (argmax or Gumbel-max sample, or the caller's forced code), apply the online LZW update,
+// and build the work list of new codebook entries for the hyper-encoder pass that follows.
+// One warp per sequence; a single block, so that the list can be compacted without a second
+// launch.
+#include "z2z_common.cuh"
+#include "z2z_internal.h"
+#include "z2z_lzw_dev.cuh"
+
+namespace z2z {
+
+__global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateArgs a, EntryList el) {
+  __shared__ int s_cnt[1024];
+  __shared__ int s_warp[32];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  for (int b = tid; b < 1024; b += blockDim.x) s_cnt[b] = 0;
+  __syncthreads();
+  for (int b = warp; b < cb.B; b += 32) {
+    // ---- merge the partial reductions of hidden row b
+    const LogitPartial* lp = a.lpart + (size_t)b * a.part_stride;
+    RowRed red; red.init();
+    for (int g = lane; g < a.part_count; g += 32) {
+      RowRed o; o.m = lp[g].m; o.s = lp[g].s; o.idx = lp[g].idx; o.gm = lp[g].gm; o.gidx = lp[g].gidx;
+      red.merge(o);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      RowRed o;
+      o.m = __shfl_xor_sync(0xffffffffu, red.m, off);
+      o.s = __shfl_xor_sync(0xffffffffu, red.s, off);
+      o.idx = __shfl_xor_sync(0xffffffffu, red.idx, off);
+      o.gm = __shfl_xor_sync(0xffffffffu, red.gm, off);
+      o.gidx = __shfl_xor_sync(0xffffffffu, red.gidx, off);
+      red.merge(o);
+    }
+    const int amax = red.idx == 0x7fffffff ? -1 : red.idx;
+    const int smp = red.gidx == 0x7fffffff ? -1 : red.gidx;
+    const int sel = a.select == Z2Z_SELECT_GUMBEL ? smp : amax;
+    const int code = a.forced ? a.forced[b] : sel;
+    if (lane == 0) {
+      if (a.lse) a.lse[b] = red.m + logf(red.s);
+      if (a.selected) a.selected[b] = sel;
+      a.next_codes[b] = code;
+    }
+    // ---- online LZW update with the applied code
+    const int created = warp_lzw_step(cb, b, code);
+    if (lane == 0) {
+      if (a.new_entry) a.new_entry[b] = created;
+      s_cnt[b] = created >= 0 ? created + 1 : 0;         // 0: none, else entry number + 1
+    }
+  }
+  __syncthreads();
+  // ---- compact the new entries into the encoder's work list (exclusive scan over sequences)
+  const int mine = tid < cb.B ? s_cnt[tid] : 0;
+  const int flag = mine > 0 ? 1 : 0;
+  int incl = flag;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += x;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = s_warp[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += x;
+    }
+    s_warp[lane] = w;
+  }
+  __syncthreads();
+  const int excl = incl - flag + (warp > 0 ? s_warp[warp - 1] : 0);
+  const int total = s_warp[31];
+  if (tid < cb.B) el.off[tid] = excl;
+  if (tid == 0) { el.off[cb.B] = total; el.off[cb.B + 1] = total < el.chunk ? total : el.chunk; }
+  if (flag && excl < el.chunk) { el.seq[excl] = tid; el.idx[excl] = mine - 1; }
+  for (int e = total + tid; e < el.chunk && e < cb.B; e += blockDim.x) { el.seq[e] = -1; el.idx[e] = 0; }
+  // both caches will hold every entry once the encoder pass that follows has run
+  if (tid < cb.B) { const int n = cb.n[tid]; cb.n_emb[tid] = n; cb.n_emb[cb.B + tid] = n; }
+}
+
+cudaError_t launch_decode_update(const CbView& cb, const DecodeUpdateArgs& a, const EntryList& el,
+                                 cudaStream_t s) {
+  k_decode_update<<<1, 1024, 0, s>>>(cb, a, el);
+  return cudaGetLastError();
+}
+
+}  // namespace z2z

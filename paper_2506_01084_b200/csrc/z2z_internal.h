@@ -38,7 +38,7 @@ struct EncoderArgs {
   int entries;                  // host bound on the entries of this pass (<= chunk)
   int* err;                     // device error word of the tensor-core kernels
 };
-bool encoder_tc_supported(int d, int dff, int dtype);
+bool encoder_tc_supported(int d, int dff, int dtype, int heads, int M);
 bool logits_tc_supported(int d, int dtype);
 // Two encoders (embedding side, unembedding side) run through the same launches.
 cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* groups, int n_groups,
@@ -71,12 +71,26 @@ struct LogitsArgs {
   void* lpart; size_t lpart_bytes;
   int row_base;                 // global index of row 0 of this launch (sampling counter)
 };
-cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, Prof* prof, cudaStream_t s);
 // Partial reduction of one hidden row over a subset of the columns.
 struct __align__(32) LogitPartial { float m, s; int idx; float gm; int gidx; int pad[3]; };
-// Tensor-core (tcgen05) version for bf16; returns cudaErrorNotSupported when the shapes do not fit.
-cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word, Prof* prof,
-                          cudaStream_t s);
+// Where a logits kernel left its partials when the caller merges them itself (decode step).
+struct LogitsPartInfo { int stride, count; };
+// When `info` is given the merge kernel is skipped and the layout of the partials is returned.
+cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, LogitsPartInfo* info, Prof* prof,
+                            cudaStream_t s);
+// Tensor-core (tcgen05) version for bf16 (d % 64 == 0).
+cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word,
+                          LogitsPartInfo* info, Prof* prof, cudaStream_t s);
+
+// ---- z2z_decode_update.cu --------------------------------------------------------------------
+struct DecodeUpdateArgs {
+  const LogitPartial* lpart; int part_stride, part_count;
+  int select;
+  const int32_t* forced;
+  int32_t* next_codes; int32_t* selected; float* lse; int32_t* new_entry;
+};
+cudaError_t launch_decode_update(const CbView& cb, const DecodeUpdateArgs& a, const EntryList& el,
+                                 cudaStream_t s);
 
 // Selected code of the decode step: sample or argmax, overridden by `forced` when given.
 cudaError_t launch_pick_codes(int B, const int32_t* argmax, const int32_t* sample,

@@ -156,7 +156,8 @@ __global__ void k_fill_nan(float* p, int n) {
   if (i < n) p[i] = __int_as_float(0x7fc00000);
 }
 
-cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, Prof* prof, cudaStream_t s) {
+cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, LogitsPartInfo* info, Prof* prof,
+                            cudaStream_t s) {
   const int n_static = (cb.V + kTJ - 1) / kTJ;
   const int tiles_per_seq = (cb.cap + kTJ - 1) / kTJ;
   const int n_tiles = n_static + cb.B * tiles_per_seq;
@@ -176,6 +177,7 @@ cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, Prof* prof, c
     else
       k_logits_simt<__nv_bfloat16><<<dim3(G, row_tiles), 256, 0, s>>>(cb, a, n_static, tiles_per_seq, n_tiles);
   }
+  if (info) { info->stride = G; info->count = G; return cudaGetLastError(); }
   ProfScope ps(prof, kProfLogitsMerge, 1, s);
   k_logits_merge<<<(a.N + 3) / 4, 128, 0, s>>>(a, G);
   return cudaGetLastError();

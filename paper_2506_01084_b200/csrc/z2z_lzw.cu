@@ -8,6 +8,7 @@
 // why the unit of parallelism is the sequence (paper Section 2.4: compression is per document).
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
+#include "z2z_lzw_dev.cuh"
 
 namespace z2z {
 
@@ -23,49 +24,6 @@ __global__ void k_codebook_clear(CbView cb) {
   for (size_t i = tid; i < (size_t)cb.B; i += stride) {
     cb.n[i] = 0; cb.prev[i] = -1; cb.status[i] = 0; cb.n_emb[i] = 0; cb.n_emb[cb.B + i] = 0;
   }
-}
-
-// Result of a warp probe.
-struct Probe {
-  int found;        // entry number, or -1
-  int slot;         // if absent: first empty slot in probe order (-1: table full)
-};
-
-// All 32 lanes must call this together.
-__device__ __forceinline__ Probe warp_probe(const unsigned long long* __restrict__ table,
-                                            int n_slots, uint32_t prefix, uint32_t token) {
-  const int lane = threadIdx.x & 31;
-  const unsigned long long key = pack_slot(prefix, token, 0) >> 16;
-  int bucket = (int)(hash_pair(prefix, token) & (uint32_t)(n_slots - 1)) & ~(kBucket - 1);
-  Probe r{-1, -1};
-  for (int it = 0; it < n_slots / kBucket; ++it) {          // bounded: at most the whole table
-    unsigned long long s = table[bucket + lane];
-    unsigned hit = __ballot_sync(0xffffffffu, (s >> 16) == key && s != kEmptySlot);
-    if (hit) {
-      int src = __ffs(hit) - 1;
-      unsigned long long v = __shfl_sync(0xffffffffu, s, src);
-      r.found = (int)(v & 0xffffu);
-      return r;
-    }
-    unsigned empty = __ballot_sync(0xffffffffu, s == kEmptySlot);
-    if (empty) { r.slot = bucket + __ffs(empty) - 1; return r; }
-    bucket = (bucket + kBucket) & (n_slots - 1);
-  }
-  return r;
-}
-
-// Write entry k = phrase(w) ++ c.  Lanes 0..M-1 each write one constituent.
-__device__ __forceinline__ void warp_write_entry(const CbView& cb, int b, int k, int w, int wlen,
-                                                 int c) {
-  const int lane = threadIdx.x & 31;
-  int32_t* dst = cb.cons + ((size_t)b * cb.cap + k) * cb.M;
-  if (lane < cb.M) {
-    int v = -1;
-    if (lane < wlen) v = (w < cb.V) ? w : cb.cons[((size_t)b * cb.cap + (w - cb.V)) * cb.M + lane];
-    else if (lane == wlen) v = c;
-    dst[lane] = v;
-  }
-  if (lane == 0) cb.len[(size_t)b * cb.cap + k] = (uint8_t)(wlen + 1);
 }
 
 // Prompt compression (Section 2.1; Section 2.3 step 2).  grid = ceil(B / warps per block).
@@ -136,47 +94,8 @@ __global__ void __launch_bounds__(128) k_lzw_step(CbView cb, const int32_t* __re
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (b >= cb.B) return;
   if (active && !active[b]) { if (lane == 0 && new_entry) new_entry[b] = -1; return; }
-  unsigned long long* table = cb.hash + (size_t)b * cb.n_slots;
-  const int z = new_codes[b];
-  const int n = cb.n[b];
-  const int prev = cb.prev[b];
-  int created = -1;
-  int st = 0;
-  bool ok = !(z < 0 || z > cb.V + n);
-  int plen = 0;
-  if (prev >= 0) plen = prev < cb.V ? 1 : (int)cb.len[(size_t)b * cb.cap + (prev - cb.V)];
-  const bool self_ref = ok && (z == cb.V + n);       // the code this very step would create
-  if (self_ref && !(prev >= 0 && plen < cb.M && n < cb.cap)) ok = false;
-  if (ok) {
-    int first;
-    if (self_ref) first = prev < cb.V ? prev : cb.cons[((size_t)b * cb.cap + (prev - cb.V)) * cb.M];
-    else first = z < cb.V ? z : cb.cons[((size_t)b * cb.cap + (z - cb.V)) * cb.M];
-    if (prev >= 0 && plen < cb.M && n < cb.cap) {
-      Probe p = warp_probe(table, cb.n_slots, (uint32_t)prev, (uint32_t)first);
-      if (p.found < 0) {
-        if (p.slot >= 0) {
-          if (lane == 0) table[p.slot] = pack_slot((uint32_t)prev, (uint32_t)first, (uint32_t)n);
-          warp_write_entry(cb, b, n, prev, plen, first);
-          created = n;
-          if (n + 1 >= cb.cap) st |= Z2Z_ST_CAP_FROZEN;
-        } else {
-          st |= Z2Z_ST_TABLE_FULL;
-        }
-      } else if (self_ref) {
-        ok = false;                                    // that phrase already has another id
-      }
-    }
-  }
-  if (lane == 0) {
-    if (!ok) {
-      st |= Z2Z_ST_BAD_TOKEN;                          // state stays as it was
-    } else {
-      cb.prev[b] = z;
-      if (created >= 0) cb.n[b] = n + 1;
-    }
-    if (new_entry) new_entry[b] = ok ? created : -1;
-    if (st) atomicOr(&cb.status[b], st);
-  }
+  const int created = warp_lzw_step(cb, b, new_codes[b]);
+  if (lane == 0 && new_entry) new_entry[b] = created;
 }
 
 cudaError_t launch_codebook_clear(const CbView& cb, cudaStream_t s) {

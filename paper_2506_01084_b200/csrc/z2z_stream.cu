@@ -45,7 +45,9 @@ struct Job {
   int kb0, kb1;          // k-step range
   long long slot;        // GEMM: partial slot
   int col0, nvalid, owner, k0;   // logits: first column id, valid rows, owning sequence, first entry
-  int rt;                // logits: hidden-row tile
+  int rt;                // hidden-row tile
+  int nrows;             // weight rows in this job (the MMA's N), multiple of 16
+  int wbox;              // rows per TMA box of W (nrows / wbox boxes per k block)
 };
 
 // ---- GEMM schedule ------------------------------------------------------------------------------
@@ -72,44 +74,53 @@ struct GemmSched {
     j.amap = g; j.wmap = g; j.arow = j.rt * 128;
     j.wrow = (rem - g * p.tiles_per_group) * NT;
     j.slot = tile + c;
+    j.nrows = NT; j.wbox = NT;
     u += j.kb1 - j.kb0;
     return true;
   }
 };
 
 // ---- logits schedule ----------------------------------------------------------------------------
+// Columns are dealt in granules of kLogitGran rows: first the granules of W_U, then those of the
+// visible rows of each sequence's U_h.  Every CTA owns the same number of granules (+-1); a job
+// is a run of up to NT / kLogitGran granules inside one segment (W_U, or one sequence).
 struct LogitSched {
   const StreamLogitsParams& p;
-  const int* pref;       // shared: prefix of ragged tile counts, [B + 1]
+  const int* pref;       // shared: prefix of per-sequence granule counts, [B + 1]
   long long u, u1;
   int n_static, vt, ksteps;
   __device__ LogitSched(const StreamLogitsParams& pp, const int* s_pref, int vt_, int NT) : p(pp), pref(s_pref) {
-    n_static = (p.cb.V + NT - 1) / NT;
+    n_static = (p.cb.V + kLogitGran - 1) / kLogitGran;
     vt = vt_;
     ksteps = p.ksteps;
     const long long U = (long long)p.row_tiles * vt, G = gridDim.x, c = blockIdx.x;
     u = c * U / G;
     u1 = (c + 1) * U / G;
+    (void)NT;
   }
   __device__ bool next(Job& j, int NT) {
     if (u >= u1) return false;
     j.rt = (int)(u / vt);
     const int v = (int)(u - (long long)j.rt * vt);
-    j.amap = 0; j.arow = j.rt * 128; j.kb0 = 0; j.kb1 = ksteps; j.slot = 0;
+    j.amap = 0; j.arow = j.rt * 128; j.kb0 = 0; j.kb1 = ksteps; j.slot = 0; j.wbox = kLogitGran;
+    int remaining, total_rows, g0;
     if (v < n_static) {
-      j.wmap = 0; j.wrow = v * NT; j.col0 = v * NT; j.owner = -1; j.k0 = 0;
-      j.nvalid = p.cb.V - j.col0 < NT ? p.cb.V - j.col0 : NT;
+      g0 = v; remaining = n_static - v; total_rows = p.cb.V;
+      j.wmap = 0; j.wrow = g0 * kLogitGran; j.col0 = g0 * kLogitGran; j.owner = -1; j.k0 = 0;
     } else {
       const int x = v - n_static;
       int lo = 0, hi = p.cb.B - 1;                 // last b with pref[b] <= x
       while (lo < hi) { int mid = (lo + hi + 1) >> 1; if (pref[mid] <= x) lo = mid; else hi = mid - 1; }
-      j.owner = lo;
-      j.k0 = (x - pref[lo]) * NT;
+      g0 = x - pref[lo]; remaining = pref[lo + 1] - pref[lo] - g0; total_rows = p.cb.n[lo];
+      j.owner = lo; j.k0 = g0 * kLogitGran;
       j.wmap = 1; j.wrow = lo * p.cb.cap + j.k0; j.col0 = p.cb.V + j.k0;
-      const int n = p.cb.n[lo];
-      j.nvalid = n - j.k0 < NT ? n - j.k0 : NT;
     }
-    ++u;
+    int ng = NT / kLogitGran;
+    if (remaining < ng) ng = remaining;
+    if (u1 - u < ng) ng = (int)(u1 - u);
+    j.nrows = ng * kLogitGran;
+    j.nvalid = total_rows - g0 * kLogitGran < j.nrows ? total_rows - g0 * kLogitGran : j.nrows;
+    u += ng;
     return true;
   }
 };
@@ -121,7 +132,7 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
                                               const CUtensorMap* const* amaps,
                                               const CUtensorMap* const* wmaps) {
   const uint32_t a_part_bytes = (uint32_t)KSB * a_box_rows * 128;
-  const uint32_t stage_bytes = a_parts * a_part_bytes + (uint32_t)KSB * NT * 128;
+  const uint32_t stage_bytes = a_parts * a_part_bytes + (uint32_t)KSB * NT * 128;   // smem stride of a stage
   const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
   int stage = 0; uint32_t phase = 0;
   Job j;
@@ -129,7 +140,7 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
     for (int ks = j.kb0; ks < j.kb1; ++ks) {
       if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) return;
       const uint32_t full = smem_u32(&ctrl->full[stage]);
-      mbar_expect_tx(full, stage_bytes);
+      mbar_expect_tx(full, a_parts * a_part_bytes + (uint32_t)KSB * j.nrows * 128);
       const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
       for (int part = 0; part < a_parts; ++part)
 #pragma unroll
@@ -138,8 +149,9 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
                       (ks * KSB + i) * 64, j.arow + part * a_part_row, full, pol_a);
 #pragma unroll
       for (int i = 0; i < KSB; ++i)
-        tma_load_2d(sb + a_parts * a_part_bytes + i * NT * 128, wmaps[j.wmap], (ks * KSB + i) * 64,
-                    j.wrow, full, pol_w);
+        for (int r0 = 0; r0 < j.nrows; r0 += j.wbox)
+          tma_load_2d(sb + a_parts * a_part_bytes + i * NT * 128 + r0 * 128, wmaps[j.wmap],
+                      (ks * KSB + i) * 64, j.wrow + r0, full, pol_w);
       if (++stage == STAGES) { stage = 0; phase ^= 1u; }
     }
   }
@@ -150,11 +162,11 @@ __device__ __forceinline__ void mma_role(Sched& sched, Ctrl* ctrl, uint32_t stag
                                          int a_box_rows, uint32_t tmem_base) {
   const uint32_t a_part_bytes = (uint32_t)KSB * a_box_rows * 128;
   const uint32_t stage_bytes = a_parts * a_part_bytes + (uint32_t)KSB * NT * 128;
-  constexpr uint32_t idesc = idesc_bf16_f32(128, NT);
   int stage = 0; uint32_t phase = 0;
   uint32_t job_i = 0;
   Job j;
   while (sched.next(j, NT)) {
+    const uint32_t idesc = idesc_bf16_f32(128, j.nrows);
     const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
     if (!mbar_wait(smem_u32(&ctrl->acc_empty[buf]), aph ^ 1u, &ctrl->abort)) return;
     tc_fence_after();
@@ -284,13 +296,13 @@ k_stream_logits(const StreamLogitsParams p, const __grid_constant__ CUtensorMap 
   const uint32_t stage_base = smem_u32(sm + 1024 + 5120);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   setup_barriers<STAGES>(ctrl);
-  for (int b = threadIdx.x; b < p.cb.B; b += kThreads) s_pref[b + 1] = (p.cb.n[b] + NT - 1) / NT;
+  for (int b = threadIdx.x; b < p.cb.B; b += kThreads) s_pref[b + 1] = (p.cb.n[b] + kLogitGran - 1) / kLogitGran;
   if (warp == 0 && lane == 0) { prefetch_tmap(&tmH); prefetch_tmap(&tmWU); prefetch_tmap(&tmUh); }
   __syncthreads();
   if (threadIdx.x == 0) {
     s_pref[0] = 0;
     for (int b = 0; b < p.cb.B; ++b) s_pref[b + 1] += s_pref[b];
-    ctrl->vt = (p.cb.V + NT - 1) / NT + s_pref[p.cb.B];
+    ctrl->vt = (p.cb.V + kLogitGran - 1) / kLogitGran + s_pref[p.cb.B];
     if (blockIdx.x == 0) *p.vt_out = ctrl->vt;
   }
   if (warp == 2) { tmem_alloc(smem_u32(&ctrl->tmem_base), tmem_cols(NT)); tmem_relinquish(); }
@@ -355,7 +367,7 @@ k_stream_logits(const StreamLogitsParams p, const __grid_constant__ CUtensorMap 
       const int rows_here = a.N - cur_rt * 128;
       if (q * 32 < rows_here && __any_sync(0xffffffffu, limit > 0)) {
 #pragma unroll 1
-        for (int c0 = 0; c0 < NT; c0 += 32) {
+        for (int c0 = 0; c0 < j.nrows; c0 += 32) {
           if (!__any_sync(0xffffffffu, limit > c0)) break;
           uint32_t v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * NT + c0, v);
@@ -509,8 +521,8 @@ static cudaError_t launch_logits_t(const StreamLogitsParams& p, const CUtensorMa
 
 bool logits_tc_supported(int d, int dtype) { return dtype == Z2Z_DTYPE_BF16 && d % 64 == 0; }
 
-cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word, Prof* prof,
-                          cudaStream_t s) {
+cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word,
+                          LogitsPartInfo* info, Prof* prof, cudaStream_t s) {
   static int n_sm = 0;
   if (!n_sm) {
     int dev = 0;
@@ -528,21 +540,25 @@ cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, i
   if ((size_t)a.N * p.part_stride * sizeof(LogitPartial) > a.lpart_bytes) return cudaErrorMemoryAllocation;
   CUtensorMap maps[3];
   if (!make_tmap_bf16(&maps[0], a.hidden, a.N, a.d, p.a_box_rows)) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16(&maps[1], a.WU, cb.V, a.d, kLogitNT)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16(&maps[1], a.WU, cb.V, a.d, kLogitGran)) return cudaErrorInvalidValue;
   if (cb.cap > 0) {
-    if (!make_tmap_bf16(&maps[2], a.Uh, (long long)cb.B * cb.cap, a.d, kLogitNT)) return cudaErrorInvalidValue;
+    if (!make_tmap_bf16(&maps[2], a.Uh, (long long)cb.B * cb.cap, a.d, kLogitGran)) return cudaErrorInvalidValue;
   } else {
     maps[2] = maps[1];
   }
   // every CTA must own at least one unit: the static tiles alone give a lower bound on the units
-  long long units_lb = (long long)p.row_tiles * ((cb.V + kLogitNT - 1) / kLogitNT);
+  long long units_lb = (long long)p.row_tiles * ((cb.V + kLogitGran - 1) / kLogitGran);
   const int grid = units_lb < n_sm ? (int)units_lb : n_sm;
   p.part_stride = (grid + p.row_tiles - 1) / p.row_tiles + 2;
-  return launch_stream_logits(p, maps, grid, prof, s);
+  if (info) {
+    if (p.row_tiles != 1) return cudaErrorInvalidValue;
+    info->stride = p.part_stride; info->count = grid;
+  }
+  return launch_stream_logits(p, maps, grid, info == nullptr, prof, s);
 }
 
-cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, Prof* prof,
-                                 cudaStream_t s) {
+cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, bool merge,
+                                 Prof* prof, cudaStream_t s) {
   constexpr int NT = kLogitNT, KSB = kLogitKSB;
   const LogitsArgs& a = p.la;
   if (a.target_logit) {
@@ -558,7 +574,7 @@ cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap*
     else if (st >= 4) e = launch_logits_t<NT, KSB, 4>(p, maps, grid, s);
     else e = cudaErrorInvalidConfiguration;
   }
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || !merge) return e;
   ProfScope ps(prof, kProfLogitsMerge, 1, s);
   k_stream_logits_merge<<<(a.N + 3) / 4, 128, 0, s>>>(p, grid);
   return cudaGetLastError();

@@ -11,6 +11,7 @@ namespace z2z {
 constexpr int kMaxStages = 8;
 constexpr int kGemmNT = 128, kGemmKSB = 1;      // weight rows per tile, 64-wide k blocks per stage
 constexpr int kLogitNT = 128, kLogitKSB = 1;
+constexpr int kLogitGran = 16;                  // rows per TMA box / scheduling granule of the logits kernel
 
 // Stream-K GEMM over `groups` independent problems of identical shape (the two hyper-encoders).
 // The unit space is (group, tile, k-step); CTA c of G owns units [floor(cU/G), floor((c+1)U/G)).
@@ -41,7 +42,7 @@ struct StreamLogitsParams {
 
 bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows);
 cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s);
-cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, Prof* prof,
-                                 cudaStream_t s);
+cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, bool merge,
+                                 Prof* prof, cudaStream_t s);
 
 }  // namespace z2z

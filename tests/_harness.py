@@ -21,8 +21,10 @@ def f64(t: torch.Tensor) -> np.ndarray:
 class Pair:
     """One workload instantiated on both sides."""
 
-    def __init__(self, w: si.Workload, seed: int, generic_encoder: bool = True, device="cuda:0"):
+    def __init__(self, w: si.Workload, seed: int, generic_encoder: bool = True, device="cuda:0",
+                 tensor_cores: bool = True):
         self.w, self.dev = w, torch.device(device)
+        self.tensor_cores = tensor_cores
         self.tokens = si.make_tokens(w, seed)                              # [B, T] int32
         self.W_E, self.W_U = si.make_tables(w, seed)
         self.enc_E = si.make_encoder(w, seed * 3 + 1, generic=generic_encoder)
@@ -36,6 +38,8 @@ class Pair:
         self.cfg = zb.make_config(w.V, w.d, w.M, w.cap, w.B, w.dtype, w.enc_layers, w.heads,
                                   w.dff, w.tied)
         self.cb = zb.Codebook(self.cfg, device)
+        if not tensor_cores:
+            zb.z2z_set_tensor_cores(self.cb, False)      # CUDA-core kernels as an on-GPU cross-check
         self.g_WE = self.W_E.to(self.dev)
         self.g_WU = self.g_WE if w.tied else self.W_U.to(self.dev)
         self.g_encE_t = [t.to(self.dev) for t in self.enc_E]

@@ -230,8 +230,8 @@ def test_hyper_embed_explicit_ranges_and_incremental():
 # ------------------------------------------------------------------------------------------------
 # Joint logits and reductions
 # ------------------------------------------------------------------------------------------------
-def _logits_case(w, seed, rows_per_seq, causal, select, temperature=0.8):
-    p = Pair(w, seed=seed, generic_encoder=False)
+def _logits_case(w, seed, rows_per_seq, causal, select, temperature=0.8, tensor_cores=True):
+    p = Pair(w, seed=seed, generic_encoder=False, tensor_cores=tensor_cores)
     codes, clen, after = p.gpu_encode()
     ocodes, oafter = p.oracle.prefill([p.tokens[b].tolist() for b in range(w.B)])
     n = [bk.n() for bk in p.oracle.books]
@@ -305,8 +305,8 @@ def test_dynamic_logits_no_hypertokens_is_plain_lm_head():
 # ------------------------------------------------------------------------------------------------
 # Whole decode step, following the GPU's selections inside the oracle's top-2 gap
 # ------------------------------------------------------------------------------------------------
-def _decode_follow(w, seed, select, steps=None, forced_every=0):
-    p = Pair(w, seed=seed)
+def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=True):
+    p = Pair(w, seed=seed, tensor_cores=tensor_cores)
     _prefill_both(p)
     for b in range(w.B):
         p.force_caches_from_oracle(b, 0, p.oracle.books[b].n())
@@ -376,3 +376,31 @@ def test_decode_step_tiny_config_sampling_and_forcing():
 def test_decode_step_small(w):
     _decode_follow(w, 23, zb.SELECT_ARGMAX, steps=w.steps)
     _decode_follow(w, 24, zb.SELECT_GUMBEL, steps=6, forced_every=2)
+
+
+# ------------------------------------------------------------------------------------------------
+# Second on-GPU path: the CUDA-core kernels on a bf16 session (tensor cores switched off), and
+# shapes that exercise more than one 128-row tile of the tensor-core kernels
+# ------------------------------------------------------------------------------------------------
+def test_cuda_core_kernels_on_bf16_session():
+    p = Pair(SMALL_BF16, seed=5, tensor_cores=False)
+    _, worst = _prefill_both(p)
+    assert worst <= TOL
+    _logits_case(SMALL_BF16, 11, [70, 0, 5], True, 1, tensor_cores=False)
+    _decode_follow(SMALL_BF16, 23, zb.SELECT_ARGMAX, steps=6, tensor_cores=False)
+
+
+MID_BF16 = si.Workload("mid_bf16", V=5000, d=384, dtype="bf16", B=40, T=96, M=3, cap=64,
+                       zipf_s=1.1, copy_p=0.4, seg_min=3, seg_max=10, steps=4, enc_layers=2,
+                       enc_heads=3, enc_dff=768)
+
+
+def test_tensor_core_kernels_many_rows_and_sequences():
+    # 40 sequences: decode rows 120 (> 64: hi and lo run as two MMAs), prefill passes span many
+    # 128-row tiles, logits with several hundred hidden rows span several row tiles
+    p = Pair(MID_BF16, seed=31)
+    _, worst = _prefill_both(p)
+    print(f"mid_bf16: max |hyper-embedding error| = {worst:.3e}")
+    worst = _logits_case(MID_BF16, 32, [9] * MID_BF16.B, True, 1)
+    print(f"mid_bf16: max |logit error| = {worst:.3e}")
+    _decode_follow(MID_BF16, 33, zb.SELECT_ARGMAX, steps=4)

@@ -183,6 +183,30 @@ int32_t z2z_profile(z2z_codebook* cb, int32_t enable);
 int32_t z2z_profile_read(z2z_codebook* cb, int32_t n_classes, double* h_ms, int64_t* h_launches,
                          z2z_stream stream);
 
+/* Joint logits with log-sum-exp, argmax and maximum for callers that cannot allocate device
+ * memory (the paper has no counterpart; this is a deployment aid).  Some callers cannot call
+ * cudaMalloc or a framework allocator: a plug-in in a serving process that gave out all device
+ * memory at start-up, a callback that must not enter the allocator, a process already at its
+ * memory limit.  They cannot provide the session workspace either, so this call takes no handle:
+ * the per-CTA partial reductions live in an array of 2 MiB that is part of the library image
+ * (every GPU that loads the library holds it until the process exits).  The library allocates
+ * nothing in this call.
+ *   d_hidden [N, d], d_row_seq [N] or NULL (row r belongs to sequence r), d_WU [V, d],
+ *   d_Uh [B, cap, d], all in `dtype`; d_n_hyper [B] DEVICE array: visible hypertokens of each
+ *   sequence; d_lse / d_argmax / d_max_logit [N] out, each may be NULL.
+ * Limits: N <= 1024 rows per call (larger N returns Z2Z_ERR_INVALID_ARG and z2z_last_error says
+ * so); the other limits are those of z2z_config.  Same arithmetic as the CUDA-core path of
+ * z2z_dynamic_logits (fp32 accumulation).
+ * The first call on a device looks up the array's address for that device: make that call with
+ * the device current and outside any stream capture.  All calls on a device share the array and
+ * leave their partials in it (nothing there needs clearing between calls); calls that overlap on
+ * one GPU, e.g. on two streams, race on it and must be ordered by the caller.                  */
+int32_t z2z_logits_static_scratch(const void* d_hidden, int32_t N, const int32_t* d_row_seq,
+                                  const int32_t* d_n_hyper, const void* d_WU, const void* d_Uh,
+                                  int32_t V, int32_t d, int32_t B, int32_t cap, int32_t dtype,
+                                  float* d_lse, int32_t* d_argmax, float* d_max_logit,
+                                  z2z_stream stream);
+
 /* Frees the host handle (never the workspace). */
 int32_t z2z_codebook_destroy(z2z_codebook* cb);
 

@@ -24,7 +24,7 @@ CACHE_EMBED, CACHE_UNEMBED = 0, 1
 EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lzw_step",
            "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
            "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error", "z2z_profile",
-           "z2z_profile_read", "z2z_set_tensor_cores"]
+           "z2z_profile_read", "z2z_set_tensor_cores", "z2z_logits_static_scratch"]
 
 
 class Config(C.Structure):
@@ -213,3 +213,24 @@ def z2z_profile_read(cb: Codebook):
 
 def z2z_set_tensor_cores(cb: Codebook, enable: bool):
     _check(lib().z2z_set_tensor_cores(cb.handle, C.c_int32(1 if enable else 0)))
+
+
+def z2z_logits_static_scratch(hidden: torch.Tensor, row_seq: Optional[torch.Tensor],
+                              n_hyper: torch.Tensor, W_U: torch.Tensor,
+                              U_h: Optional[torch.Tensor], cap: int,
+                              lse: Optional[torch.Tensor], argmax: Optional[torch.Tensor],
+                              max_logit: Optional[torch.Tensor]):
+    """Joint logits + LSE / argmax / maximum without a session handle or workspace: for callers
+    that cannot allocate device memory.  The partial reductions live in a fixed 2 MiB array
+    inside the library (at most 1024 hidden rows per call).  ``n_hyper`` is a device int32 tensor
+    [B] with the visible hypertokens of each sequence.  Calls that overlap on one GPU race on the
+    shared array; the first call on a device should be made outside stream capture."""
+    N, d = hidden.shape
+    V = W_U.shape[0]
+    B = n_hyper.shape[0]
+    dt = DTYPE_FP32 if hidden.dtype == torch.float32 else DTYPE_BF16
+    _check(lib().z2z_logits_static_scratch(_ptr(hidden), C.c_int32(N), _ptr(row_seq),
+                                           _ptr(n_hyper), _ptr(W_U), _ptr(U_h), C.c_int32(V),
+                                           C.c_int32(d), C.c_int32(B), C.c_int32(cap),
+                                           C.c_int32(dt), _ptr(lse), _ptr(argmax),
+                                           _ptr(max_logit), _stream()))

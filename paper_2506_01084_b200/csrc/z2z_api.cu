@@ -126,6 +126,11 @@ int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s, z2z::Logits
 
 }  // namespace
 
+namespace z2z {
+// Lets entry points in other files leave their message where z2z_last_error finds it.
+void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
+}  // namespace z2z
+
 extern "C" {
 
 const char* z2z_last_error(void) { return g_err; }

@@ -8,6 +8,9 @@
 
 namespace z2z {
 
+// ---- z2z_api.cu ------------------------------------------------------------------------------
+void set_last_error(const char* msg);      // text returned by z2z_last_error on this thread
+
 // ---- z2z_lzw.cu ------------------------------------------------------------------------------
 cudaError_t launch_codebook_clear(const CbView& cb, cudaStream_t s);
 cudaError_t launch_lzw_encode(const CbView& cb, const int32_t* tokens, const int32_t* lens,

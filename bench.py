@@ -48,55 +48,63 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and clock-event (throttle) reasons through NVML, the library nvidia-smi
+    itself reads, from a thread while the timed region runs (nvidia-smi's own loop cannot sample
+    faster than its start-up time, and the timed region may last only tens of milliseconds).
+    Reading only: nothing is set."""
 
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-
-    def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.index, self.period, self.samples = index, period_s, []
+        self._stop = threading.Event()
+        self.thread, self.err = None, None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
-                stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.index
+            if vis:
+                ent = [v.strip() for v in vis.split(",") if v.strip()][idx]
+                self.h = (pynvml.nvmlDeviceGetHandleByIndex(int(ent)) if ent.isdigit()
+                          else pynvml.nvmlDeviceGetHandleByUUID(ent))
+            else:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.nv = pynvml
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:                      # no NVML: report that instead of clocks
+            self.err = f"NVML unavailable: {type(e).__name__}"
+            return
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                rs = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                self.samples.append((float(mhz), int(rs), pw))
+            except Exception:
+                pass
+            time.sleep(self.period)
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            pass
-        sm, mx, reasons = [], [], set()
-        for ln in self.lines:
-            f = [x.strip() for x in ln.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
-            except ValueError:
-                continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
-                                "sw_power_cap"), f[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        busy = [s for s in sm if s > 0]
-        return {"sm_mhz": float(np.median(busy)) if busy else None,
-                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
-                "samples": len(sm)}
+        if self.thread is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [self.err or "not sampled"]}
+        self._stop.set()
+        self.thread.join(timeout=2)
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
+        reasons = sorted(k for k, bit in names.items() if any(r & bit for _, r, _ in self.samples))
+        sm = [m for m, _, _ in self.samples if m > 0]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(sm),
+                "power_w_max": max((p for _, _, p in self.samples), default=None)}
 
 
 # --------------------------------------------------------------------------------------------------
@@ -113,6 +121,33 @@ def encoder_gemm_bytes(w: si.Workload) -> float:
     es = 2 if w.dtype == "bf16" else 4
     per_layer = 4 * w.d * w.d + 2 * w.d * w.dff
     return es * per_layer * w.enc_layers * (1 if w.tied else 2)
+
+
+def kernel_source_digest() -> str:
+    """Digest of the sources of the streaming kernels; an ncu traffic figure only counts while it
+    matches the code that produced it."""
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2506_01084_b200", "csrc")
+    for f in ("z2z_stream.cu", "z2z_stream.h", "z2z_sm100.cuh"):
+        with open(os.path.join(d, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_traffic(kernel_class: str, workload: str):
+    """DRAM bytes per launch (read + write) of a kernel class from the committed ncu summary
+    profiles/dram_traffic.txt, or None when there is no figure for the present kernel sources.
+    Line format:  class workload source-digest bytes-per-launch"""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    dig = kernel_source_digest()
+    for ln in open(path):
+        f = ln.split("#")[0].split()
+        if len(f) >= 4 and f[0] == kernel_class and f[1] == workload and f[2] == dig:
+            return float(f[3])
+    return None
 
 
 # --------------------------------------------------------------------------------------------------
@@ -254,21 +289,26 @@ def run_ours(args, rank: int, world: int):
     mean_hyper = 0.5 * (n_after + n_after2)     # hyper rows visible during the profiled pass
     classes = {"logits": logits_bytes(w, mean_hyper), "encoder_gemm": encoder_gemm_bytes(w)}
     dom = max(classes, key=lambda k: cls_ms.get(k, 0.0))
-    per_launch_group_ms = cls_ms[dom] / K       # time of that class per step
-    achieved = classes[dom] / (per_launch_group_ms * 1e-3) / 1e9 if per_launch_group_ms > 0 else 0.0
-    roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": pk["hbm_gbs"],
-            "unit": "GB/s", "frac": achieved / pk["hbm_gbs"], "traffic": None,
-            "peak_source": pk["source"],
-            "algorithmic_bytes_per_step": classes[dom], "ms_per_step": per_launch_group_ms,
-            "launches_per_step": cls_launches[dom] / K,
-            "timing": "CUDA events around each launch of the class, second pass of K steps",
+
+    def class_roof(k):
+        n_launch = max(cls_launches[k], 1)
+        ms_launch = cls_ms[k] / n_launch                     # average launch duration
+        by_launch = classes[k] * K / n_launch                # algorithmic bytes per launch
+        gbs = by_launch / max(ms_launch, 1e-9) / 1e6
+        return {"algorithmic_bytes_per_launch": by_launch, "launches_per_step": n_launch / K,
+                "us_per_launch": ms_launch * 1e3, "ms_per_step": cls_ms[k] / K, "gbs": gbs,
+                "frac": gbs / pk["hbm_gbs"], "traffic": ncu_traffic(k, w.name)}
+
+    cr = {k: class_roof(k) for k in classes}
+    roof = {"bound": "hbm", "kernel": {"logits": "k_stream_logits", "encoder_gemm": "k_stream_gemm"}[dom],
+            "achieved": cr[dom]["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
+            "frac": cr[dom]["frac"], "traffic": cr[dom]["traffic"],
+            "peak_source": pk["source"] + " (STREAM-style copy, burst)",
+            "timing": "CUDA events around every launch of the kernel on the launching stream, in a "
+                      "second pass of K steps; achieved = algorithmic bytes per launch / average "
+                      "launch duration",
             "per_class_ms_per_step": {k: v / K for k, v in cls_ms.items()},
-            "logits": {"bytes": classes["logits"], "ms": cls_ms["logits"] / K,
-                       "gbs": classes["logits"] / max(cls_ms["logits"] / K, 1e-9) / 1e6,
-                       "frac": classes["logits"] / max(cls_ms["logits"] / K, 1e-9) / 1e6 / pk["hbm_gbs"]},
-            "encoder_gemm": {"bytes": classes["encoder_gemm"], "ms": cls_ms["encoder_gemm"] / K,
-                             "gbs": classes["encoder_gemm"] / max(cls_ms["encoder_gemm"] / K, 1e-9) / 1e6,
-                             "frac": classes["encoder_gemm"] / max(cls_ms["encoder_gemm"] / K, 1e-9) / 1e6 / pk["hbm_gbs"]}}
+            "logits": cr["logits"], "encoder_gemm": cr["encoder_gemm"]}
     es = 2 if w.dtype == "bf16" else 4
     line = {
         "metric": METRIC, "value": bt_dev / (dev_ms * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -350,7 +390,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="phi3_mini_head", choices=list(si.WORKLOADS))

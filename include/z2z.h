@@ -167,8 +167,12 @@ int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t*
 
 /* Kernel family used for bf16 sessions (no counterpart in the paper; cross-checking aid).
  * enable = 1 (default): tcgen05 tensor-core kernels wherever the shapes allow (d and enc_dff
- * multiples of 128).  enable = 0: the CUDA-core kernels, which keep activations in fp32 and are
- * the path fp32 sessions always take.  Both produce results within the stated tolerance.        */
+ * multiples of 128), the joint-logits kernel chosen by the number of hidden rows (weight
+ * streaming for decode batches, CTA-pair tiles from 2048 rows on).  enable = 0: the CUDA-core
+ * kernels, which keep activations in fp32 and are the path fp32 sessions always take.
+ * enable = 2 + 16 * s: as 1, but z2z_dynamic_logits always takes the CTA-pair kernel, with s
+ * column strips per row tile when 1 <= s <= 8 (s = 0: chosen by shape).  All produce results
+ * within the stated tolerance.                                                                 */
 int32_t z2z_set_tensor_cores(z2z_codebook* cb, int32_t enable);
 
 /* Launch accounting and per-kernel-class timing (no counterpart in the paper; measurement aid).

@@ -211,8 +211,11 @@ def z2z_profile_read(cb: Codebook):
             {k: int(cnt[i]) for i, k in enumerate(PROFILE_CLASSES)})
 
 
-def z2z_set_tensor_cores(cb: Codebook, enable: bool):
-    _check(lib().z2z_set_tensor_cores(cb.handle, C.c_int32(1 if enable else 0)))
+def z2z_set_tensor_cores(cb: Codebook, enable):
+    """0 / False: CUDA-core kernels; 1 / True: tensor-core kernels chosen by shape;
+    2 + 16 * s: the CTA-pair logits kernel for every z2z_dynamic_logits call, with s column strips
+    (0: chosen by shape)."""
+    _check(lib().z2z_set_tensor_cores(cb.handle, C.c_int32(int(enable))))
 
 
 def z2z_logits_static_scratch(hidden: torch.Tensor, row_seq: Optional[torch.Tensor],

@@ -6,6 +6,7 @@
 
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
+#include "z2z_stream.h"
 
 struct z2z_codebook {
   z2z_config cfg;
@@ -14,7 +15,8 @@ struct z2z_codebook {
   size_t ws_bytes;
   z2z::CbView view;
   int dff, heads;
-  int use_tensor_cores;
+  int use_tensor_cores;      // 0: CUDA cores, 1: tensor cores (kernel by shape), 2: prompt-scoring kernel always
+  int prefill_strips;        // > 0: fixed number of column strips in the prompt-scoring kernel
   z2z::Prof prof;
 };
 
@@ -94,15 +96,29 @@ int check_encoder(z2z_codebook* cb, const z2z_encoder_weights* enc) {
   return Z2Z_OK;
 }
 
+// Rows at or above which the prompt-scoring kernel (CTA pairs, 256 x 256 tiles) takes over from
+// the weight-streaming kernel: enough row tiles to give every cluster work.
+constexpr int kPrefillMinRows = 2048;
+
 int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s, z2z::LogitsPartInfo* info = nullptr) {
   // rows are processed in blocks so that the partial-reduction scratch stays bounded
   const int N = a.N;
   const size_t esz = cb->cfg.dtype == Z2Z_DTYPE_FP32 ? 4 : 2;
   const size_t ldbg = (size_t)cb->cfg.V + cb->cfg.cap;
-  for (int r0 = 0; r0 < N; r0 += z2z::kLogitRowChunk) {
+  const bool tc = cb->use_tensor_cores && z2z::logits_tc_supported(cb->cfg.d, cb->cfg.dtype);
+  const bool prefill = tc && info == nullptr && z2z::prefill_logits_supported(cb->cfg.d, cb->cfg.dtype) &&
+                       (cb->use_tensor_cores == 2 || N >= kPrefillMinRows);
+  long long chunk = z2z::kLogitRowChunk;
+  if (prefill) {
+    const int strips = cb->prefill_strips > 0 ? cb->prefill_strips : z2z::prefill_logits_strips(N);
+    chunk = z2z::prefill_logits_max_rows(cb->plan.lpart_bytes, cb->plan.plan_bytes, strips);
+    if (chunk < N)      // several launches: size them for the worst split
+      chunk = z2z::prefill_logits_max_rows(cb->plan.lpart_bytes, cb->plan.plan_bytes, z2z::kPrefillMaxStrips);
+  }
+  for (long long r0 = 0; r0 < N; r0 += chunk) {
     z2z::LogitsArgs c = a;
-    c.N = N - r0 < z2z::kLogitRowChunk ? N - r0 : z2z::kLogitRowChunk;
-    c.row_base = a.row_base + r0;
+    c.N = (int)(N - r0 < chunk ? N - r0 : chunk);
+    c.row_base = a.row_base + (int)r0;
     c.hidden = reinterpret_cast<const char*>(a.hidden) + (size_t)r0 * cb->cfg.d * esz;
     if (a.row_seq) c.row_seq = a.row_seq + r0;
     if (a.row_nvis) c.row_nvis = a.row_nvis + r0;
@@ -114,8 +130,11 @@ int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s, z2z::Logits
     if (a.target_logit) c.target_logit = a.target_logit + r0;
     if (a.logits_debug) c.logits_debug = a.logits_debug + (size_t)r0 * ldbg;
     if (a.row_seq == nullptr && r0 > 0) return fail(Z2Z_ERR_INVALID_ARG, "d_row_seq is required when N > B");
-    if (cb->use_tensor_cores && z2z::logits_tc_supported(cb->cfg.d, cb->cfg.dtype)) {
-      int* words = reinterpret_cast<int*>(cb->ws + cb->plan.off_words);
+    int* words = reinterpret_cast<int*>(cb->ws + cb->plan.off_words);
+    if (prefill) {
+      Z2Z_CUDA(z2z::run_logits_prefill(cb->view, c, reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_plan), words,
+                                       cb->prefill_strips, &cb->prof, s), "logits (prompt scoring)");
+    } else if (tc) {
       Z2Z_CUDA(z2z::run_logits_tc(cb->view, c, words + 1, words, info, &cb->prof, s), "logits (tensor cores)");
     } else {
       Z2Z_CUDA(z2z::run_logits_simt(cb->view, c, info, &cb->prof, s), "logits");
@@ -163,6 +182,7 @@ int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, 
   h->cfg = c; h->plan = plan; h->ws = reinterpret_cast<char*>(d_ws); h->ws_bytes = ws_bytes;
   h->dff = c.enc_dff; h->heads = c.enc_heads;
   h->use_tensor_cores = 1;
+  h->prefill_strips = 0;
   z2z::CbView& v = h->view;
   v.V = c.V; v.M = c.M; v.cap = c.cap; v.B = c.B; v.n_slots = plan.n_slots;
   v.hash = reinterpret_cast<unsigned long long*>(h->ws + plan.off_hash);
@@ -392,7 +412,10 @@ int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t*
 
 int32_t z2z_set_tensor_cores(z2z_codebook* cb, int32_t enable) {
   if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
-  cb->use_tensor_cores = enable != 0;
+  if (enable < 0) return fail(Z2Z_ERR_INVALID_ARG, "enable must be >= 0");
+  cb->use_tensor_cores = enable == 0 ? 0 : (enable % 16 == 2 ? 2 : 1);
+  cb->prefill_strips = enable / 16;
+  if (cb->prefill_strips > z2z::kPrefillMaxStrips) cb->prefill_strips = z2z::kPrefillMaxStrips;
   return Z2Z_OK;
 }
 

@@ -72,12 +72,14 @@ struct WsPlan {
   size_t off_words;                               // device words: [0] kernel error, [1] logits tiles
   size_t off_part, part_bytes;                    // GEMM split-K partial tiles
   size_t off_lpart, lpart_bytes;                  // logits partial reductions
+  size_t off_plan, plan_bytes;                    // per-row-tile plan of the prompt-scoring logits kernel
   size_t off_step_out;                            // small per-step outputs
   size_t total;
 };
 
 constexpr int kLogitRowChunk = 8192;              // rows per logits launch (larger N loops)
-constexpr int kLogitPartRows = 1 << 17;           // partial-reduction slots (rows x groups)
+constexpr int kLogitPartRows = 1 << 19;           // partial-reduction slots (rows x groups)
+constexpr int kPrefillPlanTiles = 1 << 14;        // 256-row tiles one prompt-scoring launch may have
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -129,6 +131,8 @@ inline WsPlan plan_workspace(const z2z_config& c) {
   p.off_words = take(256);
   p.lpart_bytes = (size_t)kLogitPartRows * 32;
   p.off_lpart = take(p.lpart_bytes);
+  p.plan_bytes = (size_t)kPrefillPlanTiles * 3 * 4;
+  p.off_plan = take(p.plan_bytes);
   p.off_step_out = take((size_t)c.B * 64);
   p.total = o;
   return p;

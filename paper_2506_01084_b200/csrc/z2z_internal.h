@@ -85,6 +85,16 @@ cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, LogitsPartInf
 cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word,
                           LogitsPartInfo* info, Prof* prof, cudaStream_t s);
 
+// ---- z2z_prefill_logits.cu -------------------------------------------------------------------
+// Same outputs as run_logits_tc, for many hidden rows (bf16, d % 64 == 0).  `plan` is scratch for
+// 3 int32 per 256-row tile.  strips_override > 0 fixes the number of column strips (tests).
+bool prefill_logits_supported(int d, int dtype);
+// Rows one launch can take with the given scratch when `strips` partials per row are needed.
+long long prefill_logits_max_rows(size_t lpart_bytes, size_t plan_bytes, int strips);
+int prefill_logits_strips(int N);
+cudaError_t run_logits_prefill(const CbView& cb, const LogitsArgs& a, int32_t* plan, int* err_word,
+                               int strips_override, Prof* prof, cudaStream_t s);
+
 // ---- z2z_decode_update.cu --------------------------------------------------------------------
 struct DecodeUpdateArgs {
   const LogitPartial* lpart; int part_stride, part_count;

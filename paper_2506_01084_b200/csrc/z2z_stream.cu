@@ -47,7 +47,8 @@ struct Job {
   int col0, nvalid, owner, k0;   // logits: first column id, valid rows, owning sequence, first entry
   int rt;                // hidden-row tile
   int nrows;             // weight rows in this job (the MMA's N), multiple of 16
-  int wbox;              // rows per TMA box of W (nrows / wbox boxes per k block)
+  int wbox_min;          // smallest TMA box of W in rows; boxes are powers of two times this, up
+  int wbox_classes;      // to wbox_min << (wbox_classes - 1); tensor map = wmap * classes + class
 };
 
 // ---- GEMM schedule ------------------------------------------------------------------------------
@@ -74,7 +75,7 @@ struct GemmSched {
     j.amap = g; j.wmap = g; j.arow = j.rt * 128;
     j.wrow = (rem - g * p.tiles_per_group) * NT;
     j.slot = tile + c;
-    j.nrows = NT; j.wbox = NT;
+    j.nrows = NT; j.wbox_min = NT; j.wbox_classes = 1;
     u += j.kb1 - j.kb0;
     return true;
   }
@@ -102,7 +103,8 @@ struct LogitSched {
     if (u >= u1) return false;
     j.rt = (int)(u / vt);
     const int v = (int)(u - (long long)j.rt * vt);
-    j.amap = 0; j.arow = j.rt * 128; j.kb0 = 0; j.kb1 = ksteps; j.slot = 0; j.wbox = kLogitGran;
+    j.amap = 0; j.arow = j.rt * 128; j.kb0 = 0; j.kb1 = ksteps; j.slot = 0;
+    j.wbox_min = kLogitGran; j.wbox_classes = kLogitBoxClasses;
     int remaining, total_rows, g0;
     if (v < n_static) {
       g0 = v; remaining = n_static - v; total_rows = p.cb.V;
@@ -147,11 +149,17 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
         for (int i = 0; i < KSB; ++i)
           tma_load_2d(sb + part * a_part_bytes + i * a_box_rows * 128, amaps[j.amap],
                       (ks * KSB + i) * 64, j.arow + part * a_part_row, full, pol_a);
+      // the W rows of the job go out as few boxes as possible: largest power-of-two box first
+      for (int r0 = 0; r0 < j.nrows;) {
+        int cls = j.wbox_classes - 1;
+        while (cls > 0 && (j.wbox_min << cls) > j.nrows - r0) --cls;
+        const CUtensorMap* wm = wmaps[j.wmap * j.wbox_classes + cls];
 #pragma unroll
-      for (int i = 0; i < KSB; ++i)
-        for (int r0 = 0; r0 < j.nrows; r0 += j.wbox)
-          tma_load_2d(sb + a_parts * a_part_bytes + i * NT * 128 + r0 * 128, wmaps[j.wmap],
+        for (int i = 0; i < KSB; ++i)
+          tma_load_2d(sb + a_parts * a_part_bytes + i * NT * 128 + r0 * 128, wm,
                       (ks * KSB + i) * 64, j.wrow + r0, full, pol_w);
+        r0 += j.wbox_min << cls;
+      }
       if (++stage == STAGES) { stage = 0; phase ^= 1u; }
     }
   }
@@ -287,8 +295,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
 // =================================================================================================
 template <int NT, int KSB, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
-k_stream_logits(const StreamLogitsParams p, const __grid_constant__ CUtensorMap tmH,
-                const __grid_constant__ CUtensorMap tmWU, const __grid_constant__ CUtensorMap tmUh) {
+k_stream_logits(const StreamLogitsParams p, const __grid_constant__ LogitMaps tm) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm);
@@ -297,7 +304,7 @@ k_stream_logits(const StreamLogitsParams p, const __grid_constant__ CUtensorMap 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   setup_barriers<STAGES>(ctrl);
   for (int b = threadIdx.x; b < p.cb.B; b += kThreads) s_pref[b + 1] = (p.cb.n[b] + kLogitGran - 1) / kLogitGran;
-  if (warp == 0 && lane == 0) { prefetch_tmap(&tmH); prefetch_tmap(&tmWU); prefetch_tmap(&tmUh); }
+  if (warp == 0 && lane < 1 + 2 * kLogitBoxClasses) prefetch_tmap(lane == 0 ? &tm.h : &tm.w[lane - 1]);
   __syncthreads();
   if (threadIdx.x == 0) {
     s_pref[0] = 0;
@@ -314,8 +321,9 @@ k_stream_logits(const StreamLogitsParams p, const __grid_constant__ CUtensorMap 
 
   if (warp == 0) {
     if (lane == 0) {
-      const CUtensorMap* amaps[1] = {&tmH};
-      const CUtensorMap* wmaps[2] = {&tmWU, &tmUh};
+      const CUtensorMap* amaps[1] = {&tm.h};
+      const CUtensorMap* wmaps[2 * kLogitBoxClasses];
+      for (int i = 0; i < 2 * kLogitBoxClasses; ++i) wmaps[i] = &tm.w[i];
       LogitSched sched(p, s_pref, vt, NT);
       producer_role<NT, KSB, STAGES>(sched, ctrl, stage_base, 1, p.a_box_rows, 0, amaps, wmaps);
     }
@@ -509,13 +517,13 @@ cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* map
 }
 
 template <int NT, int KSB, int STAGES>
-static cudaError_t launch_logits_t(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
+static cudaError_t launch_logits_t(const StreamLogitsParams& p, const LogitMaps* maps, int grid, cudaStream_t s) {
   const size_t stage = (size_t)KSB * p.a_box_rows * 128 + (size_t)KSB * NT * 128;
   const size_t smem = 1024 + 1024 + 5120 + STAGES * stage + kTailPad;
   auto kern = k_stream_logits<NT, KSB, STAGES>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<grid, kThreads, smem, s>>>(p, maps[0], maps[1], maps[2]);
+  kern<<<grid, kThreads, smem, s>>>(p, *maps);
   return cudaGetLastError();
 }
 
@@ -538,13 +546,16 @@ cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, i
   p.part_stride = (n_sm + p.row_tiles - 1) / p.row_tiles + 2;
   p.vt_out = vt_word; p.err = err_word;
   if ((size_t)a.N * p.part_stride * sizeof(LogitPartial) > a.lpart_bytes) return cudaErrorMemoryAllocation;
-  CUtensorMap maps[3];
-  if (!make_tmap_bf16(&maps[0], a.hidden, a.N, a.d, p.a_box_rows)) return cudaErrorInvalidValue;
-  if (!make_tmap_bf16(&maps[1], a.WU, cb.V, a.d, kLogitGran)) return cudaErrorInvalidValue;
-  if (cb.cap > 0) {
-    if (!make_tmap_bf16(&maps[2], a.Uh, (long long)cb.B * cb.cap, a.d, kLogitGran)) return cudaErrorInvalidValue;
-  } else {
-    maps[2] = maps[1];
+  LogitMaps maps;
+  if (!make_tmap_bf16(&maps.h, a.hidden, a.N, a.d, p.a_box_rows)) return cudaErrorInvalidValue;
+  for (int c = 0; c < kLogitBoxClasses; ++c) {
+    if (!make_tmap_bf16(&maps.w[c], a.WU, cb.V, a.d, kLogitGran << c)) return cudaErrorInvalidValue;
+    if (cb.cap > 0) {
+      if (!make_tmap_bf16(&maps.w[kLogitBoxClasses + c], a.Uh, (long long)cb.B * cb.cap, a.d, kLogitGran << c))
+        return cudaErrorInvalidValue;
+    } else {
+      maps.w[kLogitBoxClasses + c] = maps.w[c];
+    }
   }
   // every CTA must own at least one unit: the static tiles alone give a lower bound on the units
   long long units_lb = (long long)p.row_tiles * ((cb.V + kLogitGran - 1) / kLogitGran);
@@ -554,10 +565,10 @@ cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, i
     if (p.row_tiles != 1) return cudaErrorInvalidValue;
     info->stride = p.part_stride; info->count = grid;
   }
-  return launch_stream_logits(p, maps, grid, info == nullptr, prof, s);
+  return launch_stream_logits(p, &maps, grid, info == nullptr, prof, s);
 }
 
-cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, bool merge,
+cudaError_t launch_stream_logits(const StreamLogitsParams& p, const LogitMaps* maps, int grid, bool merge,
                                  Prof* prof, cudaStream_t s) {
   constexpr int NT = kLogitNT, KSB = kLogitKSB;
   const LogitsArgs& a = p.la;

@@ -11,7 +11,15 @@ namespace z2z {
 constexpr int kMaxStages = 8;
 constexpr int kGemmNT = 128, kGemmKSB = 1;      // weight rows per tile, 64-wide k blocks per stage
 constexpr int kLogitNT = 128, kLogitKSB = 1;
-constexpr int kLogitGran = 16;                  // rows per TMA box / scheduling granule of the logits kernel
+constexpr int kLogitGran = 32;                  // scheduling granule of the logits kernel, in weight rows (TMA boxes of
+                                                // fewer rows stream several times slower)
+constexpr int kLogitBoxClasses = 3;             // TMA boxes of 32, 64 and 128 weight rows
+
+// Tensor maps of the logits kernel: hidden rows, then W_U and U_h once per box size.
+struct LogitMaps {
+  CUtensorMap h;
+  CUtensorMap w[2 * kLogitBoxClasses];
+};
 
 // Stream-K GEMM over `groups` independent problems of identical shape (the two hyper-encoders).
 // The unit space is (group, tile, k-step); CTA c of G owns units [floor(cU/G), floor((c+1)U/G)).
@@ -40,9 +48,24 @@ struct StreamLogitsParams {
   int* err;
 };
 
+// Prompt-scoring logits kernel (z2z_prefill_logits.cu): CTA pairs, 256 x 256 tiles.
+constexpr int kPrefillMaxStrips = 8;            // column strips a row tile may be cut into
+struct PrefillLogitsParams {
+  CbView cb;
+  LogitsArgs la;
+  int ksteps;            // d / 64
+  int row_tiles;         // ceil(N / 256)
+  int n_static;          // ceil(V / 256)
+  int strips;            // column strips per row tile = partial reductions per hidden row
+  int32_t* tile_lo;      // [row_tiles] lowest / highest sequence owning a row of the tile
+  int32_t* tile_hi;
+  int32_t* tile_nh;      // [row_tiles] hypertoken column tiles of the tile
+  int* err;
+};
+
 bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows);
 cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s);
-cudaError_t launch_stream_logits(const StreamLogitsParams& p, const CUtensorMap* maps, int grid, bool merge,
+cudaError_t launch_stream_logits(const StreamLogitsParams& p, const LogitMaps* maps, int grid, bool merge,
                                  Prof* prof, cudaStream_t s);
 
 }  // namespace z2z

@@ -38,8 +38,9 @@ class Pair:
         self.cfg = zb.make_config(w.V, w.d, w.M, w.cap, w.B, w.dtype, w.enc_layers, w.heads,
                                   w.dff, w.tied)
         self.cb = zb.Codebook(self.cfg, device)
-        if not tensor_cores:
-            zb.z2z_set_tensor_cores(self.cb, False)      # CUDA-core kernels as an on-GPU cross-check
+        if int(tensor_cores) != 1:
+            # 0: CUDA-core kernels as an on-GPU cross-check; 2 + 16 s: CTA-pair logits kernel
+            zb.z2z_set_tensor_cores(self.cb, int(tensor_cores))
         self.g_WE = self.W_E.to(self.dev)
         self.g_WU = self.g_WE if w.tied else self.W_U.to(self.dev)
         self.g_encE_t = [t.to(self.dev) for t in self.enc_E]

@@ -230,7 +230,8 @@ def test_hyper_embed_explicit_ranges_and_incremental():
 # ------------------------------------------------------------------------------------------------
 # Joint logits and reductions
 # ------------------------------------------------------------------------------------------------
-def _logits_case(w, seed, rows_per_seq, causal, select, temperature=0.8, tensor_cores=True):
+def _logits_case(w, seed, rows_per_seq, causal, select, temperature=0.8, tensor_cores=True,
+                 debug=True):
     p = Pair(w, seed=seed, generic_encoder=False, tensor_cores=tensor_cores)
     codes, clen, after = p.gpu_encode()
     ocodes, oafter = p.oracle.prefill([p.tokens[b].tolist() for b in range(w.B)])
@@ -256,8 +257,9 @@ def _logits_case(w, seed, rows_per_seq, causal, select, temperature=0.8, tensor_
     zb.z2z_dynamic_logits(p.cb, g_hid, torch.tensor(row_seq, dtype=torch.int32, device=p.dev),
                           torch.tensor(row_nvis, dtype=torch.int32, device=p.dev) if causal else None,
                           p.g_WU, p.U_h, select, temperature, 0xABCDEF12345, 77,
-                          torch.tensor(targets, dtype=torch.int32, device=p.dev),
-                          out["lse"], am, out["max"], smp if select else None, out["tl"], dbg)
+                          torch.tensor(targets, dtype=torch.int32, device=p.dev) if debug else None,
+                          out["lse"], am, out["max"], smp if select else None,
+                          out["tl"] if debug else None, dbg if debug else None)
     dbg = dbg.cpu().double().numpy()
     lse, mx, tl = (out[k].cpu().double().numpy() for k in ("lse", "max", "tl"))
     am, smp = am.cpu().numpy(), smp.cpu().numpy()
@@ -266,20 +268,23 @@ def _logits_case(w, seed, rows_per_seq, causal, select, temperature=0.8, tensor_
     for r in range(N):
         b, nv = row_seq[r], row_nvis[r]
         l = olg.joint_logits(H[r], p.oracle.W_U, U64[b, :nv])
-        got = dbg[r, :w.V + nv]
-        err = np.abs(got - l).max()
-        worst = max(worst, err)
-        assert err <= TOL
-        assert np.all(np.isnan(dbg[r, w.V + nv:]))            # invisible columns never computed
-        assert abs(lse[r] - olg.lse(l)) <= TOL
+        if debug:
+            got = dbg[r, :w.V + nv]
+            err = np.abs(got - l).max()
+            worst = max(worst, err)
+            assert err <= TOL
+            assert np.all(np.isnan(dbg[r, w.V + nv:]))        # invisible columns never computed
+        assert abs(lse[r] - olg.lse(l)) <= TOL, (r, lse[r], olg.lse(l))
+        worst = max(worst, abs(lse[r] - olg.lse(l)))
         a, best, gap = olg.top2(l)
         assert abs(mx[r] - best) <= TOL
         if am[r] != a:
             assert gap < GAP and l[am[r]] >= best - GAP
-        if targets[r] < w.V + nv:
-            assert abs(tl[r] - l[targets[r]]) <= TOL
-        else:
-            assert np.isnan(tl[r])
+        if debug:
+            if targets[r] < w.V + nv:
+                assert abs(tl[r] - l[targets[r]]) <= TOL
+            else:
+                assert np.isnan(tl[r])
         if select:
             ch, scores, sgap = olg.select(l, 1, temperature, 0xABCDEF12345, 77, r)
             if smp[r] != ch:
@@ -404,3 +409,34 @@ def test_tensor_core_kernels_many_rows_and_sequences():
     worst = _logits_case(MID_BF16, 32, [9] * MID_BF16.B, True, 1)
     print(f"mid_bf16: max |logit error| = {worst:.3e}")
     _decode_follow(MID_BF16, 33, zb.SELECT_ARGMAX, steps=4)
+
+
+# ------------------------------------------------------------------------------------------------
+# Prompt-scoring logits kernel (CTA pairs, 256 x 256 tiles), forced on for small shapes:
+# several row tiles with a ragged tail, rows of several sequences inside one tile, sequences
+# without rows, causal per-row limits, every number of column strips, both epilogue paths
+# ------------------------------------------------------------------------------------------------
+PAIR_BF16 = si.Workload("pair_bf16", V=3000, d=256, dtype="bf16", B=5, T=1400, M=3, cap=700,
+                        zipf_s=1.1, copy_p=0.5, seg_min=3, seg_max=10, steps=0, enc_layers=0,
+                        enc_heads=2, enc_dff=512)
+
+
+@pytest.mark.parametrize("strips", [0, 1, 3, 8])
+def test_pair_logits_kernel_fast_path(strips):
+    # reductions only: the epilogue that folds whole 256-column tiles; hypertokens need > 1 tile
+    rows = [300, 0, 77, 256, 130]
+    worst = _logits_case(PAIR_BF16, 41, rows, False, 0, tensor_cores=2 + 16 * strips, debug=False)
+    print(f"pair kernel, strips={strips}: max |LSE error| = {worst:.3e}")
+
+
+@pytest.mark.parametrize("strips,causal,select", [(0, True, 1), (2, False, 1), (8, True, 0)])
+def test_pair_logits_kernel_generic_path(strips, causal, select):
+    rows = [40, 0, 300, 5, 200]
+    worst = _logits_case(PAIR_BF16, 42, rows, causal, select, tensor_cores=2 + 16 * strips)
+    print(f"pair kernel (all outputs), strips={strips}: max |logit error| = {worst:.3e}")
+
+
+def test_pair_logits_kernel_causal_fast_path_and_no_hypertokens():
+    _logits_case(PAIR_BF16, 43, [256, 256, 1, 0, 90], True, 0, tensor_cores=2, debug=False)
+    _logits_case(PAIR_BF16.scaled(cap=0, name="pair_nocap"), 44, [100, 200, 0, 0, 3], False, 0,
+                 tensor_cores=2, debug=False)

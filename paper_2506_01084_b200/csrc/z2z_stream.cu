@@ -487,6 +487,25 @@ bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map over the same matrix seen as [cols / 64 k-blocks][rows][64]: one box brings
+// `box_kb` k-blocks of `box_rows` rows, laid out k-block after k-block (each k-block is then a
+// K-major 128-byte-swizzled operand tile).
+bool make_tmap_bf16_kblocks(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows,
+                            int box_kb) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols % 64) || box_rows < 1 || box_rows > 256 || box_kb < 1 ||
+      box_kb > 256 || rows < 1)
+    return false;
+  cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_kb};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int NT, int KSB>
 static int pick_stages(int a_parts, int a_box_rows, int extra) {
   const int stage = a_parts * KSB * a_box_rows * 128 + KSB * NT * 128;
@@ -531,6 +550,7 @@ bool logits_tc_supported(int d, int dtype) { return dtype == Z2Z_DTYPE_BF16 && d
 
 cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, int* err_word,
                           LogitsPartInfo* info, Prof* prof, cudaStream_t s) {
+  if (decode_logits_applies(a)) return run_logits_decode(cb, a, vt_word + 1, err_word, info, prof, s);
   static int n_sm = 0;
   if (!n_sm) {
     int dev = 0;

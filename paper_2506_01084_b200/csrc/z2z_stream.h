@@ -25,6 +25,32 @@ struct LogitMaps {
 // The unit space is (group, tile, k-step); CTA c of G owns units [floor(cU/G), floor((c+1)U/G)).
 // Every maximal run of units inside one tile and one CTA produces one fp32 partial tile of
 // out_rows x NT values in slot (global tile index + c).
+// ---- decode logits kernel (z2z_decode_logits.cu) ---------------------------------------------
+// Tensor maps, all of the form [k-block][row][64 columns]: hidden rows as one resident operand
+// (h) and per stage with 1, 2 or 4 k-blocks (hk[0..2]); W_U and U_h as boxes of 32 rows x 4
+// k-blocks (class 0) and 128 rows x 1 k-block (class 2): w[tensor * 2 + (class == 2)].
+struct DecodeLogitMaps {
+  CUtensorMap h, hk[3];
+  CUtensorMap w[4];
+};
+struct DecodeLogitsParams {
+  CbView cb;
+  LogitsArgs la;
+  int ksteps;            // d / 64 (a multiple of 4)
+  int hid_rows;          // hidden rows held per k-block in shared memory (N rounded up to 8)
+  int hid_box_kb;        // k-blocks per TMA box of the resident hidden rows
+  int stages;            // stages of the load ring
+  int part_stride;       // partial slots per hidden row
+  int fixed_granules;    // 32-row granules of W_U every CTA owns up front (a multiple of 4)
+  int* counters;         // device words: [0] pool claims, [1] CTAs finished (both return to 0)
+  int* err;
+};
+bool make_tmap_bf16_kblocks(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows,
+                            int box_kb);
+bool decode_logits_applies(const LogitsArgs& a);
+cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counters, int* err_word,
+                              LogitsPartInfo* info, Prof* prof, cudaStream_t s);
+
 struct StreamGemmParams {
   int row_tiles;         // 128-row tiles of A (outermost dimension of the unit space)
   int groups, tiles_per_group, ksteps;

@@ -440,3 +440,41 @@ def test_pair_logits_kernel_causal_fast_path_and_no_hypertokens():
     _logits_case(PAIR_BF16, 43, [256, 256, 1, 0, 90], True, 0, tensor_cores=2, debug=False)
     _logits_case(PAIR_BF16.scaled(cap=0, name="pair_nocap"), 44, [100, 200, 0, 0, 3], False, 0,
                  tensor_cores=2, debug=False)
+
+
+# ------------------------------------------------------------------------------------------------
+# Decode logits kernel (weight rows as the MMA's M operand, one thread per vocabulary row, fixed
+# shares plus a claimed pool): every batch-size class, hidden rows resident in shared memory or
+# streamed per stage, rows that share a sequence, causal limits, all outputs, repeated launches
+# (the pool counter must come back to zero)
+# ------------------------------------------------------------------------------------------------
+WIDE_BF16 = si.Workload("wide_bf16", V=2000, d=1280, dtype="bf16", B=4, T=600, M=3, cap=300,
+                        zipf_s=1.1, copy_p=0.5, seg_min=3, seg_max=10, steps=0, enc_layers=0,
+                        enc_heads=2, enc_dff=512)
+TALL_BF16 = si.Workload("tall_bf16", V=40000, d=256, dtype="bf16", B=6, T=900, M=3, cap=500,
+                        zipf_s=1.1, copy_p=0.5, seg_min=3, seg_max=10, steps=0, enc_layers=0,
+                        enc_heads=2, enc_dff=512)
+
+
+@pytest.mark.parametrize("rows,causal,select,debug", [
+    ([2, 1, 3, 1, 1], False, 0, False),      # 8 rows, reductions only
+    ([3, 0, 5, 4, 1], True, 1, True),        # 13 rows -> 16-row class, sampling + all outputs
+    ([16, 0, 0, 0, 0], True, 0, True),       # one sequence owns every row
+    ([7, 7, 5, 5, 5], False, 0, False),      # 29 rows -> 32-row class
+    ([6, 6, 6, 7, 7], True, 0, False),       # 32 rows, causal
+])
+def test_decode_logits_kernel_batches(rows, causal, select, debug):
+    worst = _logits_case(PAIR_BF16, 51, rows, causal, select, debug=debug)
+    print(f"decode kernel rows={sum(rows)}: worst error {worst:.3e}")
+
+
+@pytest.mark.parametrize("rows,select,debug", [([8, 8, 8, 8], 0, False), ([2, 6, 3, 5], 1, True)])
+def test_decode_logits_kernel_streamed_hidden_rows(rows, select, debug):
+    # d = 1280: 32 (16) rows x 20 k-blocks exceed (fit) the resident budget
+    _logits_case(WIDE_BF16, 52, rows, True, select, debug=debug)
+
+
+def test_decode_logits_kernel_fixed_shares_and_pool():
+    # V = 40000: every CTA owns a fixed share of 128-row jobs and the pool holds both W_U and U_h
+    _logits_case(TALL_BF16, 53, [1, 1, 1, 1, 1, 1], False, 0, debug=False)
+    _logits_case(TALL_BF16, 54, [2, 3, 1, 4, 0, 2], True, 1, debug=True)

@@ -8,13 +8,15 @@
 //     (max, sum-exp, argmax[, best perturbed score]) per hidden row in registers; the threads'
 //     reductions are merged once, when the CTA has streamed its share.
 //   * every stage of the ring is ONE TMA box of 16 KB: 128 weight rows x 1 k-block (64 columns)
-//     or 32 rows x 4 k-blocks (a 3-D tensor map [k-block][row][64]).  The TMA unit's cost is per
-//     box, not per byte, so small boxes would cap the stream far below the HBM rate.
+//     or 64 rows x 2 k-blocks (a 3-D tensor map [k-block][row][64]).  The TMA unit's cost is per
+//     box, not per byte, so small boxes would cap the stream far below the HBM rate; and since an
+//     MMA always spans 128 rows, jobs of fewer than 64 rows would cost more tensor-pipe time per
+//     stage than the stage's bytes take to arrive.
 //   * the hidden rows are loaded into shared memory once when they fit (RESIDENT), else one box
 //     per stage.
 //   * work: every CTA first streams a fixed share of W_U in 128-row jobs (known without reading
 //     any codebook state, so the first loads are issued right after barrier set-up); the rest
-//     of W_U and all U_h rows form a pool of 32-row units that the CTAs claim with an atomic
+//     of W_U and all U_h rows form a pool of 64-row units that the CTAs claim with an atomic
 //     counter, which evens out the differences in streaming speed between SMs.
 //
 // Roles: warp 0 lane 0 producer (claims work, publishes each job in a shared-memory ring, issues
@@ -31,13 +33,13 @@ using namespace sm100;
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kGran = 32;                // pool unit / scheduling granule, in weight rows
+constexpr int kGran = 64;                // pool unit / scheduling granule, in weight rows
 constexpr int kJobRing = 32;             // published jobs kept (> stages + accumulators in flight)
 constexpr int kDecodeMaxStages = 12;
 constexpr int kTailPadBytes = 16384;     // readable shared memory behind the last stage
 
 struct DecodeJob {
-  int cls;               // 2: 128 rows x 1 k-block per stage, 0: 32 rows x 4 k-blocks, -1: no more work
+  int cls;               // 2: 128 rows x 1 k-block per stage, 1: 64 rows x 2 k-blocks, -1: no more work
   int wmap, wrow;        // tensor (0: W_U, 1: U_h) and first row in it
   int col0, nvalid;      // first column id of the joint logits, rows that exist
   int owner, k0;         // U_h: owning sequence and first entry number; W_U: -1, 0
@@ -77,7 +79,7 @@ __device__ __forceinline__ float key_float(int k) { return __int_as_float(k ^ ((
 __device__ __forceinline__ bool pool_job(const DecodeLogitsParams& p, const int* pref, int pool_static,
                                          int pool_total, int u, DecodeJob& j) {
   if (u >= pool_total) return false;
-  j.cls = 0; j.pad = 0;
+  j.cls = 1; j.pad = 0;
   if (u < pool_static) {
     const int g = p.fixed_granules * (int)gridDim.x + u;
     j.wmap = 0; j.wrow = g * kGran; j.col0 = j.wrow; j.owner = -1; j.k0 = 0;
@@ -108,7 +110,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
   const int hid_rows = p.hid_rows;
   const uint32_t hid_bytes = RESIDENT ? (uint32_t)p.ksteps * hid_rows * 128 : 0u;
   const uint32_t stage_base = hid_base + ((hid_bytes + 1023u) & ~1023u);
-  const uint32_t stage_hid = RESIDENT ? 0u : (uint32_t)((4 * hid_rows * 128 + 1023) & ~1023);
+  const uint32_t stage_hid = RESIDENT ? 0u : (uint32_t)((2 * hid_rows * 128 + 1023) & ~1023);
   const uint32_t stage_bytes = NT * 128 + stage_hid;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const LogitsArgs& a = p.la;
@@ -151,9 +153,9 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
       };
       auto stream = [&](const DecodeJob& j) {
         const int big = j.cls == 2;
-        const int ksb = big ? 1 : 4;
+        const int ksb = big ? 1 : 2;
         const CUtensorMap* wm = &tm.w[j.wmap * 2 + big];
-        const CUtensorMap* hm = &tm.hk[big ? 0 : 2];
+        const CUtensorMap* hm = &tm.hk[big ? 0 : 1];
         for (int ks = 0; ks < p.ksteps && ok; ks += ksb) {
           if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctrl->full[stage]);
@@ -166,26 +168,39 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
       };
       // fixed share: 128-row jobs of W_U, known without any codebook state
       const int g_first = (int)blockIdx.x * p.fixed_granules;
-      for (int g = g_first; g < g_first + p.fixed_granules && ok; g += 4) {
+      for (int g = g_first; g < g_first + p.fixed_granules && ok; g += 2) {
+        const int big = g + 2 <= g_first + p.fixed_granules;     // an odd share ends with one 64-row job
+        const int rows = big ? NT : kGran;
         DecodeJob j;
-        j.cls = 2; j.wmap = 0; j.wrow = g * kGran; j.col0 = j.wrow; j.owner = -1; j.k0 = 0; j.pad = 0;
-        j.nvalid = p.cb.V - j.wrow < NT ? p.cb.V - j.wrow : NT;
+        j.cls = big ? 2 : 1; j.wmap = 0; j.wrow = g * kGran; j.col0 = j.wrow; j.owner = -1; j.k0 = 0; j.pad = 0;
+        j.nvalid = p.cb.V - j.wrow < rows ? p.cb.V - j.wrow : rows;
         publish(j);
         stream(j);
       }
-      // pool: the rest of W_U and every visible row of U_h, claimed 32 rows at a time
+      // pool: the rest of W_U and every visible row of U_h, claimed 64 rows at a time
       if (ok && !mbar_wait(smem_u32(&ctrl->pref_ready), 0, &ctrl->abort)) ok = false;
       if (ok) {
         const int gs = (p.cb.V + kGran - 1) / kGran;
         const int pool_static = gs - p.fixed_granules * (int)gridDim.x;
         const int pool_total = pool_static + s_pref[p.cb.B];
-        int u = atomicAdd(p.counters, 1);
-        DecodeJob j;
+        // Guided claims: two consecutive granules (one 128-row job when they lie in one segment)
+        // while more than four rounds of single units are left, then single 64-row units, so that
+        // the CTAs finish within one small unit of each other.
+        const int single_from = pool_total - 4 * (int)gridDim.x;
+        int chunk = 2 <= single_from ? 2 : 1;
+        int u = atomicAdd(p.counters, chunk);
+        DecodeJob j, j2;
         while (ok && pool_job(p, s_pref, pool_static, pool_total, u, j)) {
+          const bool pair = chunk == 2 && pool_job(p, s_pref, pool_static, pool_total, u + 1, j2);
+          const bool fused = pair && j2.wmap == j.wmap && j2.owner == j.owner && j2.wrow == j.wrow + kGran;   // one segment
+          if (fused) { j.cls = 2; j.nvalid += j2.nvalid; }
           publish(j);
-          const int u_next = atomicAdd(p.counters, 1);           // in flight while this unit streams
           stream(j);
-          u = u_next;
+          if (pair && !fused && ok) { publish(j2); stream(j2); }
+          // the next claim is made only now: the stages still in flight cover its latency, and a
+          // CTA never holds a unit that another, idle CTA could already be streaming
+          chunk = u + chunk + 2 <= single_from ? 2 : 1;
+          u = atomicAdd(p.counters, chunk);
         }
       }
       DecodeJob last;
@@ -244,7 +259,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
         if (!mbar_wait(smem_u32(&ctrl->acc_empty[buf]), aph ^ 1u, &ctrl->abort)) break;
         tc_fence_after();
         const uint32_t d = tmem_base + buf * NBP;
-        const int ksb = j.cls == 2 ? 1 : 4;
+        const int ksb = j.cls == 2 ? 1 : 2;
         const uint32_t kb_bytes = (uint32_t)(j.cls == 2 ? NT : kGran) * 128;   // one k-block of the job's rows
         uint32_t acc = 0;
         for (int ks = 0; ks < p.ksteps; ks += ksb) {
@@ -398,8 +413,7 @@ __global__ void k_decode_fill_nan(float* p, int n) {
 }  // namespace
 
 // Decode batches: N <= 16 rows with any outputs, N <= 32 rows when only the plain reductions are
-// wanted (the sampling state of 32 rows does not fit the register file); d a multiple of 256
-// (a stage carries up to four 64-column k-blocks).
+// wanted (the sampling state of 32 rows does not fit the register file); d a multiple of 256.
 bool decode_logits_applies(const LogitsArgs& a) {
   const bool generic = a.select == Z2Z_SELECT_GUMBEL || a.logits_debug || a.target_logit;
   return a.dtype == Z2Z_DTYPE_BF16 && a.d % 256 == 0 && (a.N <= 16 || (a.N <= 32 && !generic));
@@ -409,7 +423,7 @@ template <int NB, bool GENERIC>
 static cudaError_t launch_decode(DecodeLogitsParams p, const DecodeLogitMaps& maps, int grid, bool resident,
                                  cudaStream_t s) {
   const size_t hid = resident ? (((size_t)p.ksteps * p.hid_rows * 128 + 1023) & ~(size_t)1023) : 0;
-  const size_t stage = 128 * 128 + (resident ? 0 : (((size_t)4 * p.hid_rows * 128 + 1023) & ~(size_t)1023));
+  const size_t stage = 128 * 128 + (resident ? 0 : (((size_t)2 * p.hid_rows * 128 + 1023) & ~(size_t)1023));
   // Shared memory behind the last stage stays readable (kTailPadBytes): an MMA always reads 128
   // weight rows from a k-block's start and 16 or 32 hidden rows, also when fewer were loaded; what
   // it reads beyond them only feeds accumulator rows and columns that nobody looks at.
@@ -446,8 +460,8 @@ cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counte
   for (int k = 16; k >= 4; --k) if (p.ksteps % k == 0) { p.hid_box_kb = k; break; }
   const int gs = (cb.V + kGran - 1) / kGran;
   const int grid = gs < n_sm ? gs : n_sm;
-  // fixed share: about three quarters of W_U, in whole 128-row jobs per CTA; the rest is pooled
-  p.fixed_granules = (int)((long long)gs * 3 / 4 / (4 * grid)) * 4;
+  // fixed share: nine tenths of W_U; the rest and all of U_h are pooled
+  p.fixed_granules = (int)((long long)gs * 9 / 10 / grid);
   DecodeLogitMaps maps;
   if (!make_tmap_bf16_kblocks(&maps.h, a.hidden, a.N, a.d, p.hid_rows, p.hid_box_kb)) return cudaErrorInvalidValue;
   for (int c = 0; c < 3; ++c)
@@ -456,7 +470,7 @@ cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counte
     const void* base = t == 0 ? a.WU : a.Uh;
     const long long rows = t == 0 ? (long long)cb.V : (long long)cb.B * cb.cap;
     if (t == 1 && cb.cap == 0) { maps.w[2] = maps.w[0]; maps.w[3] = maps.w[1]; break; }
-    if (!make_tmap_bf16_kblocks(&maps.w[t * 2 + 0], base, rows, a.d, kGran, 4)) return cudaErrorInvalidValue;
+    if (!make_tmap_bf16_kblocks(&maps.w[t * 2 + 0], base, rows, a.d, kGran, 2)) return cudaErrorInvalidValue;
     if (!make_tmap_bf16_kblocks(&maps.w[t * 2 + 1], base, rows, a.d, 128, 1)) return cudaErrorInvalidValue;
   }
   p.part_stride = grid + 2;

@@ -27,8 +27,8 @@ struct LogitMaps {
 // out_rows x NT values in slot (global tile index + c).
 // ---- decode logits kernel (z2z_decode_logits.cu) ---------------------------------------------
 // Tensor maps, all of the form [k-block][row][64 columns]: hidden rows as one resident operand
-// (h) and per stage with 1, 2 or 4 k-blocks (hk[0..2]); W_U and U_h as boxes of 32 rows x 4
-// k-blocks (class 0) and 128 rows x 1 k-block (class 2): w[tensor * 2 + (class == 2)].
+// (h) and per stage with 1, 2 or 4 k-blocks (hk[0..2]); W_U and U_h as boxes of 64 rows x 2
+// k-blocks (class 1) and 128 rows x 1 k-block (class 2): w[tensor * 2 + (class == 2)].
 struct DecodeLogitMaps {
   CUtensorMap h, hk[3];
   CUtensorMap w[4];
@@ -41,7 +41,7 @@ struct DecodeLogitsParams {
   int hid_box_kb;        // k-blocks per TMA box of the resident hidden rows
   int stages;            // stages of the load ring
   int part_stride;       // partial slots per hidden row
-  int fixed_granules;    // 32-row granules of W_U every CTA owns up front (a multiple of 4)
+  int fixed_granules;    // 64-row granules of W_U every CTA owns up front
   int* counters;         // device words: [0] pool claims, [1] CTAs finished (both return to 0)
   int* err;
 };

@@ -194,6 +194,8 @@ int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, 
   v.n_emb = reinterpret_cast<int32_t*>(h->ws + plan.off_n_emb);
   *cb = h;
   Z2Z_CUDA(cudaMemsetAsync(h->ws + plan.off_words, 0, 256, reinterpret_cast<cudaStream_t>(stream)), "codebook_init");
+  // the GEMM result matrix of the hyper-encoder passes is all zero between GEMMs; establish that once
+  Z2Z_CUDA(cudaMemsetAsync(h->ws + plan.off_part, 0, plan.part_bytes, reinterpret_cast<cudaStream_t>(stream)), "codebook_init");
   z2z::ProfScope ps(&h->prof, z2z::kProfLzw, 1, reinterpret_cast<cudaStream_t>(stream));
   Z2Z_CUDA(z2z::launch_codebook_clear(v, reinterpret_cast<cudaStream_t>(stream)), "codebook_init");
   return Z2Z_OK;

@@ -70,7 +70,7 @@ struct WsPlan {
   size_t off_Ahl, off_Hhl;                        // bf16 hi/lo activations (tensor-core path)
   size_t off_g1_X, off_g1_QKV, off_g1_Ahl, off_g1_Hhl;   // second encoder of the decode step
   size_t off_words;                               // device words: [0] kernel error, [1] logits tiles
-  size_t off_part, part_bytes;                    // GEMM split-K partial tiles
+  size_t off_part, part_bytes;                    // fp32 GEMM results of the hyper-encoder passes
   size_t off_lpart, lpart_bytes;                  // logits partial reductions
   size_t off_plan, plan_bytes;                    // per-row-tile plan of the prompt-scoring logits kernel
   size_t off_step_out;                            // small per-step outputs

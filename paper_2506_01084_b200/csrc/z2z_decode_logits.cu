@@ -130,6 +130,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
     ctrl->abort = 0;
     mbar_init_fence();
   }
+  pdl_trigger();                                    // the next kernel may get resident behind this one
   if (warp == 0 && lane < 8) prefetch_tmap(lane == 0 ? &tm.h : (lane < 4 ? &tm.hk[lane - 1] : &tm.w[lane - 4]));
   __syncthreads();                                  // barriers exist; the producer starts at once
 
@@ -137,26 +138,39 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
     if (lane == 0) {
       // ---------------- producer -------------------------------------------------------------------
       const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
-      if (RESIDENT) {
-        const uint32_t bar = smem_u32(&ctrl->hid_full);
-        mbar_expect_tx(bar, hid_bytes);
-        for (int kb = 0; kb < p.ksteps; kb += p.hid_box_kb)
-          tma_load_3d(hid_base + (uint32_t)kb * hid_rows * 128, &tm.h, 0, 0, kb, bar, pol_a);
-      }
       int stage = 0; uint32_t phase = 0, job_i = 0;
-      bool ok = true;
+      int issued = 0;
+      bool ok = true, deps = false;
+      // W_U depends on no earlier kernel: its first stages are issued at once.  Hidden rows and
+      // codebook state do: before the ring's first wrap (and before anything else that needs
+      // them) the producer waits for the preceding kernel and loads the resident hidden rows.
+      auto need_deps = [&]() {
+        if (deps) return;
+        pdl_wait();
+        if (RESIDENT) {
+          const uint32_t bar = smem_u32(&ctrl->hid_full);
+          mbar_expect_tx(bar, hid_bytes);
+          for (int kb = 0; kb < p.ksteps; kb += p.hid_box_kb)
+            tma_load_3d(hid_base + (uint32_t)kb * hid_rows * 128, &tm.h, 0, 0, kb, bar, pol_a);
+        }
+        deps = true;
+      };
+      if (!RESIDENT) need_deps();                   // every stage carries a box of hidden rows
       auto publish = [&](const DecodeJob& j) {
         const uint32_t slot = job_i % kJobRing;
         ds->jobs[slot] = j;
         mbar_arrive(smem_u32(&ctrl->job_ready[slot]));          // release: the job is visible to waiters
         ++job_i;
       };
+      const int g_first = (int)blockIdx.x * p.fixed_granules;
       auto stream = [&](const DecodeJob& j) {
         const int big = j.cls == 2;
         const int ksb = big ? 1 : 2;
         const CUtensorMap* wm = &tm.w[j.wmap * 2 + big];
         const CUtensorMap* hm = &tm.hk[big ? 0 : 1];
         for (int ks = 0; ks < p.ksteps && ok; ks += ksb) {
+          if (issued == STAGES) need_deps();
+          ++issued;
           if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctrl->full[stage]);
           mbar_expect_tx(full, NT * 128 + (RESIDENT ? 0u : (uint32_t)(ksb * hid_rows * 128)));
@@ -167,7 +181,6 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
         }
       };
       // fixed share: 128-row jobs of W_U, known without any codebook state
-      const int g_first = (int)blockIdx.x * p.fixed_granules;
       for (int g = g_first; g < g_first + p.fixed_granules && ok; g += 2) {
         const int big = g + 2 <= g_first + p.fixed_granules;     // an odd share ends with one 64-row job
         const int rows = big ? NT : kGran;
@@ -178,6 +191,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
         stream(j);
       }
       // pool: the rest of W_U and every visible row of U_h, claimed 64 rows at a time
+      need_deps();
       if (ok && !mbar_wait(smem_u32(&ctrl->pref_ready), 0, &ctrl->abort)) ok = false;
       if (ok) {
         const int gs = (p.cb.V + kGran - 1) / kGran;
@@ -209,6 +223,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
     }
   } else {
     // ---------------- warps 1-5: session state, tensor memory, then MMA and epilogue roles --------------
+    pdl_wait();                                     // codebook counters, row tables, partial slots: all dependent
     if (warp == 1) {                                // prefix of per-sequence granule counts of U_h
       int carry = 0;
       for (int base = 0; base < p.cb.B; base += 32) {
@@ -436,8 +451,7 @@ static cudaError_t launch_decode(DecodeLogitsParams p, const DecodeLogitMaps& ma
   auto kern = resident ? k_decode_logits<NB, GENERIC, true> : k_decode_logits<NB, GENERIC, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<grid, kThreads, smem, s>>>(p, maps);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(grid), dim3(kThreads), smem, s, p, maps);
 }
 
 cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counters, int* err_word,

@@ -7,12 +7,15 @@
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
 #include "z2z_lzw_dev.cuh"
+#include "z2z_sm100.cuh"
 
 namespace z2z {
 
 __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateArgs a, EntryList el) {
   __shared__ int s_cnt[1024];
   __shared__ int s_warp[32];
+  sm100::pdl_trigger();
+  sm100::pdl_wait();               // the logits partials and the codebook state come from earlier kernels
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   for (int b = tid; b < 1024; b += blockDim.x) s_cnt[b] = 0;
   __syncthreads();
@@ -84,7 +87,7 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
 
 cudaError_t launch_decode_update(const CbView& cb, const DecodeUpdateArgs& a, const EntryList& el,
                                  cudaStream_t s) {
-  k_decode_update<<<1, 1024, 0, s>>>(cb, a, el);
+  return launch_pdl(k_decode_update, dim3(1), dim3(1024), 0, s, cb, a, el);
   return cudaGetLastError();
 }
 

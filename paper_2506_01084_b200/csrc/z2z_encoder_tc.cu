@@ -10,11 +10,19 @@
 //
 // Layout of a hi/lo operand with Rt rows: bf16 [2 * Rt, K], hi rows first, lo rows after.
 //
-// Launches per layer: GEMM(qkv) -> [sum partials + bias, attention] -> GEMM(o) ->
-// [sum + bias + residual, LayerNorm 2] -> GEMM(1) -> [sum + bias, GELU] -> GEMM(2) ->
-// [sum + bias + residual, LayerNorm 1 of the next layer | mean-pool into the cache].
+// GEMM output.  Every CTA of the stream-K GEMM adds its partial tiles (hi and lo parts alike)
+// into ONE fp32 matrix Y[group][Rt][J] with vector reductions in global memory; Y is all zero
+// whenever no GEMM result is pending.  The element-wise kernel after a GEMM reads each element of
+// that GEMM's result exactly once and stores zero back ("consume and clear"), for every row of
+// the pass whether or not it belongs to a live entry, which restores the invariant for the next
+// GEMM.  The session start clears Y once.
+//
+// Launches per layer: GEMM(qkv) -> [+ bias, attention] -> GEMM(o) -> [+ bias + residual,
+// LayerNorm 2] -> GEMM(1) -> [+ bias, GELU] -> GEMM(2) -> [+ bias + residual, LayerNorm 1 of the
+// next layer | mean-pool into the cache].  All are launched with programmatic serialization.
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
+#include "z2z_sm100.cuh"
 #include "z2z_stream.h"
 
 namespace z2z {
@@ -25,48 +33,6 @@ using bf16 = __nv_bfloat16;
 constexpr int kNT = kGemmNT;
 constexpr int kRowThreads = 256;
 constexpr int kMaxVec4 = 8;            // float4 per thread in the row kernels: d <= 8192
-
-// Where the partial tiles of one GEMM live and how they were cut (mirrors GemmSched).
-struct PartView {
-  const float* part;
-  long long slot_stride;     // floats
-  long long U, G;            // units and CTAs of the GEMM launch
-  int groups, tpg, ksteps;   // tiles per group, k-steps per tile
-  int lo_off;                // >0: lo rows sit lo_off rows below the hi rows inside the slot
-};
-
-// Slots holding the partial sums of one tile: slots (tile + c) for c in [c0, c1].
-struct TileSlots { long long tile; int c0, c1; };
-__device__ __forceinline__ TileSlots tile_slots(const PartView& pv, int rt, int g, int t) {
-  TileSlots s;
-  s.tile = ((long long)rt * pv.groups + g) * pv.tpg + t;
-  s.c0 = (int)owner_of(s.tile * pv.ksteps, pv.U, pv.G);
-  s.c1 = (int)owner_of((s.tile + 1) * pv.ksteps - 1, pv.U, pv.G);
-  return s;
-}
-// Sum over the slots, in slot order (deterministic), of 4 consecutive columns of local row lr.
-__device__ __forceinline__ float4 part_sum4(const PartView& pv, const TileSlots& ts, int lr, int cj) {
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c = ts.c0; c <= ts.c1; ++c) {
-    const float* s = pv.part + (ts.tile + c) * pv.slot_stride + (long long)lr * kNT + cj;
-    const float4 a = *reinterpret_cast<const float4*>(s);
-    acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
-    if (pv.lo_off) {
-      const float4 b = *reinterpret_cast<const float4*>(s + (long long)pv.lo_off * kNT);
-      acc.x += b.x; acc.y += b.y; acc.z += b.z; acc.w += b.w;
-    }
-  }
-  return acc;
-}
-__device__ __forceinline__ float part_sum1(const PartView& pv, const TileSlots& ts, int lr, int cj) {
-  float acc = 0.f;
-  for (int c = ts.c0; c <= ts.c1; ++c) {
-    const float* s = pv.part + (ts.tile + c) * pv.slot_stride + (long long)lr * kNT + cj;
-    acc += s[0];
-    if (pv.lo_off) acc += s[(long long)pv.lo_off * kNT];
-  }
-  return acc;
-}
 
 struct Ptr2 { const void* p[2]; };
 struct MPtr2 { void* p[2]; };
@@ -92,6 +58,12 @@ __device__ __forceinline__ void split_store4(bf16* hi, bf16* lo, float4 x) {
   L.y = pack_bf16(x.z - __bfloat162float(h2), x.w - __bfloat162float(h3));
   *reinterpret_cast<uint2*>(hi) = H;
   *reinterpret_cast<uint2*>(lo) = L;
+}
+// Read 4 consecutive GEMM results and leave zeros behind.
+__device__ __forceinline__ float4 take4(float* y) {
+  const float4 v = *reinterpret_cast<const float4*>(y);
+  *reinterpret_cast<float4*>(y) = make_float4(0.f, 0.f, 0.f, 0.f);
+  return v;
 }
 
 __device__ __forceinline__ int entry_len_tc(const CbView& cb, const EntryList& el, int e) {
@@ -149,6 +121,8 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
                                                               Ptr2 ln_w, Ptr2 ln_b, MPtr2 X, MPtr2 Ahl,
                                                               int d, int Rt, int has_ln) {
   __shared__ float sm[32];
+  sm100::pdl_trigger();            // the next kernel may start its prologue and weight prefetch
+  sm100::pdl_wait();               // everything read or written below depends on earlier kernels
   const int r = blockIdx.x, g = blockIdx.y, e = r / cb.M, i = r - e * cb.M;
   if (e >= el.off[cb.B + 1]) return;
   const int L = entry_len_tc(cb, el, e);
@@ -182,90 +156,73 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
                          reinterpret_cast<const bf16*>(ln_b.p[g]), hi, lo, d, sm);
 }
 
-// One row: x = X[r] + sum(partials) + bias, in registers.  Tiles' slot ranges are staged in smem.
-__device__ __forceinline__ void row_reduce_resid(const PartView& pv, int r, int g, const float* xrow,
-                                                 const bf16* bias, int d, int* s_c0, int* s_c1,
-                                                 float4 (&xv)[kMaxVec4]) {
-  const int nvec = d / 4, rt = r >> 7, lr = r & 127;
+// x = X[r] + Y[r] + bias for a valid row (Y consumed and cleared for every row); then
+// LayerNorm -> hi/lo for the next GEMM.  grid (rows, groups).
+__global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, EntryList el, float* Y, Ptr2 bias,
+                                                                    MPtr2 X, Ptr2 ln_w, Ptr2 ln_b, MPtr2 Ahl,
+                                                                    int d, int Rt) {
+  __shared__ float sm[32];
+  sm100::pdl_trigger();
+  sm100::pdl_wait();
+  const int r = blockIdx.x, g = blockIdx.y, e = r / cb.M, i = r - e * cb.M;
+  const bool valid = e < el.off[cb.B + 1] && i < entry_len_tc(cb, el, e);
+  float* y = Y + ((size_t)g * Rt + r) * d;
+  float* x = reinterpret_cast<float*>(X.p[g]) + (size_t)r * d;
+  const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
+  const int nvec = d / 4;
+  float4 xv[kMaxVec4];
 #pragma unroll
   for (int v = 0; v < kMaxVec4; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
-      const int col = idx * 4, t = col / kNT;
-      TileSlots ts;
-      ts.tile = ((long long)rt * pv.groups + g) * pv.tpg + t; ts.c0 = s_c0[t]; ts.c1 = s_c1[t];
-      const float4 p = part_sum4(pv, ts, lr, col - t * kNT);
-      const float4 xo = *reinterpret_cast<const float4*>(xrow + col);
-      const float4 bs = load_bf16x4(bias + col);
-      xv[v] = make_float4(xo.x + p.x + bs.x, xo.y + p.y + bs.y, xo.z + p.z + bs.z, xo.w + p.w + bs.w);
+      const float4 p = take4(y + idx * 4);
+      if (valid) {
+        const float4 xo = *reinterpret_cast<const float4*>(x + idx * 4);
+        const float4 b = load_bf16x4(bs + idx * 4);
+        xv[v] = make_float4(xo.x + p.x + b.x, xo.y + p.y + b.y, xo.z + p.z + b.z, xo.w + p.w + b.w);
+        *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
+      }
     }
   }
-}
-
-__device__ __forceinline__ void stage_tile_slots(const PartView& pv, int rt, int g, int n_tiles, int* s_c0,
-                                                 int* s_c1) {
-  for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
-    const TileSlots ts = tile_slots(pv, rt, g, t);
-    s_c0[t] = ts.c0; s_c1[t] = ts.c1;
-  }
-  __syncthreads();
-}
-
-// X[r] += sum(partials) + bias; then LayerNorm -> hi/lo for the next GEMM.  grid (rows, groups).
-__global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, EntryList el, PartView pv,
-                                                                    Ptr2 bias, MPtr2 X, Ptr2 ln_w, Ptr2 ln_b,
-                                                                    MPtr2 Ahl, int d, int Rt) {
-  __shared__ float sm[32];
-  __shared__ int s_c0[64], s_c1[64];
-  const int r = blockIdx.x, g = blockIdx.y, e = r / cb.M, i = r - e * cb.M;
-  if (e >= el.off[cb.B + 1]) return;
-  if (i >= entry_len_tc(cb, el, e)) return;      // padding rows stay zero in X and in hi/lo
-  stage_tile_slots(pv, r >> 7, g, d / kNT, s_c0, s_c1);
-  float* x = reinterpret_cast<float*>(X.p[g]) + (size_t)r * d;
-  float4 xv[kMaxVec4];
-  row_reduce_resid(pv, r, g, x, reinterpret_cast<const bf16*>(bias.p[g]), d, s_c0, s_c1, xv);
-  const int nvec = d / 4;
-#pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
-    const int idx = (int)threadIdx.x + v * kRowThreads;
-    if (idx < nvec) *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
-  }
+  if (!valid) return;                             // padding rows stay zero in X and in hi/lo
   bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)r * d;
   layernorm_split_regs(xv, nvec, reinterpret_cast<const bf16*>(ln_w.p[g]),
                        reinterpret_cast<const bf16*>(ln_b.p[g]), hi, hi + (size_t)Rt * d, d, sm);
 }
 
-// Last layer: x_i = X[r_i] + sum(partials) + bias for the entry's valid rows, cache row = mean_i x_i.
+// Last layer: x_i = X[r_i] + Y[r_i] + bias for the entry's valid rows, cache row = mean_i x_i.
 // grid (entries, groups).
-__global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb, EntryList el, PartView pv,
-                                                                      Ptr2 bias, MPtr2 X, MPtr2 cache,
-                                                                      MPtr2 cache_f32, int d) {
-  __shared__ int s_c0[64], s_c1[64];
+__global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb, EntryList el, float* Y, Ptr2 bias,
+                                                                      MPtr2 X, MPtr2 cache, MPtr2 cache_f32, int d,
+                                                                      int Rt) {
+  sm100::pdl_trigger();
+  sm100::pdl_wait();
   const int e = blockIdx.x, g = blockIdx.y;
-  if (e >= el.off[cb.B + 1]) return;
-  const int L = entry_len_tc(cb, el, e);
-  if (L <= 0) return;
+  const int L = e < el.off[cb.B + 1] ? entry_len_tc(cb, el, e) : 0;
   const int nvec = d / 4;
+  const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
   float4 acc[kMaxVec4];
 #pragma unroll
   for (int v = 0; v < kMaxVec4; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-  int staged_rt = -1;
-  for (int i = 0; i < L; ++i) {
+  for (int i = 0; i < cb.M; ++i) {
     const int r = e * cb.M + i;
-    if ((r >> 7) != staged_rt) {
-      __syncthreads();
-      stage_tile_slots(pv, r >> 7, g, d / kNT, s_c0, s_c1);
-      staged_rt = r >> 7;
-    }
-    float4 xv[kMaxVec4];
-    row_reduce_resid(pv, r, g, reinterpret_cast<const float*>(X.p[g]) + (size_t)r * d,
-                     reinterpret_cast<const bf16*>(bias.p[g]), d, s_c0, s_c1, xv);
+    float* y = Y + ((size_t)g * Rt + r) * d;
+    const float* x = reinterpret_cast<const float*>(X.p[g]) + (size_t)r * d;
 #pragma unroll
-    for (int v = 0; v < kMaxVec4; ++v)
-      if ((int)threadIdx.x + v * kRowThreads < nvec) {
-        acc[v].x += xv[v].x; acc[v].y += xv[v].y; acc[v].z += xv[v].z; acc[v].w += xv[v].w;
+    for (int v = 0; v < kMaxVec4; ++v) {
+      const int idx = (int)threadIdx.x + v * kRowThreads;
+      if (idx < nvec) {
+        const float4 p = take4(y + idx * 4);
+        if (i < L) {
+          const float4 xo = *reinterpret_cast<const float4*>(x + idx * 4);
+          const float4 b = load_bf16x4(bs + idx * 4);
+          acc[v].x += xo.x + p.x + b.x; acc[v].y += xo.y + p.y + b.y;
+          acc[v].z += xo.z + p.z + b.z; acc[v].w += xo.w + p.w + b.w;
+        }
       }
+    }
   }
+  if (L <= 0) return;
   const size_t dst = ((size_t)el.seq[e] * cb.cap + el.idx[e]) * d;
   const float inv = 1.0f / (float)L;
   bf16* out = reinterpret_cast<bf16*>(cache.p[g]);
@@ -285,6 +242,8 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb,
 // Zero-layer encoder (the parameter-free averaging variant): cache row = mean of X rows.
 __global__ void __launch_bounds__(kRowThreads) k_tc_pool(CbView cb, EntryList el, MPtr2 X, MPtr2 cache,
                                                          MPtr2 cache_f32, int d) {
+  sm100::pdl_trigger();
+  sm100::pdl_wait();
   const int e = blockIdx.x, g = blockIdx.y;
   if (e >= el.off[cb.B + 1]) return;
   const int L = entry_len_tc(cb, el, e);
@@ -303,16 +262,18 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_pool(CbView cb, EntryList el
   }
 }
 
-// H = GELU(sum(partials) + bias) -> hi/lo.  grid (tiles, ceil(rows / 4), groups), block 128:
-// warp w handles row 4 * blockIdx.y + w, each lane 4 columns of the tile.
-__global__ void __launch_bounds__(128) k_tc_reduce_gelu(CbView cb, EntryList el, PartView pv, Ptr2 bias,
-                                                        MPtr2 Hhl, int J, int R, int Rt) {
+// H = GELU(Y + bias) -> hi/lo (Y consumed and cleared).  grid (J / 128, ceil(rows / 4), groups),
+// block 128: warp w handles row 4 * blockIdx.y + w, each lane 4 columns of the 128-column tile.
+__global__ void __launch_bounds__(128) k_tc_reduce_gelu(CbView cb, EntryList el, float* Y, Ptr2 bias, MPtr2 Hhl,
+                                                        int J, int R, int Rt) {
+  sm100::pdl_trigger();
+  sm100::pdl_wait();
   const int t = blockIdx.x, g = blockIdx.z;
   const int r = blockIdx.y * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (r >= R || r / cb.M >= el.off[cb.B + 1]) return;
-  const TileSlots ts = tile_slots(pv, r >> 7, g, t);
-  const float4 p = part_sum4(pv, ts, r & 127, lane * 4);
+  if (r >= R) return;
   const int j = t * kNT + lane * 4;
+  const float4 p = take4(Y + ((size_t)g * Rt + r) * J + j);
+  if (r / cb.M >= el.off[cb.B + 1]) return;
   const float4 bs = load_bf16x4(reinterpret_cast<const bf16*>(bias.p[g]) + j);
   float4 v = make_float4(p.x + bs.x, p.y + bs.y, p.z + bs.z, p.w + bs.w);
   v.x = 0.5f * v.x * (1.0f + erff(v.x * 0.70710678118654752440f));
@@ -323,26 +284,29 @@ __global__ void __launch_bounds__(128) k_tc_reduce_gelu(CbView cb, EntryList el,
   split_store4(hi, hi + (size_t)Rt * J, v);
 }
 
-// q, k, v = sum(partials) + bias for one head of one entry (staged in shared memory), then
+// q, k, v = Y + bias for one head of one entry (consumed, cleared, staged in shared memory), then
 // bidirectional attention over the entry's valid rows; output as hi/lo.
-// grid (entries, heads, groups), block (32, M), dynamic smem M * 3 * dh floats.
-__global__ void k_tc_qkv_attention(CbView cb, EntryList el, PartView pv, Ptr2 bias, MPtr2 Ohl, int d,
-                                   int heads, int Rt) {
+// grid (entries, heads, groups), block (32, M), dynamic smem M * 3 * dh floats; dh % 4 == 0.
+__global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias, MPtr2 Ohl, int d, int heads,
+                                   int Rt) {
   extern __shared__ float s_qkv[];
+  sm100::pdl_trigger();
+  sm100::pdl_wait();
   const int e = blockIdx.x, h = blockIdx.y, g = blockIdx.z, i = threadIdx.y, lane = threadIdx.x;
-  if (e >= el.off[cb.B + 1]) return;
-  const int L = entry_len_tc(cb, el, e);
+  const int L = e < el.off[cb.B + 1] ? entry_len_tc(cb, el, e) : 0;
   const int dh = d / heads;
   const int r = e * cb.M + i;
-  if (i < L) {
+  {
     const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
-    TileSlots ts; ts.tile = -1; ts.c0 = ts.c1 = 0;
-    int cur_t = -1;
+    float* y = Y + ((size_t)g * Rt + r) * 3 * d;
     for (int w = 0; w < 3; ++w)
-      for (int c = lane; c < dh; c += 32) {
-        const int col = w * d + h * dh + c, t = col / kNT;
-        if (t != cur_t) { ts = tile_slots(pv, r >> 7, g, t); cur_t = t; }
-        s_qkv[(i * 3 + w) * dh + c] = part_sum1(pv, ts, r & 127, col - t * kNT) + __bfloat162float(bs[col]);
+      for (int c = lane * 4; c < dh; c += 128) {
+        const int col = w * d + h * dh + c;
+        const float4 p = take4(y + col);
+        if (i < L) {
+          const float4 b = load_bf16x4(bs + col);
+          *reinterpret_cast<float4*>(&s_qkv[(i * 3 + w) * dh + c]) = make_float4(p.x + b.x, p.y + b.y, p.z + b.z, p.w + b.w);
+        }
       }
   }
   __syncthreads();
@@ -395,7 +359,7 @@ int sm_count() {
 }  // namespace
 
 bool encoder_tc_supported(int d, int dff, int dtype, int heads, int M) {
-  if (heads < 1 || (size_t)M * 3 * (d / heads) * 4 > 48 * 1024) return false;
+  if (heads < 1 || (d / heads) % 4 != 0 || (size_t)M * 3 * (d / heads) * 4 > 48 * 1024) return false;
   return dtype == Z2Z_DTYPE_BF16 && d % kNT == 0 && dff % kNT == 0 && d <= 4 * kRowThreads * kMaxVec4;
 }
 
@@ -409,7 +373,9 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   const int row_tiles = (Rt + 127) / 128;
   const bool stacked = 2 * Rt <= 128;                  // hi and lo rows share one 128-row MMA
   const int n_sm = sm_count();
-  int G = n_sm;
+  float* Y = a0.part;                                  // GEMM results, all zero between GEMMs
+  const size_t wide = (size_t)(3 * d > dff ? 3 * d : dff);
+  if ((size_t)ng * Rt * wide * sizeof(float) > a0.part_bytes) return cudaErrorMemoryAllocation;
   auto P2 = [&](auto f) { Ptr2 p; p.p[0] = f(grp[0]); p.p[1] = ng > 1 ? f(grp[1]) : f(grp[0]); return p; };
   auto M2 = [&](auto f) { MPtr2 p; p.p[0] = f(grp[0]); p.p[1] = ng > 1 ? f(grp[1]) : f(grp[0]); return p; };
   auto W = [&](int i) { return P2([&](const EncoderArgs& a) { return a.w[i]; }); };
@@ -420,8 +386,8 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   const MPtr2 c32 = M2([](const EncoderArgs& a) { return (void*)a.cache_f32; });
   const Ptr2 table = P2([](const EncoderArgs& a) { return a.table; });
 
-  // one GEMM: activations (hi/lo, K columns) x weight [J, K] -> partial tiles
-  auto gemm = [&](const MPtr2& act, int K, int widx, int J, PartView& pv) -> cudaError_t {
+  // one GEMM: activations (hi/lo, K columns) x weight [J, K], added into Y[group][Rt][J]
+  auto gemm = [&](const MPtr2& act, int K, int widx, int J) -> cudaError_t {
     StreamGemmParams p{};
     p.row_tiles = row_tiles; p.groups = ng; p.tiles_per_group = J / kNT;
     p.ksteps = (K / 64 + kGemmKSB - 1) / kGemmKSB;
@@ -429,21 +395,16 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
     p.a_box_rows = stacked ? 2 * Rt : (Rt < 128 ? Rt : 128);
     p.a_part_row = Rt;
     p.out_rows = stacked ? 2 * Rt : (Rt < 128 ? Rt : 128);
-    p.part = a0.part;
-    p.slot_stride = (long long)p.out_rows * kNT;
+    p.out = Y; p.J = J; p.Rt = Rt; p.valid_rows = R; p.stacked = stacked ? 1 : 0;
     p.err = a0.err;
     const long long tiles = (long long)row_tiles * ng * p.tiles_per_group;
-    G = tiles * p.ksteps < n_sm ? (int)(tiles * p.ksteps) : n_sm;     // every CTA owns >= 1 unit
-    if ((size_t)(tiles + G) * p.slot_stride * 4 > a0.part_bytes) return cudaErrorMemoryAllocation;
+    const int G = tiles * p.ksteps < n_sm ? (int)(tiles * p.ksteps) : n_sm;     // every CTA owns >= 1 unit
     CUtensorMap maps[4];
     for (int g = 0; g < 2; ++g) {
       const int gg = g < ng ? g : 0;
       if (!make_tmap_bf16(&maps[g], act.p[gg], 2ll * Rt, K, p.a_box_rows)) return cudaErrorInvalidValue;
       if (!make_tmap_bf16(&maps[2 + g], grp[gg].w[widx], J, K, kNT)) return cudaErrorInvalidValue;
     }
-    pv.part = p.part; pv.slot_stride = p.slot_stride;
-    pv.U = tiles * p.ksteps; pv.G = G; pv.groups = ng; pv.tpg = p.tiles_per_group; pv.ksteps = p.ksteps;
-    pv.lo_off = stacked ? Rt : 0;
     ProfScope ps(prof, kProfEncGemm, 1, s);
     return launch_stream_gemm(p, maps, G, s);
   };
@@ -451,43 +412,44 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   cudaError_t e;
   {
     ProfScope ps(prof, kProfEncOther, 1, s);
-    k_tc_gather_ln<<<dim3(R, ng), kRowThreads, 0, s>>>(cb, el, table, W(0), a0.layers ? W(1) : W(0),
-                                                       a0.layers ? W(2) : W(0), X, Ahl, d, Rt, a0.layers > 0);
+    launch_pdl(k_tc_gather_ln, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, table, W(0), a0.layers ? W(1) : W(0),
+               a0.layers ? W(2) : W(0), X, Ahl, d, Rt, a0.layers > 0 ? 1 : 0);
   }
   if (a0.layers == 0) {
     ProfScope ps(prof, kProfEncOther, 1, s);
-    k_tc_pool<<<dim3(E, ng), kRowThreads, 0, s>>>(cb, el, X, cache, c32, d);
+    launch_pdl(k_tc_pool, dim3(E, ng), dim3(kRowThreads), 0, s, cb, el, X, cache, c32, d);
   }
   const int dh = d / a0.heads;
   for (int l = 0; l < a0.layers; ++l) {
     const int o = 1 + 12 * l;
     const bool last = l + 1 == a0.layers;
-    PartView pv{};
-    if ((e = gemm(Ahl, d, o + 2, 3 * d, pv)) != cudaSuccess) return e;
+    if ((e = gemm(Ahl, d, o + 2, 3 * d)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_qkv_attention<<<dim3(E, a0.heads, ng), dim3(32, M), (size_t)M * 3 * dh * 4, s>>>(
-          cb, el, pv, W(o + 3), Ahl, d, a0.heads, Rt);
+      launch_pdl(k_tc_qkv_attention, dim3(E, a0.heads, ng), dim3(32, M), (size_t)M * 3 * dh * 4, s, cb, el, Y,
+                 W(o + 3), Ahl, d, a0.heads, Rt);
     }
-    if ((e = gemm(Ahl, d, o + 4, d, pv)) != cudaSuccess) return e;
+    if ((e = gemm(Ahl, d, o + 4, d)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_reduce_resid_ln<<<dim3(R, ng), kRowThreads, 0, s>>>(cb, el, pv, W(o + 5), X, W(o + 6), W(o + 7),
-                                                               Ahl, d, Rt);
+      launch_pdl(k_tc_reduce_resid_ln, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 5), X, W(o + 6),
+                 W(o + 7), Ahl, d, Rt);
     }
-    if ((e = gemm(Ahl, d, o + 8, dff, pv)) != cudaSuccess) return e;
+    if ((e = gemm(Ahl, d, o + 8, dff)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_reduce_gelu<<<dim3(dff / kNT, (R + 3) / 4, ng), 128, 0, s>>>(cb, el, pv, W(o + 9), Hhl, dff, R, Rt);
+      launch_pdl(k_tc_reduce_gelu, dim3(dff / kNT, (R + 3) / 4, ng), dim3(128), 0, s, cb, el, Y, W(o + 9), Hhl, dff,
+                 R, Rt);
     }
-    if ((e = gemm(Hhl, dff, o + 10, d, pv)) != cudaSuccess) return e;
+    if ((e = gemm(Hhl, dff, o + 10, d)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
       if (last)
-        k_tc_reduce_resid_pool<<<dim3(E, ng), kRowThreads, 0, s>>>(cb, el, pv, W(o + 11), X, cache, c32, d);
+        launch_pdl(k_tc_reduce_resid_pool, dim3(E, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 11), X, cache, c32,
+                   d, Rt);
       else
-        k_tc_reduce_resid_ln<<<dim3(R, ng), kRowThreads, 0, s>>>(cb, el, pv, W(o + 11), X, W(o + 12), W(o + 13),
-                                                                 Ahl, d, Rt);
+        launch_pdl(k_tc_reduce_resid_ln, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 11), X, W(o + 12),
+                   W(o + 13), Ahl, d, Rt);
     }
   }
   return cudaGetLastError();

@@ -8,6 +8,21 @@
 
 namespace z2z {
 
+// Launch with programmatic stream serialization: the kernel may begin (up to its pdl_wait())
+// while the previous kernel of the stream is still running.  Every kernel launched this way
+// calls pdl_wait() before it reads what earlier kernels wrote and before it writes anything.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(static_cast<Args&&>(args))...);
+}
+
 // ---- z2z_api.cu ------------------------------------------------------------------------------
 void set_last_error(const char* msg);      // text returned by z2z_last_error on this thread
 
@@ -36,7 +51,7 @@ struct EncoderArgs {
   float* cache_f32;             // optional
   float *X, *A, *QKV, *H;       // fp32 scratch, rows = chunk * M
   __nv_bfloat16 *Ahl, *Hhl;     // bf16 hi/lo scratch for the tensor-core path
-  float* part;                  // split-K partial tiles
+  float* part;                  // fp32 GEMM results [groups][rows][J], zero between GEMMs
   size_t part_bytes;
   int entries;                  // host bound on the entries of this pass (<= chunk)
   int* err;                     // device error word of the tensor-core kernels

@@ -137,18 +137,36 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
   const uint32_t stage_bytes = a_parts * a_part_bytes + (uint32_t)KSB * NT * 128;   // smem stride of a stage
   const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
   int stage = 0; uint32_t phase = 0;
+  // The weight tiles depend on no earlier kernel, the activation tiles do.  During the first
+  // pass over the ring only the weight boxes are issued and the activation boxes are noted; once
+  // the ring is full (or the work ends) the producer waits for the preceding kernel and issues
+  // them.  With an ordinary launch the wait returns at once.
+  struct Deferred { uint32_t dst, bar; int map, x, y; };
+  Deferred def[kMaxStages * 2 * KSB];
+  int n_def = 0, issued = 0;
+  bool deps = false;
+  auto need_deps = [&]() {
+    if (deps) return;
+    pdl_wait();
+    for (int i = 0; i < n_def; ++i) tma_load_2d(def[i].dst, amaps[def[i].map], def[i].x, def[i].y, def[i].bar, pol_a);
+    deps = true;
+  };
   Job j;
   while (sched.next(j, NT)) {
     for (int ks = j.kb0; ks < j.kb1; ++ks) {
+      if (issued == STAGES) need_deps();
       if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) return;
       const uint32_t full = smem_u32(&ctrl->full[stage]);
       mbar_expect_tx(full, a_parts * a_part_bytes + (uint32_t)KSB * j.nrows * 128);
       const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
       for (int part = 0; part < a_parts; ++part)
 #pragma unroll
-        for (int i = 0; i < KSB; ++i)
-          tma_load_2d(sb + part * a_part_bytes + i * a_box_rows * 128, amaps[j.amap],
-                      (ks * KSB + i) * 64, j.arow + part * a_part_row, full, pol_a);
+        for (int i = 0; i < KSB; ++i) {
+          const uint32_t dst = sb + part * a_part_bytes + i * a_box_rows * 128;
+          const int x = (ks * KSB + i) * 64, y = j.arow + part * a_part_row;
+          if (deps) tma_load_2d(dst, amaps[j.amap], x, y, full, pol_a);
+          else { def[n_def].dst = dst; def[n_def].bar = full; def[n_def].map = j.amap; def[n_def].x = x; def[n_def].y = y; ++n_def; }
+        }
       // the W rows of the job go out as few boxes as possible: largest power-of-two box first
       for (int r0 = 0; r0 < j.nrows;) {
         int cls = j.wbox_classes - 1;
@@ -160,9 +178,11 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
                       (ks * KSB + i) * 64, j.wrow + r0, full, pol_w);
         r0 += j.wbox_min << cls;
       }
+      ++issued;
       if (++stage == STAGES) { stage = 0; phase ^= 1u; }
     }
   }
+  need_deps();
 }
 
 template <int NT, int KSB, int STAGES, class Sched>
@@ -233,6 +253,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm);
   const uint32_t stage_base = smem_u32(sm + 1024);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_trigger();                                   // the next kernel may get resident behind this one
   setup_barriers<STAGES>(ctrl);
   if (warp == 0 && lane == 0) { prefetch_tmap(&tmA0); prefetch_tmap(&tmW0); if (p.groups > 1) { prefetch_tmap(&tmA1); prefetch_tmap(&tmW1); } }
   __syncthreads();
@@ -255,6 +276,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
       mma_role<NT, KSB, STAGES>(sched, ctrl, stage_base, p.a_parts, p.a_box_rows, tmem_base);
     }
   } else {
+    pdl_wait();                                      // the partial slots may still be read by the kernel before
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
     const int row = q * 32 + lane;
     GemmSched sched(p, NT);
@@ -265,16 +287,21 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
       if (!mbar_wait(smem_u32(&ctrl->acc_full[buf]), aph, &ctrl->abort)) break;
       tc_fence_after();
       if (q * 32 < p.out_rows) {
-        float* dst = p.part + j.slot * p.slot_stride + (long long)row * NT;
+        // accumulator row -> result row: with hi and lo stacked in one tile the lo rows lie Rt below
+        const int orow = (p.stacked && row >= p.Rt) ? row - p.Rt : row;
+        const int grow = j.arow + orow;
+        const bool live = row < p.out_rows && grow < p.valid_rows;
+        float* dst = p.out + ((size_t)j.amap * p.Rt + grow) * p.J + j.wrow;
 #pragma unroll 1
         for (int c0 = 0; c0 < NT; c0 += 32) {
           uint32_t v[32];
           tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * NT + c0, v);
           tmem_ld_wait();
-          if (row < p.out_rows) {
+          if (live) {
 #pragma unroll
             for (int x = 0; x < 32; x += 4)
-              *reinterpret_cast<uint4*>(dst + c0 + x) = make_uint4(v[x], v[x + 1], v[x + 2], v[x + 3]);
+              red_add_f32x4(dst + c0 + x, __uint_as_float(v[x]), __uint_as_float(v[x + 1]), __uint_as_float(v[x + 2]),
+                            __uint_as_float(v[x + 3]));
           }
         }
       }
@@ -302,6 +329,7 @@ k_stream_logits(const StreamLogitsParams p, const __grid_constant__ LogitMaps tm
   int* s_pref = reinterpret_cast<int*>(sm + 1024);              // [B + 1] <= 4100 bytes
   const uint32_t stage_base = smem_u32(sm + 1024 + 5120);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_wait();                                      // the prologue already reads codebook state
   setup_barriers<STAGES>(ctrl);
   for (int b = threadIdx.x; b < p.cb.B; b += kThreads) s_pref[b + 1] = (p.cb.n[b] + kLogitGran - 1) / kLogitGran;
   if (warp == 0 && lane < 1 + 2 * kLogitBoxClasses) prefetch_tmap(lane == 0 ? &tm.h : &tm.w[lane - 1]);
@@ -520,8 +548,7 @@ static cudaError_t launch_gemm_t(const StreamGemmParams& p, const CUtensorMap* m
   auto kern = k_stream_gemm<NT, KSB, STAGES>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<grid, kThreads, smem, s>>>(p, maps[0], maps[1], maps[2], maps[3]);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(grid), dim3(kThreads), smem, s, p, maps[0], maps[1], maps[2], maps[3]);
 }
 
 // Launches the stream-K GEMM.  maps = {A group 0, A group 1, W group 0, W group 1}.

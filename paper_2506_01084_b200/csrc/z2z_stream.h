@@ -21,10 +21,6 @@ struct LogitMaps {
   CUtensorMap w[2 * kLogitBoxClasses];
 };
 
-// Stream-K GEMM over `groups` independent problems of identical shape (the two hyper-encoders).
-// The unit space is (group, tile, k-step); CTA c of G owns units [floor(cU/G), floor((c+1)U/G)).
-// Every maximal run of units inside one tile and one CTA produces one fp32 partial tile of
-// out_rows x NT values in slot (global tile index + c).
 // ---- decode logits kernel (z2z_decode_logits.cu) ---------------------------------------------
 // Tensor maps, all of the form [k-block][row][64 columns]: hidden rows as one resident operand
 // (h) and per stage with 1, 2 or 4 k-blocks (hk[0..2]); W_U and U_h as boxes of 64 rows x 2
@@ -51,15 +47,21 @@ bool decode_logits_applies(const LogitsArgs& a);
 cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counters, int* err_word,
                               LogitsPartInfo* info, Prof* prof, cudaStream_t s);
 
+// Stream-K GEMM over `groups` independent problems of identical shape (the two hyper-encoders).
+// The unit space is (group, tile, k-step); CTA c of G owns units [floor(cU/G), floor((c+1)U/G)).
+// Every maximal run of units inside one tile and one CTA is one accumulator, which the CTA adds
+// into the fp32 result matrix out[group][Rt][J] with reductions in global memory.
 struct StreamGemmParams {
   int row_tiles;         // 128-row tiles of A (outermost dimension of the unit space)
   int groups, tiles_per_group, ksteps;
   int a_box_rows;        // rows per TMA box of A (multiple of 8, <= 128)
   int a_parts;           // MMA row groups per k16: 1, or 2 when hi and lo rows do not fit 128 rows
   int a_part_row;        // first global row of part 1
-  int out_rows;          // accumulator rows stored
-  float* part;
-  long long slot_stride; // floats per slot
+  int out_rows;          // accumulator rows that carry results
+  float* out;            // [groups][Rt][J] fp32, zero before the first add
+  int J, Rt;
+  int valid_rows;        // rows of the pass (results of rows beyond them are dropped)
+  int stacked;           // 1: accumulator rows [Rt, 2 Rt) are the lo parts of rows [0, Rt)
   int* err;
 };
 

@@ -390,7 +390,8 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   auto gemm = [&](const MPtr2& act, int K, int widx, int J) -> cudaError_t {
     StreamGemmParams p{};
     p.row_tiles = row_tiles; p.groups = ng; p.tiles_per_group = J / kNT;
-    p.ksteps = (K / 64 + kGemmKSB - 1) / kGemmKSB;
+    p.ksb = stacked ? 2 : 1;                       // few rows: larger boxes, fewer TMA operations per byte
+    p.ksteps = (K / 64 + p.ksb - 1) / p.ksb;
     p.a_parts = stacked ? 1 : 2;
     p.a_box_rows = stacked ? 2 * Rt : (Rt < 128 ? Rt : 128);
     p.a_part_row = Rt;
@@ -402,8 +403,8 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
     CUtensorMap maps[4];
     for (int g = 0; g < 2; ++g) {
       const int gg = g < ng ? g : 0;
-      if (!make_tmap_bf16(&maps[g], act.p[gg], 2ll * Rt, K, p.a_box_rows)) return cudaErrorInvalidValue;
-      if (!make_tmap_bf16(&maps[2 + g], grp[gg].w[widx], J, K, kNT)) return cudaErrorInvalidValue;
+      if (!make_tmap_bf16_kblocks(&maps[g], act.p[gg], 2ll * Rt, K, p.a_box_rows, p.ksb)) return cudaErrorInvalidValue;
+      if (!make_tmap_bf16_kblocks(&maps[2 + g], grp[gg].w[widx], J, K, kNT, p.ksb)) return cudaErrorInvalidValue;
     }
     ProfScope ps(prof, kProfEncGemm, 1, s);
     return launch_stream_gemm(p, maps, G, s);

@@ -141,14 +141,14 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
   // pass over the ring only the weight boxes are issued and the activation boxes are noted; once
   // the ring is full (or the work ends) the producer waits for the preceding kernel and issues
   // them.  With an ordinary launch the wait returns at once.
-  struct Deferred { uint32_t dst, bar; int map, x, y; };
-  Deferred def[kMaxStages * 2 * KSB];
+  struct Deferred { uint32_t dst, bar; int map, row, kb; };
+  Deferred def[kMaxStages * 2];
   int n_def = 0, issued = 0;
   bool deps = false;
   auto need_deps = [&]() {
     if (deps) return;
     pdl_wait();
-    for (int i = 0; i < n_def; ++i) tma_load_2d(def[i].dst, amaps[def[i].map], def[i].x, def[i].y, def[i].bar, pol_a);
+    for (int i = 0; i < n_def; ++i) tma_load_3d(def[i].dst, amaps[def[i].map], 0, def[i].row, def[i].kb, def[i].bar, pol_a);
     deps = true;
   };
   Job j;
@@ -159,23 +159,20 @@ __device__ __forceinline__ void producer_role(Sched& sched, Ctrl* ctrl, uint32_t
       const uint32_t full = smem_u32(&ctrl->full[stage]);
       mbar_expect_tx(full, a_parts * a_part_bytes + (uint32_t)KSB * j.nrows * 128);
       const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
-      for (int part = 0; part < a_parts; ++part)
-#pragma unroll
-        for (int i = 0; i < KSB; ++i) {
-          const uint32_t dst = sb + part * a_part_bytes + i * a_box_rows * 128;
-          const int x = (ks * KSB + i) * 64, y = j.arow + part * a_part_row;
-          if (deps) tma_load_2d(dst, amaps[j.amap], x, y, full, pol_a);
-          else { def[n_def].dst = dst; def[n_def].bar = full; def[n_def].map = j.amap; def[n_def].x = x; def[n_def].y = y; ++n_def; }
-        }
+      // one box per operand part: KSB k-blocks of the rows, laid out k-block after k-block
+      for (int part = 0; part < a_parts; ++part) {
+        const uint32_t dst = sb + part * a_part_bytes;
+        const int row = j.arow + part * a_part_row;
+        if (deps) tma_load_3d(dst, amaps[j.amap], 0, row, ks * KSB, full, pol_a);
+        else { def[n_def].dst = dst; def[n_def].bar = full; def[n_def].map = j.amap; def[n_def].row = row; def[n_def].kb = ks * KSB; ++n_def; }
+      }
       // the W rows of the job go out as few boxes as possible: largest power-of-two box first
+      // (several boxes only with KSB == 1: a box's k-blocks lie one box height apart)
       for (int r0 = 0; r0 < j.nrows;) {
         int cls = j.wbox_classes - 1;
         while (cls > 0 && (j.wbox_min << cls) > j.nrows - r0) --cls;
-        const CUtensorMap* wm = wmaps[j.wmap * j.wbox_classes + cls];
-#pragma unroll
-        for (int i = 0; i < KSB; ++i)
-          tma_load_2d(sb + a_parts * a_part_bytes + i * NT * 128 + r0 * 128, wm,
-                      (ks * KSB + i) * 64, j.wrow + r0, full, pol_w);
+        tma_load_3d(sb + a_parts * a_part_bytes + r0 * 128, wmaps[j.wmap * j.wbox_classes + cls], 0, j.wrow + r0,
+                    ks * KSB, full, pol_w);
         r0 += j.wbox_min << cls;
       }
       ++issued;
@@ -551,15 +548,22 @@ static cudaError_t launch_gemm_t(const StreamGemmParams& p, const CUtensorMap* m
   return launch_pdl(kern, dim3(grid), dim3(kThreads), smem, s, p, maps[0], maps[1], maps[2], maps[3]);
 }
 
-// Launches the stream-K GEMM.  maps = {A group 0, A group 1, W group 0, W group 1}.
-cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
-  constexpr int NT = kGemmNT, KSB = kGemmKSB;
+// Launches the stream-K GEMM.  maps = {A group 0, A group 1, W group 0, W group 1}, built for
+// p.ksb k-blocks per box.
+template <int KSB>
+static cudaError_t launch_stream_gemm_k(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
+  constexpr int NT = kGemmNT;
   const int st = pick_stages<NT, KSB>(p.a_parts, p.a_box_rows, 0);
   if (st >= 8) return launch_gemm_t<NT, KSB, 8>(p, maps, grid, s);
   if (st >= 6) return launch_gemm_t<NT, KSB, 6>(p, maps, grid, s);
   if (st >= 4) return launch_gemm_t<NT, KSB, 4>(p, maps, grid, s);
   if (st >= 3) return launch_gemm_t<NT, KSB, 3>(p, maps, grid, s);
   return cudaErrorInvalidConfiguration;
+}
+cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
+  if (p.ksb == 2) return launch_stream_gemm_k<2>(p, maps, grid, s);
+  if (p.ksb == 1) return launch_stream_gemm_k<1>(p, maps, grid, s);
+  return cudaErrorInvalidValue;
 }
 
 template <int NT, int KSB, int STAGES>
@@ -594,11 +598,11 @@ cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, i
   p.vt_out = vt_word; p.err = err_word;
   if ((size_t)a.N * p.part_stride * sizeof(LogitPartial) > a.lpart_bytes) return cudaErrorMemoryAllocation;
   LogitMaps maps;
-  if (!make_tmap_bf16(&maps.h, a.hidden, a.N, a.d, p.a_box_rows)) return cudaErrorInvalidValue;
+  if (!make_tmap_bf16_kblocks(&maps.h, a.hidden, a.N, a.d, p.a_box_rows, kLogitKSB)) return cudaErrorInvalidValue;
   for (int c = 0; c < kLogitBoxClasses; ++c) {
-    if (!make_tmap_bf16(&maps.w[c], a.WU, cb.V, a.d, kLogitGran << c)) return cudaErrorInvalidValue;
+    if (!make_tmap_bf16_kblocks(&maps.w[c], a.WU, cb.V, a.d, kLogitGran << c, kLogitKSB)) return cudaErrorInvalidValue;
     if (cb.cap > 0) {
-      if (!make_tmap_bf16(&maps.w[kLogitBoxClasses + c], a.Uh, (long long)cb.B * cb.cap, a.d, kLogitGran << c))
+      if (!make_tmap_bf16_kblocks(&maps.w[kLogitBoxClasses + c], a.Uh, (long long)cb.B * cb.cap, a.d, kLogitGran << c, kLogitKSB))
         return cudaErrorInvalidValue;
     } else {
       maps.w[kLogitBoxClasses + c] = maps.w[c];

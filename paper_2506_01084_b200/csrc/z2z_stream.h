@@ -9,7 +9,7 @@
 namespace z2z {
 
 constexpr int kMaxStages = 8;
-constexpr int kGemmNT = 128, kGemmKSB = 1;      // weight rows per tile, 64-wide k blocks per stage
+constexpr int kGemmNT = 128;                    // weight rows per tile of the stream-K GEMM
 constexpr int kLogitNT = 128, kLogitKSB = 1;
 constexpr int kLogitGran = 32;                  // scheduling granule of the logits kernel, in weight rows (TMA boxes of
                                                 // fewer rows stream several times slower)
@@ -54,6 +54,7 @@ cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counte
 struct StreamGemmParams {
   int row_tiles;         // 128-row tiles of A (outermost dimension of the unit space)
   int groups, tiles_per_group, ksteps;
+  int ksb;               // 64-column k-blocks per stage and TMA box: 2 for few rows (decode), else 1
   int a_box_rows;        // rows per TMA box of A (multiple of 8, <= 128)
   int a_parts;           // MMA row groups per k16: 1, or 2 when hi and lo rows do not fit 128 rows
   int a_part_row;        // first global row of part 1

@@ -33,6 +33,7 @@ using bf16 = __nv_bfloat16;
 constexpr int kNT = kGemmNT;
 constexpr int kRowThreads = 256;
 constexpr int kMaxVec4 = 8;            // float4 per thread in the row kernels: d <= 8192
+constexpr int kPairPassMinRows = 1024; // passes of at least this many rows use the CTA-pair GEMM
 
 struct Ptr2 { const void* p[2]; };
 struct MPtr2 { void* p[2]; };
@@ -345,6 +346,76 @@ __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias,
   }
 }
 
+// LayerNorm of the valid rows of X -> hi/lo (prompt-sized passes: the GEMM epilogue has already
+// added bias and residual into X).  grid (rows), one encoder.
+__global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(CbView cb, EntryList el, const float* X, const bf16* ln_w,
+                                                            const bf16* ln_b, bf16* Ahl, int d, int Rt) {
+  __shared__ float sm[32];
+  const int r = blockIdx.x, e = r / cb.M, i = r - e * cb.M;
+  if (e >= el.off[cb.B + 1] || i >= entry_len_tc(cb, el, e)) return;     // padding rows stay zero in hi/lo
+  const float* x = X + (size_t)r * d;
+  const int nvec = d / 4;
+  float4 xv[kMaxVec4];
+#pragma unroll
+  for (int v = 0; v < kMaxVec4; ++v) {
+    const int idx = (int)threadIdx.x + v * kRowThreads;
+    if (idx < nvec) xv[v] = *reinterpret_cast<const float4*>(x + idx * 4);
+  }
+  bf16* hi = Ahl + (size_t)r * d;
+  layernorm_split_regs(xv, nvec, ln_w, ln_b, hi, hi + (size_t)Rt * d, d, sm);
+}
+
+// Bidirectional attention inside one entry from fp32 q, k, v rows [R, 3d] (bias already added);
+// output as hi/lo.  grid (entries, heads), block (32, M), dynamic smem M * 3 * dh floats.
+__global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, bf16* Ohl, int d, int heads, int Rt) {
+  extern __shared__ float s_qkv[];
+  const int e = blockIdx.x, h = blockIdx.y, i = threadIdx.y, lane = threadIdx.x;
+  if (e >= el.off[cb.B + 1]) return;
+  const int L = entry_len_tc(cb, el, e);
+  const int dh = d / heads;
+  const int r = e * cb.M + i;
+  if (i < L) {
+    const float* y = QKV + (size_t)r * 3 * d;
+    for (int w = 0; w < 3; ++w)
+      for (int c = lane * 4; c < dh; c += 128)
+        *reinterpret_cast<float4*>(&s_qkv[(i * 3 + w) * dh + c]) = *reinterpret_cast<const float4*>(y + w * d + h * dh + c);
+  }
+  __syncthreads();
+  if (i >= L) return;                          // padding rows of the operand stay zero
+  const float* q = s_qkv + (i * 3) * dh;
+  const float scale = 1.0f / sqrtf((float)dh);
+  float s[kMaxM];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < kMaxM; ++j) {
+    s[j] = -INFINITY;
+    if (j < L) {
+      const float* kp = s_qkv + (j * 3 + 1) * dh;
+      float p = 0.f;
+      for (int c = lane; c < dh; c += 32) p = fmaf(q[c], kp[c], p);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) p += __shfl_xor_sync(0xffffffffu, p, off);
+      s[j] = p * scale;
+      mx = fmaxf(mx, s[j]);
+    }
+  }
+  float den = 0.f;
+#pragma unroll
+  for (int j = 0; j < kMaxM; ++j) { s[j] = j < L ? expf(s[j] - mx) : 0.f; den += s[j]; }
+  const float inv = 1.0f / den;
+  bf16* hi = Ohl + (size_t)r * d + (size_t)h * dh;
+  bf16* lo = hi + (size_t)Rt * d;
+  for (int c = lane; c < dh; c += 32) {
+    float v = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxM; ++j)
+      if (j < L) v = fmaf(s[j] * inv, s_qkv[(j * 3 + 2) * dh + c], v);
+    const bf16 hh = __float2bfloat16_rn(v);
+    hi[c] = hh;
+    lo[c] = __float2bfloat16_rn(v - __bfloat162float(hh));
+  }
+}
+
 int sm_count() {
   static int n = 0;
   if (!n) {
@@ -363,12 +434,65 @@ bool encoder_tc_supported(int d, int dff, int dtype, int heads, int M) {
   return dtype == Z2Z_DTYPE_BF16 && d % kNT == 0 && dff % kNT == 0 && d <= 4 * kRowThreads * kMaxVec4;
 }
 
+// Prompt-sized pass of ONE encoder (thousands of rows): the linear layers run as CTA-pair GEMMs
+// that own whole output tiles, so bias, residual and GELU are applied in their epilogues; only
+// attention, LayerNorm and pooling remain as separate kernels.
+static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a, const EntryList& el, int E,
+                                         Prof* prof, cudaStream_t s) {
+  const int d = a.d, dff = a.dff, M = cb.M;
+  const int R = E * M, Rt = (R + 7) / 8 * 8;
+  auto Wp = [&](int i) { return reinterpret_cast<const bf16*>(a.w[i]); };
+  Ptr2 table, pos, lw, lb; MPtr2 X, Ahl, cache, c32;
+  table.p[0] = table.p[1] = a.table; pos.p[0] = pos.p[1] = a.w[0];
+  lw.p[0] = lw.p[1] = a.layers ? a.w[1] : a.w[0]; lb.p[0] = lb.p[1] = a.layers ? a.w[2] : a.w[0];
+  X.p[0] = X.p[1] = a.X; Ahl.p[0] = Ahl.p[1] = a.Ahl; cache.p[0] = cache.p[1] = a.cache; c32.p[0] = c32.p[1] = a.cache_f32;
+  PairGemmParams g{};
+  g.cb = cb; g.el = el; g.R = R; g.Rt = Rt; g.err = a.err;
+  auto gemm = [&](const bf16* act, int K, int widx, int J, int epi, float* out, bf16* out_hl) -> cudaError_t {
+    PairGemmParams p = g;
+    p.J = J; p.bias = a.w[widx + 1]; p.out = out; p.out_hl = out_hl;
+    ProfScope ps(prof, kProfEncGemm, 1, s);
+    return launch_pair_gemm(p, act, a.w[widx], K, epi, s);
+  };
+  {
+    ProfScope ps(prof, kProfEncOther, 1, s);
+    launch_pdl(k_tc_gather_ln, dim3(R, 1), dim3(kRowThreads), 0, s, cb, el, table, pos, lw, lb, X, Ahl, d, Rt,
+               a.layers > 0 ? 1 : 0);
+  }
+  const int dh = d / a.heads;
+  cudaError_t e;
+  for (int l = 0; l < a.layers; ++l) {
+    const int o = 1 + 12 * l;
+    if ((e = gemm(a.Ahl, d, o + 2, 3 * d, kEpiStore, a.QKV, nullptr)) != cudaSuccess) return e;
+    {
+      ProfScope ps(prof, kProfEncOther, 1, s);
+      k_tc_attention_rows<<<dim3(E, a.heads), dim3(32, M), (size_t)M * 3 * dh * 4, s>>>(cb, el, a.QKV, a.Ahl, d,
+                                                                                         a.heads, Rt);
+    }
+    if ((e = gemm(a.Ahl, d, o + 4, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
+    {
+      ProfScope ps(prof, kProfEncOther, 1, s);
+      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(cb, el, a.X, Wp(o + 6), Wp(o + 7), a.Ahl, d, Rt);
+    }
+    if ((e = gemm(a.Ahl, d, o + 8, dff, kEpiGelu, nullptr, a.Hhl)) != cudaSuccess) return e;
+    if ((e = gemm(a.Hhl, dff, o + 10, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
+    if (l + 1 < a.layers) {
+      ProfScope ps(prof, kProfEncOther, 1, s);
+      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(cb, el, a.X, Wp(o + 12), Wp(o + 13), a.Ahl, d, Rt);
+    }
+  }
+  ProfScope ps(prof, kProfEncOther, 1, s);
+  launch_pdl(k_tc_pool, dim3(E, 1), dim3(kRowThreads), 0, s, cb, el, X, cache, c32, d);
+  return cudaGetLastError();
+}
+
 cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng, const EntryList& el,
                                 Prof* prof, cudaStream_t s) {
   const EncoderArgs& a0 = grp[0];
   const int d = a0.d, dff = a0.dff, M = cb.M;
   const int E = a0.entries < el.chunk ? a0.entries : el.chunk;
   const int R = E * M;                                 // rows of this pass
+  if (ng == 1 && R >= kPairPassMinRows) return run_encoder_pass_pair(cb, a0, el, E, prof, s);
   const int Rt = (R + 7) / 8 * 8;                      // rows per hi (or lo) block
   const int row_tiles = (Rt + 127) / 128;
   const bool stacked = 2 * Rt <= 128;                  // hi and lo rows share one 128-row MMA

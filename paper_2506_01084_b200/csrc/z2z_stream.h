@@ -92,6 +92,22 @@ struct PrefillLogitsParams {
   int* err;
 };
 
+// CTA-pair GEMM of the prompt-sized hyper-encoder passes (z2z_pair_gemm.cu).
+enum { kEpiStore = 0, kEpiResid = 1, kEpiGelu = 2 };
+struct PairGemmParams {
+  CbView cb;
+  EntryList el;
+  int R, Rt;             // rows of the pass; rows per hi (or lo) block of the operands
+  int J;                 // output columns (a multiple of 128)
+  const void* bias;      // [J] bf16
+  float* out;            // kEpiStore / kEpiResid: fp32 [R, J]
+  __nv_bfloat16* out_hl; // kEpiGelu: bf16 [2 Rt, J], hi rows then lo rows
+  int ksteps, row_tiles, col_tiles;
+  int* err;
+};
+cudaError_t launch_pair_gemm(const PairGemmParams& p, const void* act_hl, const void* W, int K, int epi,
+                             cudaStream_t s);
+
 bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows);
 cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s);
 cudaError_t launch_stream_logits(const StreamLogitsParams& p, const LogitMaps* maps, int grid, bool merge,

@@ -123,6 +123,24 @@ def encoder_gemm_bytes(w: si.Workload) -> float:
     return es * per_layer * w.enc_layers * (1 if w.tied else 2)
 
 
+def replica_seed(rank: int) -> int:
+    """Seed of a rank's replica of the workload: ranks run independent replicas (different token
+    streams, weights and hidden states), the path has no exchange step between sequences."""
+    return 1000 + rank
+
+
+def reduce_over_ranks(times_ms, counts, world: int, device):
+    """Whole-job numbers from per-rank ones: every time becomes the MAX over ranks, every count
+    the SUM over ranks.  The only collectives of the benchmark (the data path has none)."""
+    if world <= 1:
+        return list(times_ms), list(counts)
+    tt = torch.tensor(list(times_ms), device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
+    cc = torch.tensor(list(counts), device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(cc, op=torch.distributed.ReduceOp.SUM)
+    return tt.tolist(), cc.tolist()
+
+
 def kernel_source_digest() -> str:
     """Digest of the sources of the streaming kernels; an ncu traffic figure only counts while it
     matches the code that produced it."""
@@ -162,7 +180,7 @@ def run_ours(args, rank: int, world: int):
     if w.steps == 0:
         raise SystemExit("this workload has no decode steps; use tests for the prefill path")
     K, Wm = args.steps, args.warmup
-    seed = 1000 + rank
+    seed = replica_seed(rank)
     tokens = si.make_tokens(w, seed)
     W_E, W_U = si.make_tables(w, seed)
     encE_t = [t.to(dev) for t in si.make_encoder(w, seed * 3 + 1)]
@@ -276,13 +294,7 @@ def run_ours(args, rank: int, world: int):
     bad = int(sum(1 for s in stt.tolist() if s & (zb.ST_BAD_TOKEN | zb.ST_TABLE_FULL | zb.ST_WAIT_TIMEOUT)))
 
     # ---- reduce over ranks: max time, summed tokens ----
-    if world > 1:
-        tt = torch.tensor([dev_ms, e2e_ms], device=dev)
-        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
-        dev_ms, e2e_ms = tt.tolist()
-        cc = torch.tensor([bt_dev, bt_e2e], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(cc)
-        bt_dev, bt_e2e = cc.tolist()
+    (dev_ms, e2e_ms), (bt_dev, bt_e2e) = reduce_over_ranks([dev_ms, e2e_ms], [bt_dev, bt_e2e], world, dev)
 
     pk = peaks()
     # dominant kernel class by measured time
@@ -403,7 +415,7 @@ def run_prompt_scoring(args, rank: int, world: int):
     if args.seqs:
         w = w.scaled(B=args.seqs)
     K, Wm = args.steps, args.warmup
-    seed = 1000 + rank
+    seed = replica_seed(rank)
     tokens = si.make_tokens(w, seed)
     W_E, W_U = si.make_tables(w, seed)
     encE_t = [t.to(dev) for t in si.make_encoder(w, seed * 3 + 1)]
@@ -477,10 +489,7 @@ def run_prompt_scoring(args, rank: int, world: int):
         lse_host.copy_(lse, non_blocking=True)
         torch.cuda.current_stream().synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3
-    if world > 1:
-        tt = torch.tensor([dev_ms, e2e_ms], device=dev)
-        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
-        dev_ms, e2e_ms = tt.tolist()
+    (dev_ms, e2e_ms), _ = reduce_over_ranks([dev_ms, e2e_ms], [0.0], world, dev)
     pk = peaks()
     n_rows = torch.bincount(row_seq.cpu().to(torch.int64), minlength=w.B).numpy()
     flops = 2.0 * w.d * float(sum(int(n_rows[b]) * (w.V + int(n_fin[b])) for b in range(w.B)))

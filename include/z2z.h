@@ -47,7 +47,8 @@ enum {
   Z2Z_ST_CAP_FROZEN = 1,     /* codebook reached cap: matching continues, inserting stopped  */
   Z2Z_ST_BAD_TOKEN = 2,      /* a code named a hypertoken that does not exist; state unchanged */
   Z2Z_ST_TABLE_FULL = 4,     /* hash probe ran through the whole table (cannot happen at load <= 1/2) */
-  Z2Z_ST_WAIT_TIMEOUT = 8    /* a bounded wait inside a kernel gave up                          */
+  Z2Z_ST_WAIT_TIMEOUT = 8,   /* a bounded wait inside a kernel gave up                          */
+  Z2Z_ST_OUTPUT_TRUNCATED = 16 /* z2z_lzw_decode: the base tokens did not fit in T_out_max       */
 };
 
 enum { Z2Z_DTYPE_FP32 = 0, Z2Z_DTYPE_BF16 = 1 };
@@ -155,6 +156,34 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
                         const int32_t* d_forced, int32_t* d_next_codes, int32_t* d_selected,
                         float* d_lse, int32_t* d_new_entry, float* d_Eh_f32, float* d_Uh_f32,
                         z2z_stream stream);
+
+/* Section 2.1 (second property of LZW: the stream decodes without a shipped codebook) and
+ * Section 2.3 steps 11-12: turn each sequence's code stream back into base tokens.
+ *   d_codes [B, Tc_max] int32; d_code_lens [B] valid codes per row, or NULL (= Tc_max);
+ *   d_tokens [B, T_out_max] int32 out; d_token_lens [B] out.
+ * mode Z2Z_DECODE_RESIDENT: every code is looked up in the codebook the session already holds
+ *   (the state at the end of generation); the codebook is not changed.
+ * mode Z2Z_DECODE_REPLAY: the codebook is grown from the codes themselves, one online update
+ *   (as z2z_lzw_step) per code starting from the sequence's current state - after
+ *   z2z_codebook_init this is plain LZW decompression - and the codes are then expanded.  The
+ *   sequence is left as z2z_lzw_step would leave it after the last accepted code.
+ * A code that names no hypertoken sets Z2Z_ST_BAD_TOKEN; that sequence's output ends before it
+ * (in REPLAY mode the state is the one after the last accepted code).  Output beyond T_out_max
+ * is dropped, d_token_lens[b] = T_out_max and Z2Z_ST_OUTPUT_TRUNCATED is set.  All device
+ * pointers; work is enqueued on the stream.                                                    */
+enum { Z2Z_DECODE_RESIDENT = 0, Z2Z_DECODE_REPLAY = 1 };
+int32_t z2z_lzw_decode(z2z_codebook* cb, const int32_t* d_codes, const int32_t* d_code_lens,
+                       int32_t Tc_max, int32_t mode, int32_t* d_tokens, int32_t* d_token_lens,
+                       int32_t T_out_max, z2z_stream stream);
+
+/* Figure 2a / Section 2.3 steps 3-4: input embedding of a mixed stream.  Row r of d_out is
+ * W_E[z] for a base token z < V and the cached hyper-embedding E_h[b][z - V] otherwise, where
+ * b = d_row_seq[r] (or r when d_row_seq is NULL, which needs N <= B).
+ *   d_codes [N] int32; d_WE [V, d]; d_Eh [B, cap, d]; d_out [N, d]; all in the configured dtype.
+ * A code outside [0, V + n_b) sets Z2Z_ST_BAD_TOKEN for that sequence and its row is zero-filled. */
+int32_t z2z_embed_lookup(z2z_codebook* cb, const int32_t* d_codes, int32_t N,
+                         const int32_t* d_row_seq, const void* d_WE, const void* d_Eh,
+                         void* d_out, z2z_stream stream);
 
 /* Waits for the stream, then copies per-sequence status bits and hypertoken counts to the host.
  * Either output may be NULL.                                                                  */

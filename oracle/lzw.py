@@ -16,7 +16,8 @@ Conventions (the paper leaves these open; the readings are listed in the design 
   * at ``cap`` entries the codebook freezes: matching continues, inserting stops.
 
 Pins: tests/test_oracle_lzw.py (worked example after Figure 1, round trip, prefix property,
-bounds, replay equivalence, brute-force longest-match check on tiny vocabularies).
+bounds, replay equivalence, brute-force longest-match check on tiny vocabularies; expand()
+against the self-contained decode and the original tokens).
 """
 from __future__ import annotations
 
@@ -148,6 +149,21 @@ def decode(codes: Sequence[int], V: int, M: int, cap: int):
             raise ValueError(f"code {z} names no hypertoken")
         toks.extend(cb.phrase(int(z)))
     return toks, cb
+
+
+def expand(cb: Codebook, codes: Sequence[int]):
+    """Codes -> base tokens with a codebook that already holds every entry (the state at the end
+    of generation; Section 2.3 steps 11-12).  The codebook is not changed.  Stops before the
+    first code that names no entry; returns (tokens, number of codes expanded)."""
+    toks: List[int] = []
+    done = 0
+    for z in codes:
+        z = int(z)
+        if z < 0 or z >= cb.V + cb.n():
+            break
+        toks.extend(cb.phrase(z))
+        done += 1
+    return toks, done
 
 
 def base_token_count(cb: Codebook, codes: Sequence[int]) -> int:

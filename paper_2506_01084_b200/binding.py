@@ -16,15 +16,17 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libz2z.so")
 
 OK = 0
-ST_CAP_FROZEN, ST_BAD_TOKEN, ST_TABLE_FULL, ST_WAIT_TIMEOUT = 1, 2, 4, 8
+ST_CAP_FROZEN, ST_BAD_TOKEN, ST_TABLE_FULL, ST_WAIT_TIMEOUT, ST_OUTPUT_TRUNCATED = 1, 2, 4, 8, 16
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 SELECT_ARGMAX, SELECT_GUMBEL = 0, 1
 CACHE_EMBED, CACHE_UNEMBED = 0, 1
+DECODE_RESIDENT, DECODE_REPLAY = 0, 1
 
 EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lzw_step",
            "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
            "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error", "z2z_profile",
-           "z2z_profile_read", "z2z_set_tensor_cores", "z2z_logits_static_scratch"]
+           "z2z_profile_read", "z2z_set_tensor_cores", "z2z_logits_static_scratch",
+           "z2z_lzw_decode", "z2z_embed_lookup"]
 
 
 class Config(C.Structure):
@@ -175,6 +177,23 @@ def z2z_decode_step(cb: Codebook, hidden: torch.Tensor, W_E: torch.Tensor, W_U: 
                                  C.c_float(temperature), C.c_uint64(seed), C.c_uint64(step),
                                  _ptr(forced), _ptr(next_codes), _ptr(selected), _ptr(lse),
                                  _ptr(new_entry), _ptr(E_h_f32), _ptr(U_h_f32), _stream()))
+
+
+def z2z_lzw_decode(cb: Codebook, codes: torch.Tensor, code_lens: Optional[torch.Tensor], mode: int,
+                   tokens: torch.Tensor, token_lens: torch.Tensor):
+    """codes [B, Tc_max] int32 -> tokens [B, T_out_max] int32, token_lens [B] (device tensors)."""
+    Tc_max = codes.shape[1] if codes.dim() == 2 else 0
+    T_out = tokens.shape[1] if tokens.dim() == 2 else 0
+    _check(lib().z2z_lzw_decode(cb.handle, _ptr(codes), _ptr(code_lens), C.c_int32(Tc_max),
+                                C.c_int32(mode), _ptr(tokens), _ptr(token_lens), C.c_int32(T_out),
+                                _stream()))
+
+
+def z2z_embed_lookup(cb: Codebook, codes: torch.Tensor, row_seq: Optional[torch.Tensor],
+                     W_E: torch.Tensor, E_h: torch.Tensor, out: torch.Tensor):
+    """codes [N] int32 -> out [N, d]: W_E rows for base tokens, cached E_h rows for hypertokens."""
+    _check(lib().z2z_embed_lookup(cb.handle, _ptr(codes), C.c_int32(codes.numel()), _ptr(row_seq),
+                                  _ptr(W_E), _ptr(E_h), _ptr(out), _stream()))
 
 
 def z2z_status(cb: Codebook):

@@ -225,6 +225,38 @@ int32_t z2z_lzw_step(z2z_codebook* cb, const int32_t* d_new_codes, const uint8_t
   return Z2Z_OK;
 }
 
+int32_t z2z_lzw_decode(z2z_codebook* cb, const int32_t* d_codes, const int32_t* d_code_lens,
+                       int32_t Tc_max, int32_t mode, int32_t* d_tokens, int32_t* d_token_lens,
+                       int32_t T_out_max, z2z_stream stream) {
+  if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
+  if (mode != Z2Z_DECODE_RESIDENT && mode != Z2Z_DECODE_REPLAY) return fail(Z2Z_ERR_INVALID_ARG, "mode must be Z2Z_DECODE_RESIDENT or Z2Z_DECODE_REPLAY");
+  if (Tc_max < 0 || T_out_max < 0) return fail(Z2Z_ERR_INVALID_ARG, "Tc_max / T_out_max < 0");
+  if (!d_token_lens) return fail(Z2Z_ERR_INVALID_ARG, "d_token_lens is NULL");
+  if (Tc_max > 0 && !d_codes) return fail(Z2Z_ERR_INVALID_ARG, "d_codes is NULL");
+  if (T_out_max > 0 && !d_tokens) return fail(Z2Z_ERR_INVALID_ARG, "d_tokens is NULL");
+  z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, reinterpret_cast<cudaStream_t>(stream));
+  int32_t* n_valid = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_new_entry);
+  Z2Z_CUDA(z2z::launch_lzw_decode(cb->view, d_codes, d_code_lens, Tc_max, mode == Z2Z_DECODE_REPLAY,
+                                  n_valid, d_tokens, d_token_lens, T_out_max,
+                                  reinterpret_cast<cudaStream_t>(stream)), "lzw_decode");
+  return Z2Z_OK;
+}
+
+int32_t z2z_embed_lookup(z2z_codebook* cb, const int32_t* d_codes, int32_t N,
+                         const int32_t* d_row_seq, const void* d_WE, const void* d_Eh,
+                         void* d_out, z2z_stream stream) {
+  if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
+  if (N < 0) return fail(Z2Z_ERR_INVALID_ARG, "N < 0");
+  if (N == 0) return Z2Z_OK;
+  if (!d_codes || !d_WE || !d_out) return fail(Z2Z_ERR_INVALID_ARG, "d_codes / d_WE / d_out is NULL");
+  if (!d_Eh && cb->cfg.cap > 0) return fail(Z2Z_ERR_INVALID_ARG, "d_Eh is NULL");
+  if (!d_row_seq && N > cb->cfg.B) return fail(Z2Z_ERR_INVALID_ARG, "d_row_seq is required when N > B");
+  const int eb = cb->cfg.dtype == Z2Z_DTYPE_BF16 ? 2 : 4;
+  Z2Z_CUDA(z2z::launch_embed_lookup(cb->view, d_codes, N, d_row_seq, d_WE, d_Eh, d_out, cb->cfg.d, eb,
+                                    reinterpret_cast<cudaStream_t>(stream)), "embed_lookup");
+  return Z2Z_OK;
+}
+
 int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
                         const z2z_encoder_weights* enc, const int32_t* d_first,
                         const int32_t* d_count, int32_t max_entries, void* d_cache,

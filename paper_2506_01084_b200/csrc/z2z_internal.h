@@ -31,6 +31,12 @@ cudaError_t launch_codebook_clear(const CbView& cb, cudaStream_t s);
 cudaError_t launch_lzw_encode(const CbView& cb, const int32_t* tokens, const int32_t* lens,
                               int T_max, int32_t* codes, int32_t* code_lens,
                               int32_t* entries_after, cudaStream_t s);
+cudaError_t launch_lzw_decode(const CbView& cb, const int32_t* codes, const int32_t* code_lens,
+                              int Tc_max, int replay, int32_t* n_valid, int32_t* tokens,
+                              int32_t* token_lens, int T_out_max, cudaStream_t s);
+cudaError_t launch_embed_lookup(const CbView& cb, const int32_t* codes, int N,
+                                const int32_t* row_seq, const void* WE, const void* Eh, void* out,
+                                int d, int elem_bytes, cudaStream_t s);
 cudaError_t launch_lzw_step(const CbView& cb, const int32_t* new_codes, const uint8_t* active,
                             int32_t* new_entry, cudaStream_t s);
 

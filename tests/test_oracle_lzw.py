@@ -164,3 +164,65 @@ def test_generator_compression_is_in_a_plausible_range():
     x = si.token_stream(w.V, 2048, w.zipf_s, w.copy_p, w.seg_min, w.seg_max, 5)
     codes, _, _ = lzw.encode([int(t) for t in x], w.V, w.M, w.cap)
     assert 0.45 < len(codes) / len(x) < 0.98
+
+
+def test_expand_with_resident_codebook_matches_self_contained_decode():
+    """expand() reads the finished codebook, decode() rebuilds its own: both must give back the
+    original tokens; a code past the end of the codebook stops the expansion before it."""
+    for V, x in _streams():
+        x = [int(t) for t in x]
+        for M, cap in ((3, 100000), (4, 17), (2, 0)):
+            codes, _, cb = lzw.encode(x, V, M, cap)
+            toks, done = lzw.expand(cb, codes)
+            assert toks == x and done == len(codes)
+            back, _ = lzw.decode(codes, V, M, cap)
+            assert back == toks
+            if len(codes) >= 3:
+                broken = list(codes)
+                broken[2] = V + cb.n()                       # names no entry of the finished book
+                t2, d2 = lzw.expand(cb, broken)
+                assert d2 == 2 and t2 == x[:len(t2)]
+                assert len(t2) == lzw.base_token_count(cb, codes[:2])
+
+
+def test_lookup_of_base_tokens_is_a_row_gather_and_flags_missing_hypertokens():
+    from oracle import embedding as oemb
+    rng = np.random.default_rng(5)
+    V, d, B, cap = 11, 8, 2, 4
+    W = rng.standard_normal((V, d))
+    E = rng.standard_normal((B, cap, d))
+    codes = [3, 10, 0, 7]
+    out, bad = oemb.lookup(codes, [0, 1, 1, 0], W, E, [0, 0])
+    assert bad == [] and np.array_equal(out, np.take(W, codes, axis=0))
+    out, bad = oemb.lookup([V + 1, V + 2, V], [0, 0, 1], W, E, [2, 3])
+    assert bad == [0] and np.array_equal(out[0], E[0, 1]) and not out[1].any()
+    assert np.array_equal(out[2], E[1, 0])
+
+
+def test_lookup_of_a_hypertoken_under_the_averaging_encoder_is_the_mean_of_its_base_rows():
+    """Ties the lookup to the codebook: with the parameter-free averaging hyper-encoder a
+    hypertoken's cached row is the mean of W_E over the base tokens it decompresses to, so the
+    lookup of the compressed stream, weighted by phrase lengths, sums to the lookup of the
+    original stream."""
+    from oracle import embedding as oemb
+    from oracle import hyper_encoder as ohe
+    rng = np.random.default_rng(6)
+    V, d, M, cap = 7, 4, 3, 64
+    x = [int(t) for t in rng.integers(0, V, size=200)]
+    codes, _, cb = lzw.encode(x, V, M, cap)
+    W = rng.standard_normal((V, d))
+    pos0 = [np.zeros((M, d))]                               # no layers, zero positions: averaging
+    E = np.zeros((1, cap, d))
+    for k, e in enumerate(cb.entries):
+        E[0, k] = ohe.hyper_embed_one(list(e), W, pos0, 1)
+    rows, bad = oemb.lookup(codes, [0] * len(codes), W, E, [cb.n()])
+    assert bad == []
+    lens = np.array([len(cb.phrase(z)) for z in codes], dtype=np.float64)
+    base_rows, _ = oemb.lookup(x, [0] * len(x), W, E, [cb.n()])
+    np.testing.assert_allclose((rows * lens[:, None]).sum(0), base_rows.sum(0), rtol=0, atol=1e-9)
+    # and one by one: each compressed row is the mean of its own slice of the base rows
+    at = 0
+    for r, z in enumerate(codes):
+        L = int(lens[r])
+        np.testing.assert_allclose(rows[r], base_rows[at:at + L].mean(0), rtol=0, atol=1e-12)
+        at += L

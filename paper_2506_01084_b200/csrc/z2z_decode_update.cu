@@ -79,8 +79,11 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
   const int total = s_warp[31];
   if (tid < cb.B) el.off[tid] = excl;
   if (tid == 0) { el.off[cb.B] = total; el.off[cb.B + 1] = total < el.chunk ? total : el.chunk; }
-  if (flag && excl < el.chunk) { el.seq[excl] = tid; el.idx[excl] = mine - 1; }
-  for (int e = total + tid; e < el.chunk && e < cb.B; e += blockDim.x) { el.seq[e] = -1; el.idx[e] = 0; }
+  if (flag && excl < el.chunk) {
+    el.seq[excl] = tid; el.idx[excl] = mine - 1;
+    el.len[excl] = (int)cb.len[(size_t)tid * cb.cap + (mine - 1)];     // written above by this block
+  }
+  for (int e = total + tid; e < el.chunk && e < cb.B; e += blockDim.x) { el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0; }
   // both caches will hold every entry once the encoder pass that follows has run
   if (tid < cb.B) { const int n = cb.n[tid]; cb.n_emb[tid] = n; cb.n_emb[cb.B + tid] = n; }
 }

@@ -65,7 +65,7 @@ __global__ void k_entry_fill(CbView cb, int which, int mode, const int32_t* __re
   }
   if (e >= el.chunk) return;
   const long long g = (long long)chunk_index * el.chunk + e;
-  if (g >= total) { el.seq[e] = -1; el.idx[e] = 0; return; }
+  if (g >= total) { el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0; return; }
   int lo = 0, hi = cb.B - 1;                     // last b with off[b] <= g
   while (lo < hi) {
     int mid = (lo + hi + 1) >> 1;
@@ -79,8 +79,10 @@ __global__ void k_entry_fill(CbView cb, int which, int mode, const int32_t* __re
     const int n = cb.n[b];
     f = f < 0 ? 0 : (f > n ? n : f);
   }
+  const int k = f + (int)(g - el.off[b]);
   el.seq[e] = b;
-  el.idx[e] = f + (int)(g - el.off[b]);
+  el.idx[e] = k;
+  el.len[e] = (k >= 0 && k < cb.cap) ? (int)cb.len[(size_t)b * cb.cap + k] : 0;
 }
 
 __global__ void k_mark_embedded(CbView cb, int which) {

@@ -67,9 +67,14 @@ __device__ __forceinline__ float4 take4(float* y) {
   return v;
 }
 
+// Base tokens of work-list entry e (0 for an unused slot): one load, so that the kernels below can
+// issue it together with their data loads instead of ahead of them.
 __device__ __forceinline__ int entry_len_tc(const CbView& cb, const EntryList& el, int e) {
-  const int s = el.seq[e];
-  return s < 0 ? 0 : (int)cb.len[(size_t)s * cb.cap + el.idx[e]];
+  (void)cb;
+  return el.len[e];
+}
+__device__ __forceinline__ float4 unpack_bf16x4(uint2 u) {
+  return make_float4(bf_lo(u.x), bf_hi(u.x), bf_lo(u.y), bf_hi(u.y));
 }
 
 __device__ __forceinline__ float block_sum(float v, float* sm) {
@@ -87,8 +92,10 @@ __device__ __forceinline__ float block_sum(float v, float* sm) {
 
 // LayerNorm of a row held in registers (x[v] = 4 columns starting at (tid + v * 256) * 4),
 // written as hi/lo bf16.  eps 1e-5, biased variance, two-pass.
-__device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[kMaxVec4], int nvec, const bf16* g,
-                                                     const bf16* b, bf16* hi, bf16* lo, int d, float* sm) {
+// gw / gb: gamma and beta of the thread's columns, packed 4 bf16 per uint2 and loaded by the caller
+// together with the row, so that no load waits behind the reductions.
+__device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[kMaxVec4], int nvec, const uint2 (&gw)[kMaxVec4],
+                                                     const uint2 (&gb)[kMaxVec4], bf16* hi, bf16* lo, int d, float* sm) {
   float s = 0.f;
 #pragma unroll
   for (int v = 0; v < kMaxVec4; ++v)
@@ -106,7 +113,7 @@ __device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[kMaxVec4]
   for (int v = 0; v < kMaxVec4; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
-      const float4 gg = load_bf16x4(g + idx * 4), bb = load_bf16x4(b + idx * 4);
+      const float4 gg = unpack_bf16x4(gw[v]), bb = unpack_bf16x4(gb[v]);
       float4 y;
       y.x = (x[v].x - mean) * rstd * gg.x + bb.x;
       y.y = (x[v].y - mean) * rstd * gg.y + bb.y;
@@ -142,23 +149,26 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
   const int y = cb.cons[((size_t)el.seq[e] * cb.cap + el.idx[e]) * cb.M + i];
   const bf16* row = reinterpret_cast<const bf16*>(table.p[g]) + (size_t)y * d;
   const bf16* pp = reinterpret_cast<const bf16*>(pos.p[g]) + (size_t)i * d;
+  const uint2* lw = reinterpret_cast<const uint2*>(ln_w.p[g]);
+  const uint2* lb = reinterpret_cast<const uint2*>(ln_b.p[g]);
   float4 xv[kMaxVec4];
+  uint2 gw[kMaxVec4], gb[kMaxVec4];
 #pragma unroll
   for (int v = 0; v < kMaxVec4; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       const float4 a = load_bf16x4(row + idx * 4), b = load_bf16x4(pp + idx * 4);
+      gw[v] = lw[idx]; gb[v] = lb[idx];
       xv[v] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
       *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
     }
   }
-  if (has_ln)
-    layernorm_split_regs(xv, nvec, reinterpret_cast<const bf16*>(ln_w.p[g]),
-                         reinterpret_cast<const bf16*>(ln_b.p[g]), hi, lo, d, sm);
+  if (has_ln) layernorm_split_regs(xv, nvec, gw, gb, hi, lo, d, sm);
 }
 
 // x = X[r] + Y[r] + bias for a valid row (Y consumed and cleared for every row); then
-// LayerNorm -> hi/lo for the next GEMM.  grid (rows, groups).
+// LayerNorm -> hi/lo for the next GEMM.  grid (rows, groups).  All loads (entry length, Y, X, bias,
+// gamma, beta) are issued together; whether the row is valid only decides what is stored.
 __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, EntryList el, float* Y, Ptr2 bias,
                                                                     MPtr2 X, Ptr2 ln_w, Ptr2 ln_b, MPtr2 Ahl,
                                                                     int d, int Rt) {
@@ -166,29 +176,41 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, E
   sm100::pdl_trigger();
   sm100::pdl_wait();
   const int r = blockIdx.x, g = blockIdx.y, e = r / cb.M, i = r - e * cb.M;
-  const bool valid = e < el.off[cb.B + 1] && i < entry_len_tc(cb, el, e);
+  const int L = entry_len_tc(cb, el, e);
   float* y = Y + ((size_t)g * Rt + r) * d;
   float* x = reinterpret_cast<float*>(X.p[g]) + (size_t)r * d;
-  const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
+  const uint2* bs = reinterpret_cast<const uint2*>(bias.p[g]);
+  const uint2* lw = reinterpret_cast<const uint2*>(ln_w.p[g]);
+  const uint2* lb = reinterpret_cast<const uint2*>(ln_b.p[g]);
   const int nvec = d / 4;
-  float4 xv[kMaxVec4];
+  float4 xv[kMaxVec4], yv[kMaxVec4];
+  uint2 bv[kMaxVec4], gw[kMaxVec4], gb[kMaxVec4];
 #pragma unroll
   for (int v = 0; v < kMaxVec4; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
-      const float4 p = take4(y + idx * 4);
+      yv[v] = *reinterpret_cast<const float4*>(y + idx * 4);
+      xv[v] = *reinterpret_cast<const float4*>(x + idx * 4);
+      bv[v] = bs[idx]; gw[v] = lw[idx]; gb[v] = lb[idx];
+    }
+  }
+  const bool valid = i < L;
+#pragma unroll
+  for (int v = 0; v < kMaxVec4; ++v) {
+    const int idx = (int)threadIdx.x + v * kRowThreads;
+    if (idx < nvec) {
+      *reinterpret_cast<float4*>(y + idx * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
       if (valid) {
-        const float4 xo = *reinterpret_cast<const float4*>(x + idx * 4);
-        const float4 b = load_bf16x4(bs + idx * 4);
-        xv[v] = make_float4(xo.x + p.x + b.x, xo.y + p.y + b.y, xo.z + p.z + b.z, xo.w + p.w + b.w);
+        const float4 b = unpack_bf16x4(bv[v]);
+        xv[v] = make_float4(xv[v].x + yv[v].x + b.x, xv[v].y + yv[v].y + b.y, xv[v].z + yv[v].z + b.z,
+                            xv[v].w + yv[v].w + b.w);
         *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
       }
     }
   }
   if (!valid) return;                             // padding rows stay zero in X and in hi/lo
   bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)r * d;
-  layernorm_split_regs(xv, nvec, reinterpret_cast<const bf16*>(ln_w.p[g]),
-                       reinterpret_cast<const bf16*>(ln_b.p[g]), hi, hi + (size_t)Rt * d, d, sm);
+  layernorm_split_regs(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
 // Last layer: x_i = X[r_i] + Y[r_i] + bias for the entry's valid rows, cache row = mean_i x_i.
@@ -199,7 +221,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb,
   sm100::pdl_trigger();
   sm100::pdl_wait();
   const int e = blockIdx.x, g = blockIdx.y;
-  const int L = e < el.off[cb.B + 1] ? entry_len_tc(cb, el, e) : 0;
+  const int L = entry_len_tc(cb, el, e);
   const int nvec = d / 4;
   const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
   float4 acc[kMaxVec4];
@@ -213,10 +235,10 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb,
     for (int v = 0; v < kMaxVec4; ++v) {
       const int idx = (int)threadIdx.x + v * kRowThreads;
       if (idx < nvec) {
+        const float4 xo = *reinterpret_cast<const float4*>(x + idx * 4);      // loaded whether or not the row
+        const float4 b = load_bf16x4(bs + idx * 4);                           // is valid: no load waits for L
         const float4 p = take4(y + idx * 4);
         if (i < L) {
-          const float4 xo = *reinterpret_cast<const float4*>(x + idx * 4);
-          const float4 b = load_bf16x4(bs + idx * 4);
           acc[v].x += xo.x + p.x + b.x; acc[v].y += xo.y + p.y + b.y;
           acc[v].z += xo.z + p.z + b.z; acc[v].w += xo.w + p.w + b.w;
         }
@@ -246,7 +268,6 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_pool(CbView cb, EntryList el
   sm100::pdl_trigger();
   sm100::pdl_wait();
   const int e = blockIdx.x, g = blockIdx.y;
-  if (e >= el.off[cb.B + 1]) return;
   const int L = entry_len_tc(cb, el, e);
   if (L <= 0) return;
   const float* x = reinterpret_cast<const float*>(X.p[g]);
@@ -273,9 +294,10 @@ __global__ void __launch_bounds__(128) k_tc_reduce_gelu(CbView cb, EntryList el,
   const int r = blockIdx.y * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (r >= R) return;
   const int j = t * kNT + lane * 4;
-  const float4 p = take4(Y + ((size_t)g * Rt + r) * J + j);
-  if (r / cb.M >= el.off[cb.B + 1]) return;
+  const int L = entry_len_tc(cb, el, r / cb.M);
   const float4 bs = load_bf16x4(reinterpret_cast<const bf16*>(bias.p[g]) + j);
+  const float4 p = take4(Y + ((size_t)g * Rt + r) * J + j);
+  if (L <= 0) return;                              // unused slot: nothing reads its rows
   float4 v = make_float4(p.x + bs.x, p.y + bs.y, p.z + bs.z, p.w + bs.w);
   v.x = 0.5f * v.x * (1.0f + erff(v.x * 0.70710678118654752440f));
   v.y = 0.5f * v.y * (1.0f + erff(v.y * 0.70710678118654752440f));
@@ -294,21 +316,28 @@ __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias,
   sm100::pdl_trigger();
   sm100::pdl_wait();
   const int e = blockIdx.x, h = blockIdx.y, g = blockIdx.z, i = threadIdx.y, lane = threadIdx.x;
-  const int L = e < el.off[cb.B + 1] ? entry_len_tc(cb, el, e) : 0;
+  const int L = entry_len_tc(cb, el, e);
   const int dh = d / heads;
   const int r = e * cb.M + i;
   {
     const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
     float* y = Y + ((size_t)g * Rt + r) * 3 * d;
-    for (int w = 0; w < 3; ++w)
-      for (int c = lane * 4; c < dh; c += 128) {
+    for (int c = lane * 4; c < dh; c += 128) {
+      float4 p[3], b[3];
+#pragma unroll
+      for (int w = 0; w < 3; ++w) {                // the six loads are independent of one another and of L
         const int col = w * d + h * dh + c;
-        const float4 p = take4(y + col);
-        if (i < L) {
-          const float4 b = load_bf16x4(bs + col);
-          *reinterpret_cast<float4*>(&s_qkv[(i * 3 + w) * dh + c]) = make_float4(p.x + b.x, p.y + b.y, p.z + b.z, p.w + b.w);
-        }
+        p[w] = *reinterpret_cast<const float4*>(y + col);
+        b[w] = load_bf16x4(bs + col);
       }
+#pragma unroll
+      for (int w = 0; w < 3; ++w) {
+        *reinterpret_cast<float4*>(y + w * d + h * dh + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < L)
+          *reinterpret_cast<float4*>(&s_qkv[(i * 3 + w) * dh + c]) =
+              make_float4(p[w].x + b[w].x, p[w].y + b[w].y, p[w].z + b[w].z, p[w].w + b[w].w);
+      }
+    }
   }
   __syncthreads();
   if (i >= L) return;                          // padding rows of the operand stay zero
@@ -352,17 +381,22 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(CbView cb, EntryList
                                                             const bf16* ln_b, bf16* Ahl, int d, int Rt) {
   __shared__ float sm[32];
   const int r = blockIdx.x, e = r / cb.M, i = r - e * cb.M;
-  if (e >= el.off[cb.B + 1] || i >= entry_len_tc(cb, el, e)) return;     // padding rows stay zero in hi/lo
+  if (i >= entry_len_tc(cb, el, e)) return;                              // padding rows stay zero in hi/lo
   const float* x = X + (size_t)r * d;
   const int nvec = d / 4;
   float4 xv[kMaxVec4];
+  uint2 gw[kMaxVec4], gb[kMaxVec4];
 #pragma unroll
   for (int v = 0; v < kMaxVec4; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
-    if (idx < nvec) xv[v] = *reinterpret_cast<const float4*>(x + idx * 4);
+    if (idx < nvec) {
+      xv[v] = *reinterpret_cast<const float4*>(x + idx * 4);
+      gw[v] = reinterpret_cast<const uint2*>(ln_w)[idx];
+      gb[v] = reinterpret_cast<const uint2*>(ln_b)[idx];
+    }
   }
   bf16* hi = Ahl + (size_t)r * d;
-  layernorm_split_regs(xv, nvec, ln_w, ln_b, hi, hi + (size_t)Rt * d, d, sm);
+  layernorm_split_regs(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
 // Bidirectional attention inside one entry from fp32 q, k, v rows [R, 3d] (bias already added);
@@ -370,8 +404,8 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(CbView cb, EntryList
 __global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, bf16* Ohl, int d, int heads, int Rt) {
   extern __shared__ float s_qkv[];
   const int e = blockIdx.x, h = blockIdx.y, i = threadIdx.y, lane = threadIdx.x;
-  if (e >= el.off[cb.B + 1]) return;
   const int L = entry_len_tc(cb, el, e);
+  if (L <= 0) return;
   const int dh = d / heads;
   const int r = e * cb.M + i;
   if (i < L) {

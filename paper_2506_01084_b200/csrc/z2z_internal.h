@@ -45,6 +45,7 @@ cudaError_t launch_lzw_step(const CbView& cb, const int32_t* new_codes, const ui
 struct EntryList {
   int32_t* seq;       // [chunk]  sequence of entry e, -1 = unused slot
   int32_t* idx;       // [chunk]  entry number within the sequence
+  int32_t* len;       // [chunk]  base tokens of the entry, 0 for an unused slot
   int32_t* off;       // [B + 2]  exclusive prefix sum of per-sequence counts, then the total
   int chunk;
 };

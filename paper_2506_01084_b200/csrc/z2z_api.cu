@@ -59,6 +59,7 @@ z2z::EntryList entry_list(z2z_codebook* cb) {
   el.seq = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_seq);
   el.idx = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_idx);
   el.len = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_len);
+  el.tok = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_tok);
   el.off = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_off);
   el.chunk = cb->plan.enc_chunk_entries;
   return el;

@@ -20,6 +20,7 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
   for (int b = tid; b < 1024; b += blockDim.x) s_cnt[b] = 0;
   __syncthreads();
   for (int b = warp; b < cb.B; b += 32) {
+    const LzwPrev state = warp_lzw_load(cb, b);            // independent of the selection: loaded ahead of it
     // ---- merge the partial reductions of hidden row b
     const LogitPartial* lp = a.lpart + (size_t)b * a.part_stride;
     RowRed red; red.init();
@@ -47,7 +48,7 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
       a.next_codes[b] = code;
     }
     // ---- online LZW update with the applied code
-    const int created = warp_lzw_step(cb, b, code);
+    const int created = warp_lzw_step(cb, b, code, state);
     if (lane == 0) {
       if (a.new_entry) a.new_entry[b] = created;
       s_cnt[b] = created >= 0 ? created + 1 : 0;         // 0: none, else entry number + 1
@@ -82,8 +83,12 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
   if (flag && excl < el.chunk) {
     el.seq[excl] = tid; el.idx[excl] = mine - 1;
     el.len[excl] = (int)cb.len[(size_t)tid * cb.cap + (mine - 1)];     // written above by this block
+    for (int i = 0; i < cb.M; ++i) el.tok[(size_t)excl * cb.M + i] = cb.cons[((size_t)tid * cb.cap + (mine - 1)) * cb.M + i];
   }
-  for (int e = total + tid; e < el.chunk && e < cb.B; e += blockDim.x) { el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0; }
+  for (int e = total + tid; e < el.chunk && e < cb.B; e += blockDim.x) {
+    el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0;
+    for (int i = 0; i < cb.M; ++i) el.tok[(size_t)e * cb.M + i] = -1;
+  }
   // both caches will hold every entry once the encoder pass that follows has run
   if (tid < cb.B) { const int n = cb.n[tid]; cb.n_emb[tid] = n; cb.n_emb[cb.B + tid] = n; }
 }

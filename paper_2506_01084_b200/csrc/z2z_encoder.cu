@@ -65,7 +65,11 @@ __global__ void k_entry_fill(CbView cb, int which, int mode, const int32_t* __re
   }
   if (e >= el.chunk) return;
   const long long g = (long long)chunk_index * el.chunk + e;
-  if (g >= total) { el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0; return; }
+  if (g >= total) {
+    el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0;
+    for (int i = 0; i < cb.M; ++i) el.tok[(size_t)e * cb.M + i] = -1;
+    return;
+  }
   int lo = 0, hi = cb.B - 1;                     // last b with off[b] <= g
   while (lo < hi) {
     int mid = (lo + hi + 1) >> 1;
@@ -82,7 +86,10 @@ __global__ void k_entry_fill(CbView cb, int which, int mode, const int32_t* __re
   const int k = f + (int)(g - el.off[b]);
   el.seq[e] = b;
   el.idx[e] = k;
-  el.len[e] = (k >= 0 && k < cb.cap) ? (int)cb.len[(size_t)b * cb.cap + k] : 0;
+  const bool in_book = k >= 0 && k < cb.cap;
+  el.len[e] = in_book ? (int)cb.len[(size_t)b * cb.cap + k] : 0;
+  for (int i = 0; i < cb.M; ++i)                       // constituents are -1 padded behind the entry's length
+    el.tok[(size_t)e * cb.M + i] = in_book ? cb.cons[((size_t)b * cb.cap + k) * cb.M + i] : -1;
 }
 
 __global__ void k_mark_embedded(CbView cb, int which) {

@@ -132,13 +132,13 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
   sm100::pdl_trigger();            // the next kernel may start its prologue and weight prefetch
   sm100::pdl_wait();               // everything read or written below depends on earlier kernels
   const int r = blockIdx.x, g = blockIdx.y, e = r / cb.M, i = r - e * cb.M;
+  const int y = el.tok[r];                        // the row's base token; loaded together with the count
   if (e >= el.off[cb.B + 1]) return;
-  const int L = entry_len_tc(cb, el, e);
   float* x = reinterpret_cast<float*>(X.p[g]) + (size_t)r * d;
   bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)r * d;
   bf16* lo = hi + (size_t)Rt * d;
   const int nvec = d / 4;
-  if (i >= L) {                                   // padding row: zero everywhere
+  if (y < 0) {                                    // padding row: zero everywhere
     for (int idx = threadIdx.x; idx < nvec; idx += kRowThreads) {
       *reinterpret_cast<float4*>(x + idx * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
       *reinterpret_cast<uint2*>(hi + idx * 4) = make_uint2(0u, 0u);
@@ -146,7 +146,6 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
     }
     return;
   }
-  const int y = cb.cons[((size_t)el.seq[e] * cb.cap + el.idx[e]) * cb.M + i];
   const bf16* row = reinterpret_cast<const bf16*>(table.p[g]) + (size_t)y * d;
   const bf16* pp = reinterpret_cast<const bf16*>(pos.p[g]) + (size_t)i * d;
   const uint2* lw = reinterpret_cast<const uint2*>(ln_w.p[g]);

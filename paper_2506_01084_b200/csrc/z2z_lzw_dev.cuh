@@ -48,20 +48,30 @@ __device__ __forceinline__ void warp_write_entry(const CbView& cb, int b, int k,
   if (lane == 0) cb.len[(size_t)b * cb.cap + k] = (uint8_t)(wlen + 1);
 }
 
+// The part of a sequence's state that the update needs and that does not depend on the new code;
+// a caller that still has to compute the code can load it ahead.
+struct LzwPrev { int n, prev, plen; };
+__device__ __forceinline__ LzwPrev warp_lzw_load(const CbView& cb, int b) {
+  LzwPrev s;
+  s.n = cb.n[b];
+  s.prev = cb.prev[b];
+  s.plen = 0;
+  if (s.prev >= 0) s.plen = s.prev < cb.V ? 1 : (int)cb.len[(size_t)b * cb.cap + (s.prev - cb.V)];
+  return s;
+}
 // Online update of sequence b with the newly selected code z (Figure 1; Section 2.3 step 10).
 // Candidate entry = phrase(prev) ++ first(phrase(z)); returns the entry created, or -1.
 // A code that names no existing (or about-to-exist) hypertoken raises BAD_TOKEN and leaves the
 // sequence untouched.
-__device__ __forceinline__ int warp_lzw_step(const CbView& cb, int b, int z) {
+__device__ __forceinline__ int warp_lzw_step(const CbView& cb, int b, int z, const LzwPrev& s) {
   const int lane = threadIdx.x & 31;
   unsigned long long* table = cb.hash + (size_t)b * cb.n_slots;
-  const int n = cb.n[b];
-  const int prev = cb.prev[b];
+  const int n = s.n;
+  const int prev = s.prev;
   int created = -1;
   int st = 0;
   bool ok = !(z < 0 || z > cb.V + n);
-  int plen = 0;
-  if (prev >= 0) plen = prev < cb.V ? 1 : (int)cb.len[(size_t)b * cb.cap + (prev - cb.V)];
+  const int plen = s.plen;
   const bool self_ref = ok && (z == cb.V + n);       // the code this very step would create
   if (self_ref && !(prev >= 0 && plen < cb.M && n < cb.cap)) ok = false;
   if (ok) {
@@ -94,6 +104,10 @@ __device__ __forceinline__ int warp_lzw_step(const CbView& cb, int b, int z) {
     if (st) atomicOr(&cb.status[b], st);
   }
   return ok ? created : -1;
+}
+
+__device__ __forceinline__ int warp_lzw_step(const CbView& cb, int b, int z) {
+  return warp_lzw_step(cb, b, z, warp_lzw_load(cb, b));
 }
 
 }  // namespace z2z

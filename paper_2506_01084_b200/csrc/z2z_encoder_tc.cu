@@ -213,52 +213,46 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, E
 }
 
 // Last layer: x_i = X[r_i] + Y[r_i] + bias for the entry's valid rows, cache row = mean_i x_i.
-// grid (entries, groups).
+// grid (entries, groups, ceil(d / (4 * kRowThreads))): a thread owns 4 columns of the entry and
+// issues the loads of all its rows before it adds.
 __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb, EntryList el, float* Y, Ptr2 bias,
                                                                       MPtr2 X, MPtr2 cache, MPtr2 cache_f32, int d,
                                                                       int Rt) {
   sm100::pdl_trigger();
   sm100::pdl_wait();
   const int e = blockIdx.x, g = blockIdx.y;
+  const int col = ((int)blockIdx.z * kRowThreads + (int)threadIdx.x) * 4;
+  if (col >= d) return;
   const int L = entry_len_tc(cb, el, e);
-  const int nvec = d / 4;
-  const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
-  float4 acc[kMaxVec4];
+  const int seq = el.seq[e], idx = el.idx[e];
+  const float4 b = load_bf16x4(reinterpret_cast<const bf16*>(bias.p[g]) + col);
+  float4 yv[kMaxM], xv[kMaxM];
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int i = 0; i < cb.M; ++i) {
-    const int r = e * cb.M + i;
-    float* y = Y + ((size_t)g * Rt + r) * d;
-    const float* x = reinterpret_cast<const float*>(X.p[g]) + (size_t)r * d;
+  for (int i = 0; i < kMaxM; ++i)
+    if (i < cb.M) {
+      const size_t r = (size_t)e * cb.M + i;
+      yv[i] = *reinterpret_cast<const float4*>(Y + ((size_t)g * Rt + r) * d + col);
+      xv[i] = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X.p[g]) + r * d + col);
+    }
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int v = 0; v < kMaxVec4; ++v) {
-      const int idx = (int)threadIdx.x + v * kRowThreads;
-      if (idx < nvec) {
-        const float4 xo = *reinterpret_cast<const float4*>(x + idx * 4);      // loaded whether or not the row
-        const float4 b = load_bf16x4(bs + idx * 4);                           // is valid: no load waits for L
-        const float4 p = take4(y + idx * 4);
-        if (i < L) {
-          acc[v].x += xo.x + p.x + b.x; acc[v].y += xo.y + p.y + b.y;
-          acc[v].z += xo.z + p.z + b.z; acc[v].w += xo.w + p.w + b.w;
-        }
+  for (int i = 0; i < kMaxM; ++i)
+    if (i < cb.M) {
+      const size_t r = (size_t)e * cb.M + i;
+      *reinterpret_cast<float4*>(Y + ((size_t)g * Rt + r) * d + col) = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < L) {
+        acc.x += xv[i].x + yv[i].x + b.x; acc.y += xv[i].y + yv[i].y + b.y;
+        acc.z += xv[i].z + yv[i].z + b.z; acc.w += xv[i].w + yv[i].w + b.w;
       }
     }
-  }
   if (L <= 0) return;
-  const size_t dst = ((size_t)el.seq[e] * cb.cap + el.idx[e]) * d;
+  const size_t dst = ((size_t)seq * cb.cap + idx) * d + col;
   const float inv = 1.0f / (float)L;
-  bf16* out = reinterpret_cast<bf16*>(cache.p[g]);
+  const float4 m = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+  uint2 o; o.x = pack_bf16(m.x, m.y); o.y = pack_bf16(m.z, m.w);
+  *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(cache.p[g]) + dst) = o;
   float* out32 = reinterpret_cast<float*>(cache_f32.p[g]);
-#pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
-    const int idx = (int)threadIdx.x + v * kRowThreads;
-    if (idx < nvec) {
-      const float4 m = make_float4(acc[v].x * inv, acc[v].y * inv, acc[v].z * inv, acc[v].w * inv);
-      uint2 o; o.x = pack_bf16(m.x, m.y); o.y = pack_bf16(m.z, m.w);
-      *reinterpret_cast<uint2*>(out + dst + idx * 4) = o;
-      if (out32) *reinterpret_cast<float4*>(out32 + dst + idx * 4) = m;
-    }
-  }
+  if (out32) *reinterpret_cast<float4*>(out32 + dst) = m;
 }
 
 // Zero-layer encoder (the parameter-free averaging variant): cache row = mean of X rows.
@@ -283,27 +277,46 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_pool(CbView cb, EntryList el
   }
 }
 
-// H = GELU(Y + bias) -> hi/lo (Y consumed and cleared).  grid (J / 128, ceil(rows / 4), groups),
-// block 128: warp w handles row 4 * blockIdx.y + w, each lane 4 columns of the 128-column tile.
-__global__ void __launch_bounds__(128) k_tc_reduce_gelu(CbView cb, EntryList el, float* Y, Ptr2 bias, MPtr2 Hhl,
-                                                        int J, int R, int Rt) {
+// H = GELU(Y + bias) -> hi/lo (Y consumed and cleared).  The [groups * R, J] results are one flat
+// range of float4; every thread takes kGeluPerThread of them, kGeluThreads apart, and issues all of
+// its loads before it computes.  grid = ceil(groups * R * J / 4 / (kGeluThreads * kGeluPerThread)).
+constexpr int kGeluThreads = 256, kGeluPerThread = 4;
+__global__ void __launch_bounds__(kGeluThreads) k_tc_reduce_gelu(CbView cb, EntryList el, float* Y, Ptr2 bias, MPtr2 Hhl,
+                                                                 int J, int R, int Rt, int ng) {
   sm100::pdl_trigger();
   sm100::pdl_wait();
-  const int t = blockIdx.x, g = blockIdx.z;
-  const int r = blockIdx.y * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (r >= R) return;
-  const int j = t * kNT + lane * 4;
-  const int L = entry_len_tc(cb, el, r / cb.M);
-  const float4 bs = load_bf16x4(reinterpret_cast<const bf16*>(bias.p[g]) + j);
-  const float4 p = take4(Y + ((size_t)g * Rt + r) * J + j);
-  if (L <= 0) return;                              // unused slot: nothing reads its rows
-  float4 v = make_float4(p.x + bs.x, p.y + bs.y, p.z + bs.z, p.w + bs.w);
-  v.x = 0.5f * v.x * (1.0f + erff(v.x * 0.70710678118654752440f));
-  v.y = 0.5f * v.y * (1.0f + erff(v.y * 0.70710678118654752440f));
-  v.z = 0.5f * v.z * (1.0f + erff(v.z * 0.70710678118654752440f));
-  v.w = 0.5f * v.w * (1.0f + erff(v.w * 0.70710678118654752440f));
-  bf16* hi = reinterpret_cast<bf16*>(Hhl.p[g]) + (size_t)r * J + j;
-  split_store4(hi, hi + (size_t)Rt * J, v);
+  const int J4 = J / 4;
+  const long long total = (long long)ng * R * J4;
+  const long long base = (long long)blockIdx.x * (kGeluThreads * kGeluPerThread) + threadIdx.x;
+  float4 q[kGeluPerThread], bs[kGeluPerThread];
+  int row[kGeluPerThread], jj[kGeluPerThread], len[kGeluPerThread];
+#pragma unroll
+  for (int k = 0; k < kGeluPerThread; ++k) {
+    const long long f = base + (long long)k * kGeluThreads;
+    row[k] = -1;
+    if (f < total) {
+      row[k] = (int)(f / J4);
+      jj[k] = (int)(f - (long long)row[k] * J4) * 4;
+      const int g = row[k] / R, r = row[k] - g * R;
+      q[k] = *reinterpret_cast<const float4*>(Y + ((size_t)g * Rt + r) * J + jj[k]);
+      bs[k] = load_bf16x4(reinterpret_cast<const bf16*>(bias.p[g]) + jj[k]);
+      len[k] = entry_len_tc(cb, el, r / cb.M);
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < kGeluPerThread; ++k) {
+    if (row[k] < 0) continue;
+    const int g = row[k] / R, r = row[k] - g * R;
+    *reinterpret_cast<float4*>(Y + ((size_t)g * Rt + r) * J + jj[k]) = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (len[k] <= 0) continue;                     // unused slot: nothing reads its rows
+    float4 v = make_float4(q[k].x + bs[k].x, q[k].y + bs[k].y, q[k].z + bs[k].z, q[k].w + bs[k].w);
+    v.x = 0.5f * v.x * (1.0f + erff(v.x * 0.70710678118654752440f));
+    v.y = 0.5f * v.y * (1.0f + erff(v.y * 0.70710678118654752440f));
+    v.z = 0.5f * v.z * (1.0f + erff(v.z * 0.70710678118654752440f));
+    v.w = 0.5f * v.w * (1.0f + erff(v.w * 0.70710678118654752440f));
+    bf16* hi = reinterpret_cast<bf16*>(Hhl.p[g]) + (size_t)r * J + jj[k];
+    split_store4(hi, hi + (size_t)Rt * J, v);
+  }
 }
 
 // q, k, v = Y + bias for one head of one entry (consumed, cleared, staged in shared memory), then
@@ -596,15 +609,17 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
     if ((e = gemm(Ahl, d, o + 8, dff)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      launch_pdl(k_tc_reduce_gelu, dim3(dff / kNT, (R + 3) / 4, ng), dim3(128), 0, s, cb, el, Y, W(o + 9), Hhl, dff,
-                 R, Rt);
+      const long long f4 = (long long)ng * R * (dff / 4);
+      const int per_cta = kGeluThreads * kGeluPerThread;
+      launch_pdl(k_tc_reduce_gelu, dim3((unsigned)((f4 + per_cta - 1) / per_cta)), dim3(kGeluThreads), 0, s, cb, el, Y,
+                 W(o + 9), Hhl, dff, R, Rt, ng);
     }
     if ((e = gemm(Hhl, dff, o + 10, d)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
       if (last)
-        launch_pdl(k_tc_reduce_resid_pool, dim3(E, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 11), X, cache, c32,
-                   d, Rt);
+        launch_pdl(k_tc_reduce_resid_pool, dim3(E, ng, (d / 4 + kRowThreads - 1) / kRowThreads), dim3(kRowThreads), 0,
+                   s, cb, el, Y, W(o + 11), X, cache, c32, d, Rt);
       else
         launch_pdl(k_tc_reduce_resid_ln, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 11), X, W(o + 12),
                    W(o + 13), Ahl, d, Rt);

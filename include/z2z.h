@@ -148,14 +148,17 @@ int32_t z2z_dynamic_logits(z2z_codebook* cb, const void* d_hidden, int32_t N,
  *            the selection is still computed and returned in d_selected).
  *   d_next_codes [B] out: the code that was applied; d_selected [B] out or NULL: argmax/sample;
  *   d_lse [B] out; d_new_entry [B] out or NULL.
- *   d_Eh_f32 / d_Uh_f32: optional fp32 copies of the new rows, as in z2z_hyper_embed.          */
+ *   d_Eh_f32 / d_Uh_f32: optional fp32 copies of the new rows, as in z2z_hyper_embed.
+ *   d_next_embed [B, d] out or NULL: input embedding of the applied codes for the model's next
+ *            step (Figure 2a): W_E row of a base token, else the sequence's cached hyper-embedding,
+ *            including the row this very step created; as z2z_embed_lookup on d_next_codes.     */
 int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE,
                         const void* d_WU, const z2z_encoder_weights* enc_E,
                         const z2z_encoder_weights* enc_U, void* d_Eh, void* d_Uh,
                         int32_t select, float temperature, uint64_t seed, uint64_t step,
                         const int32_t* d_forced, int32_t* d_next_codes, int32_t* d_selected,
                         float* d_lse, int32_t* d_new_entry, float* d_Eh_f32, float* d_Uh_f32,
-                        z2z_stream stream);
+                        void* d_next_embed, z2z_stream stream);
 
 /* Section 2.1 (second property of LZW: the stream decodes without a shipped codebook) and
  * Section 2.3 steps 11-12: turn each sequence's code stream back into base tokens.

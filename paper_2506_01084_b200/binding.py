@@ -171,12 +171,13 @@ def z2z_decode_step(cb: Codebook, hidden: torch.Tensor, W_E: torch.Tensor, W_U: 
                     forced: Optional[torch.Tensor], next_codes: torch.Tensor,
                     selected: Optional[torch.Tensor], lse: Optional[torch.Tensor],
                     new_entry: Optional[torch.Tensor] = None,
-                    E_h_f32: Optional[torch.Tensor] = None, U_h_f32: Optional[torch.Tensor] = None):
+                    E_h_f32: Optional[torch.Tensor] = None, U_h_f32: Optional[torch.Tensor] = None,
+                    next_embed: Optional[torch.Tensor] = None):
     _check(lib().z2z_decode_step(cb.handle, _ptr(hidden), _ptr(W_E), _ptr(W_U), C.byref(enc_E),
                                  C.byref(enc_U), _ptr(E_h), _ptr(U_h), C.c_int32(select),
                                  C.c_float(temperature), C.c_uint64(seed), C.c_uint64(step),
                                  _ptr(forced), _ptr(next_codes), _ptr(selected), _ptr(lse),
-                                 _ptr(new_entry), _ptr(E_h_f32), _ptr(U_h_f32), _stream()))
+                                 _ptr(new_entry), _ptr(E_h_f32), _ptr(U_h_f32), _ptr(next_embed), _stream()))
 
 
 def z2z_lzw_decode(cb: Codebook, codes: torch.Tensor, code_lens: Optional[torch.Tensor], mode: int,

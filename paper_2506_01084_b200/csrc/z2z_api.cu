@@ -332,7 +332,7 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
                         int32_t select, float temperature, uint64_t seed, uint64_t step,
                         const int32_t* d_forced, int32_t* d_next_codes, int32_t* d_selected,
                         float* d_lse, int32_t* d_new_entry, float* d_Eh_f32, float* d_Uh_f32,
-                        z2z_stream stream) {
+                        void* d_next_embed, z2z_stream stream) {
   if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
   if (!d_hidden || !d_WE || !d_WU || !d_Eh || !d_Uh || !d_next_codes) return fail(Z2Z_ERR_INVALID_ARG, "a required pointer is NULL");
   if (select != Z2Z_SELECT_ARGMAX && select != Z2Z_SELECT_GUMBEL) return fail(Z2Z_ERR_INVALID_ARG, "unknown select mode");
@@ -406,6 +406,11 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
         Z2Z_CUDA(z2z::run_encoder_pass(cb->view, g[1], el, false, &cb->prof, s), "decode_step");
       }
     }
+  }
+  if (d_next_embed) {                              // after the cache update: the new row may be the one looked up
+    z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
+    Z2Z_CUDA(z2z::launch_embed_lookup(cb->view, d_next_codes, B, nullptr, d_WE, d_Eh, d_next_embed, cb->cfg.d,
+                                      cb->cfg.dtype == Z2Z_DTYPE_BF16 ? 2 : 4, s), "decode_step (next embedding)");
   }
   return Z2Z_OK;
 }

@@ -42,4 +42,6 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.z2z_workspace_bytes(ctypes.byref(ok), ctypes.byref(out)) == 0 and out.value > 0
     # a NULL handle is rejected, not dereferenced
     assert lib.z2z_lzw_step(None, None, None, None, None) == -1
+    assert lib.z2z_lzw_decode(None, None, None, 0, 0, None, None, 0, None) == -1
+    assert lib.z2z_embed_lookup(None, None, 0, None, None, None, None, None) == -1
     assert lib.z2z_codebook_destroy(None) == 0

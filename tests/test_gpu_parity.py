@@ -8,7 +8,7 @@ import numpy as np
 import pytest
 import torch
 
-from oracle import lzw as olzw, logits as olg
+from oracle import embedding as oemb, lzw as olzw, logits as olg
 from paper_2506_01084_b200 import binding as zb
 from paper_2506_01084_b200 import synth_inputs as si
 from tests._harness import GAP, TOL, Pair, f64
@@ -323,6 +323,7 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
     sel = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
     lse = torch.zeros(w.B, dtype=torch.float32, device=p.dev)
     new = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    nxt_emb = torch.zeros(w.B, w.d, dtype=w.torch_dtype, device=p.dev)
     followed = 0
     worst_lse = 0.0
     rng = np.random.default_rng(seed)
@@ -339,8 +340,9 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
                            select, 0.9, 4242, t,
                            None if forced is None else torch.tensor(forced, dtype=torch.int32,
                                                                     device=p.dev),
-                           nxt, sel, lse, new, p.E_f32, p.U_f32)
+                           nxt, sel, lse, new, p.E_f32, p.U_f32, nxt_emb)
         g_sel, g_nxt, g_lse, g_new = (x.cpu().numpy() for x in (sel, nxt, lse, new))
+        g_emb = f64(nxt_emb)
         sc = p.oracle.score(H[t], select, 0.9, 4242, t)
         apply = []
         for b in range(w.B):
@@ -357,6 +359,19 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
             apply.append(want_next)
         onew = p.oracle.advance(apply)
         assert g_new.tolist() == onew, (t, g_new.tolist(), onew)
+        # input embedding of the applied codes for the next model step (Figure 2a): a base token's
+        # row is a copy; a hypertoken's row is the cached hyper-embedding (the row created by this
+        # very step included), held to the tolerance of the hyper-encoder
+        E_pad = np.zeros((w.B, max(w.cap, 1), w.d))
+        for b in range(w.B):
+            E_pad[b, :p.oracle.E_h[b].shape[0]] = p.oracle.E_h[b]
+        want_emb, bad = oemb.lookup(apply, None, f64(p.W_E), E_pad, [bk.n() for bk in p.oracle.books])
+        assert bad == []
+        for b in range(w.B):
+            if apply[b] < w.V:
+                assert np.array_equal(g_emb[b], want_emb[b])
+            else:
+                assert np.abs(g_emb[b] - want_emb[b]).max() <= TOL, (t, b, apply[b])
         for b in range(w.B):
             if onew[b] >= 0:
                 p.check_cache_rows(b, onew[b], onew[b] + 1)

@@ -147,7 +147,9 @@ int32_t z2z_dynamic_logits(z2z_codebook* cb, const void* d_hidden, int32_t N,
  *   d_forced [B] or NULL: codes to feed the update instead of the selection (teacher forcing;
  *            the selection is still computed and returned in d_selected).
  *   d_next_codes [B] out: the code that was applied; d_selected [B] out or NULL: argmax/sample;
- *   d_lse [B] out; d_new_entry [B] out or NULL.
+ *   d_lse [B] out; d_new_entry [B] out or NULL.  These small result arrays may also be pinned host
+ *            memory that is mapped into the device's address space: the kernels then store the
+ *            results straight into host memory and no separate copy is needed.
  *   d_Eh_f32 / d_Uh_f32: optional fp32 copies of the new rows, as in z2z_hyper_embed.
  *   d_next_embed [B, d] out or NULL: input embedding of the applied codes for the model's next
  *            step (Figure 2a): W_E row of a base token, else the sequence's cached hyper-embedding,

@@ -310,7 +310,7 @@ def test_dynamic_logits_no_hypertokens_is_plain_lm_head():
 # ------------------------------------------------------------------------------------------------
 # Whole decode step, following the GPU's selections inside the oracle's top-2 gap
 # ------------------------------------------------------------------------------------------------
-def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=True):
+def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=True, host_results=False):
     p = Pair(w, seed=seed, tensor_cores=tensor_cores)
     _prefill_both(p)
     for b in range(w.B):
@@ -323,6 +323,8 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
     sel = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
     lse = torch.zeros(w.B, dtype=torch.float32, device=p.dev)
     new = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    if host_results:          # pinned host memory, mapped into the device's address space
+        nxt, sel, lse, new = (x.cpu().pin_memory() for x in (nxt, sel, lse, new))
     nxt_emb = torch.zeros(w.B, w.d, dtype=w.torch_dtype, device=p.dev)
     followed = 0
     worst_lse = 0.0
@@ -341,7 +343,9 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
                            None if forced is None else torch.tensor(forced, dtype=torch.int32,
                                                                     device=p.dev),
                            nxt, sel, lse, new, p.E_f32, p.U_f32, nxt_emb)
-        g_sel, g_nxt, g_lse, g_new = (x.cpu().numpy() for x in (sel, nxt, lse, new))
+        if host_results:
+            torch.cuda.synchronize()
+        g_sel, g_nxt, g_lse, g_new = (x.cpu().numpy().copy() for x in (sel, nxt, lse, new))
         g_emb = f64(nxt_emb)
         sc = p.oracle.score(H[t], select, 0.9, 4242, t)
         apply = []
@@ -385,6 +389,11 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
 def test_decode_step_tiny_config_argmax():
     followed, worst = _decode_follow(si.WORKLOADS["tiny"], 21, zb.SELECT_ARGMAX)
     print(f"tiny: followed {followed} near-ties, worst |LSE error| {worst:.2e}")
+
+
+def test_decode_step_results_written_to_pinned_host_memory():
+    for w, sel in ((si.WORKLOADS["tiny"], zb.SELECT_ARGMAX), (SMALL_BF16, zb.SELECT_GUMBEL)):
+        _decode_follow(w, 27, sel, steps=6, forced_every=3, host_results=True)
 
 
 def test_decode_step_tiny_config_sampling_and_forcing():

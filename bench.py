@@ -265,16 +265,27 @@ def run_ours(args, rank: int, world: int):
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record()
     nx_e2e = np.zeros((K, w.B), dtype=np.int32)
-    out_np = out_host.numpy()
+    out_np, lse_np = out_host.numpy(), lse_host.numpy()
+    out_np[:] = -1
+    lse_np[:] = np.nan
     for i, t in enumerate(range(Wm + 2 * K, Wm + 3 * K)):
-        hid_dev.copy_(hidden_host[t], non_blocking=True)
+        zb.z2z_upload_rows(hidden_host[t], hid_dev)    # host -> device by a kernel the logits kernel overlaps
         # the applied codes and the LSE go straight into pinned host memory: the result pointers of
         # the call may be host memory that is mapped into the device's address space, so the
         # device -> host transfer of the result is the kernel's own stores
         zb.z2z_decode_step(cb, hid_dev, g_WE, g_WU, encE, encU, E_h, U_h, zb.SELECT_ARGMAX, 1.0, 0, t,
                            None, out_host, None, lse_host)
-        torch.cuda.current_stream().synchronize()      # the caller needs the token to go on
+        # the caller needs the token to go on: it watches the result land in host memory instead of
+        # waiting for the whole stream (the cache update of this step is still running then, and
+        # the next step's launches queue up behind it)
+        t_wait = time.perf_counter()
+        while (out_np < 0).any() or np.isnan(lse_np).any():
+            if time.perf_counter() - t_wait > 5.0:
+                raise RuntimeError("decode step result did not arrive in host memory")
         nx_e2e[i] = out_np
+        out_np[:] = -1
+        lse_np[:] = np.nan
+    torch.cuda.current_stream().synchronize()
     e3.record()
     barrier()
     e2e_ms = max(e2.elapsed_time(e3), (time.perf_counter() - t0) * 1e3)

@@ -190,6 +190,14 @@ int32_t z2z_embed_lookup(z2z_codebook* cb, const int32_t* d_codes, int32_t N,
                          const int32_t* d_row_seq, const void* d_WE, const void* d_Eh,
                          void* d_out, z2z_stream stream);
 
+/* Host -> device transfer of a small per-step input (the hidden rows of a decode step) by a kernel
+ * instead of a copy-engine transfer (no counterpart in the paper; end-to-end latency aid).  The
+ * kernel that follows on the stream may start its independent part - z2z_decode_step's logits
+ * kernel streams W_U before it needs the hidden rows - while the transfer runs.
+ *   h_mapped_src: pinned host memory that is mapped into the device's address space;
+ *   d_dst: device memory; bytes: multiple of 16, at most 256 MiB; both pointers 16-byte aligned. */
+int32_t z2z_upload_rows(const void* h_mapped_src, void* d_dst, size_t bytes, z2z_stream stream);
+
 /* Waits for the stream, then copies per-sequence status bits and hypertoken counts to the host.
  * Either output may be NULL.                                                                  */
 int32_t z2z_status(z2z_codebook* cb, int32_t* h_status, int32_t* h_n, z2z_stream stream);

@@ -26,7 +26,7 @@ EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lz
            "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
            "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error", "z2z_profile",
            "z2z_profile_read", "z2z_set_tensor_cores", "z2z_logits_static_scratch",
-           "z2z_lzw_decode", "z2z_embed_lookup"]
+           "z2z_lzw_decode", "z2z_embed_lookup", "z2z_upload_rows"]
 
 
 class Config(C.Structure):
@@ -195,6 +195,13 @@ def z2z_embed_lookup(cb: Codebook, codes: torch.Tensor, row_seq: Optional[torch.
     """codes [N] int32 -> out [N, d]: W_E rows for base tokens, cached E_h rows for hypertokens."""
     _check(lib().z2z_embed_lookup(cb.handle, _ptr(codes), C.c_int32(codes.numel()), _ptr(row_seq),
                                   _ptr(W_E), _ptr(E_h), _ptr(out), _stream()))
+
+
+def z2z_upload_rows(src_pinned: torch.Tensor, dst: torch.Tensor):
+    """Pinned host tensor -> device tensor of the same size, by a kernel (see z2z.h)."""
+    nbytes = src_pinned.numel() * src_pinned.element_size()
+    assert src_pinned.is_pinned() and nbytes == dst.numel() * dst.element_size()
+    _check(lib().z2z_upload_rows(_ptr(src_pinned), _ptr(dst), C.c_size_t(nbytes), _stream()))
 
 
 def z2z_status(cb: Codebook):

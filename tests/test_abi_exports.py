@@ -44,4 +44,6 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.z2z_lzw_step(None, None, None, None, None) == -1
     assert lib.z2z_lzw_decode(None, None, None, 0, 0, None, None, 0, None) == -1
     assert lib.z2z_embed_lookup(None, None, 0, None, None, None, None, None) == -1
+    assert lib.z2z_upload_rows(None, None, ctypes.c_size_t(16), None) == -1
+    assert lib.z2z_upload_rows(None, None, ctypes.c_size_t(0), None) == 0
     assert lib.z2z_codebook_destroy(None) == 0

@@ -202,3 +202,15 @@ def test_embed_lookup_matches_oracle(dtype, d):
     zb.z2z_embed_lookup(cb, torch.tensor(z, dtype=torch.int32, device=DEV), None, W_E.to(DEV), E_h.to(DEV), out2)
     want2, _ = oemb.lookup(z, None, W_E.double().numpy(), E_h.double().numpy(), n.tolist())
     assert np.array_equal(out2.cpu().double().numpy(), want2)
+
+
+def test_upload_rows_copies_pinned_host_memory():
+    src = si.normal_tensor((8, 3072), 1.0, 41, torch.bfloat16).pin_memory()
+    dst = torch.zeros(8, 3072, dtype=torch.bfloat16, device=DEV)
+    zb.z2z_upload_rows(src, dst)
+    assert torch.equal(dst.cpu(), src)
+    src2 = si.normal_tensor((3, 8), 1.0, 42, torch.float32).pin_memory()     # 96 bytes: a ragged tail of the last block
+    dst2 = torch.zeros(3, 8, dtype=torch.float32, device=DEV)
+    zb.z2z_upload_rows(src2, dst2)
+    zb.z2z_upload_rows(src2[1:2], dst2[0:1])                                  # a view: row 1 over row 0
+    assert torch.equal(dst2.cpu()[1:], src2[1:]) and torch.equal(dst2.cpu()[0], src2[1])

@@ -541,7 +541,7 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   if (ng == 1 && R >= kPairPassMinRows) return run_encoder_pass_pair(cb, a0, el, E, prof, s);
   const int Rt = (R + 7) / 8 * 8;                      // rows per hi (or lo) block
   const int row_tiles = (Rt + 127) / 128;
-  const bool stacked = 2 * Rt <= 128;                  // hi and lo rows share one 128-row MMA
+  const bool one_box = row_tiles == 1;                 // hi and lo rows (2 Rt <= 256) are one operand box
   const int n_sm = sm_count();
   float* Y = a0.part;                                  // GEMM results, all zero between GEMMs
   const size_t wide = (size_t)(3 * d > dff ? 3 * d : dff);
@@ -560,13 +560,17 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   auto gemm = [&](const MPtr2& act, int K, int widx, int J) -> cudaError_t {
     StreamGemmParams p{};
     p.row_tiles = row_tiles; p.groups = ng; p.tiles_per_group = J / kNT;
-    p.ksb = stacked ? 2 : 1;                       // few rows: larger boxes, fewer TMA operations per byte
-    p.ksteps = (K / 64 + p.ksb - 1) / p.ksb;
-    p.a_parts = stacked ? 1 : 2;
-    p.a_box_rows = stacked ? 2 * Rt : (Rt < 128 ? Rt : 128);
+    // hi rows [0, Rt) and lo rows [Rt, 2 Rt) of the operand are one contiguous box while they fit
+    // the MMA's N (256); beyond that a row tile takes its 128 hi rows and its 128 lo rows as two boxes
+    p.a_parts = one_box ? 1 : 2;
+    p.a_box_rows = one_box ? 2 * Rt : 128;
     p.a_part_row = Rt;
-    p.out_rows = stacked ? 2 * Rt : (Rt < 128 ? Rt : 128);
-    p.out = Y; p.J = J; p.Rt = Rt; p.valid_rows = R; p.stacked = stacked ? 1 : 0;
+    p.n_act = p.a_parts * p.a_box_rows;
+    p.lo_col = one_box ? Rt : 128;
+    // two k-blocks per stage (fewer TMA operations per byte) while at least four stages still fit
+    p.ksb = (one_box && K % 128 == 0 && stream_gemm_stages(2, p.n_act) >= 4) ? 2 : 1;
+    p.ksteps = (K / 64 + p.ksb - 1) / p.ksb;
+    p.out = Y; p.J = J; p.Rt = Rt; p.valid_rows = R;
     p.err = a0.err;
     const long long tiles = (long long)row_tiles * ng * p.tiles_per_group;
     const int G = tiles * p.ksteps < n_sm ? (int)(tiles * p.ksteps) : n_sm;     // every CTA owns >= 1 unit

@@ -24,6 +24,10 @@ __device__ __forceinline__ void red_add_f32x4(float* out, float a, float b, floa
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
+__device__ __forceinline__ void red_add_f32(float* out, float a) {
+  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(out), "f"(a) : "memory");
+}
+
 // ---- mbarrier ---------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

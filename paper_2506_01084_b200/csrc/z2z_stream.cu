@@ -51,36 +51,6 @@ struct Job {
   int wbox_classes;      // to wbox_min << (wbox_classes - 1); tensor map = wmap * classes + class
 };
 
-// ---- GEMM schedule ------------------------------------------------------------------------------
-struct GemmSched {
-  const StreamGemmParams& p;
-  long long u, u1, c;
-  __device__ GemmSched(const StreamGemmParams& pp, int NT) : p(pp) {
-    const long long U = (long long)p.row_tiles * p.groups * p.tiles_per_group * p.ksteps, G = gridDim.x;
-    c = blockIdx.x;
-    u = c * U / G;
-    u1 = (c + 1) * U / G;
-    (void)NT;
-  }
-  __device__ bool next(Job& j, int NT) {
-    if (u >= u1) return false;
-    const long long tile = u / p.ksteps;
-    j.kb0 = (int)(u - tile * p.ksteps);
-    long long left = u1 - u;
-    j.kb1 = (int)((p.ksteps - j.kb0) < left ? p.ksteps : j.kb0 + left);
-    const int per_rt = p.groups * p.tiles_per_group;
-    j.rt = (int)(tile / per_rt);
-    const int rem = (int)(tile - (long long)j.rt * per_rt);
-    const int g = rem / p.tiles_per_group;
-    j.amap = g; j.wmap = g; j.arow = j.rt * 128;
-    j.wrow = (rem - g * p.tiles_per_group) * NT;
-    j.slot = tile + c;
-    j.nrows = NT; j.wbox_min = NT; j.wbox_classes = 1;
-    u += j.kb1 - j.kb0;
-    return true;
-  }
-};
-
 // ---- logits schedule ----------------------------------------------------------------------------
 // Columns are dealt in granules of kLogitGran rows: first the granules of W_U, then those of the
 // visible rows of each sequence's U_h.  Every CTA owns the same number of granules (+-1); a job
@@ -238,23 +208,57 @@ __device__ __forceinline__ void setup_barriers(Ctrl* ctrl) {
 }
 
 // =================================================================================================
-// GEMM kernel: partial tiles out
+// GEMM kernel: weights as the M operand, activation rows (hi | lo) as the N operand
 // =================================================================================================
-template <int NT, int KSB, int STAGES>
+struct GemmJob { int g, arow, wrow, kb0, kb1; };
+struct GemmWalk {
+  const StreamGemmParams& p;
+  long long u, u1;
+  __device__ GemmWalk(const StreamGemmParams& pp) : p(pp) {
+    const long long U = (long long)p.row_tiles * p.groups * p.tiles_per_group * p.ksteps, G = gridDim.x, c = blockIdx.x;
+    u = c * U / G;
+    u1 = (c + 1) * U / G;
+  }
+  __device__ bool next(GemmJob& j) {
+    if (u >= u1) return false;
+    const long long tile = u / p.ksteps;
+    j.kb0 = (int)(u - tile * p.ksteps);
+    const long long left = u1 - u;
+    j.kb1 = (int)((p.ksteps - j.kb0) < left ? p.ksteps : j.kb0 + left);
+    const int per_rt = p.groups * p.tiles_per_group;
+    const int rt = (int)(tile / per_rt);
+    const int rem = (int)(tile - (long long)rt * per_rt);
+    j.g = rem / p.tiles_per_group;
+    j.arow = rt * 128;
+    j.wrow = (rem - j.g * p.tiles_per_group) * kGemmNT;
+    u += j.kb1 - j.kb0;
+    return true;
+  }
+};
+
+__host__ __device__ constexpr uint32_t gemm_tmem_cols(int n_act) {
+  return 2 * n_act <= 32 ? 32u : (2 * n_act <= 64 ? 64u : (2 * n_act <= 128 ? 128u : (2 * n_act <= 256 ? 256u : 512u)));
+}
+
+template <int KSB, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0,
               const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmW0,
               const __grid_constant__ CUtensorMap tmW1) {
+  constexpr int NT = kGemmNT;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm);
   const uint32_t stage_base = smem_u32(sm + 1024);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t a_part_bytes = (uint32_t)KSB * p.a_box_rows * 128;
+  const uint32_t a_bytes = p.a_parts * a_part_bytes;
+  const uint32_t stage_bytes = a_bytes + (uint32_t)KSB * NT * 128;
   pdl_trigger();                                   // the next kernel may get resident behind this one
   setup_barriers<STAGES>(ctrl);
   if (warp == 0 && lane == 0) { prefetch_tmap(&tmA0); prefetch_tmap(&tmW0); if (p.groups > 1) { prefetch_tmap(&tmA1); prefetch_tmap(&tmW1); } }
   __syncthreads();
-  if (warp == 2) { tmem_alloc(smem_u32(&ctrl->tmem_base), tmem_cols(NT)); tmem_relinquish(); }
+  if (warp == 2) { tmem_alloc(smem_u32(&ctrl->tmem_base), gemm_tmem_cols(p.n_act)); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -262,45 +266,109 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
 
   if (warp == 0) {
     if (lane == 0) {
+      // ---- TMA producer.  The weight tiles depend on no earlier kernel, the activation tiles do:
+      // during the first pass over the ring only the weight boxes are issued and the activation
+      // boxes are noted; once the ring is full (or the work ends) the producer waits for the
+      // preceding kernel and issues them.  With an ordinary launch the wait returns at once.
       const CUtensorMap* amaps[2] = {&tmA0, &tmA1};
       const CUtensorMap* wmaps[2] = {&tmW0, &tmW1};
-      GemmSched sched(p, NT);
-      producer_role<NT, KSB, STAGES>(sched, ctrl, stage_base, p.a_parts, p.a_box_rows, p.a_part_row, amaps, wmaps);
+      const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
+      struct Deferred { uint32_t dst, bar; int map, row, kb; };
+      Deferred def[kMaxStages * 2];
+      int n_def = 0, issued = 0;
+      bool deps = false, ok = true;
+      auto need_deps = [&]() {
+        if (deps) return;
+        pdl_wait();
+        for (int i = 0; i < n_def; ++i) tma_load_3d(def[i].dst, amaps[def[i].map], 0, def[i].row, def[i].kb, def[i].bar, pol_a);
+        deps = true;
+      };
+      int stage = 0; uint32_t phase = 0;
+      GemmWalk walk(p);
+      GemmJob j;
+      while (ok && walk.next(j)) {
+        for (int ks = j.kb0; ks < j.kb1; ++ks) {
+          if (issued == STAGES) need_deps();
+          if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) { ok = false; break; }
+          const uint32_t full = smem_u32(&ctrl->full[stage]);
+          mbar_expect_tx(full, stage_bytes);
+          const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
+          tma_load_3d(sb + a_bytes, wmaps[j.g], 0, j.wrow, ks * KSB, full, pol_w);
+          for (int part = 0; part < p.a_parts; ++part) {
+            const uint32_t dst = sb + part * a_part_bytes;
+            const int row = j.arow + part * p.a_part_row;
+            if (deps) tma_load_3d(dst, amaps[j.g], 0, row, ks * KSB, full, pol_a);
+            else { def[n_def].dst = dst; def[n_def].bar = full; def[n_def].map = j.g; def[n_def].row = row; def[n_def].kb = ks * KSB; ++n_def; }
+          }
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      need_deps();
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      GemmSched sched(p, NT);
-      mma_role<NT, KSB, STAGES>(sched, ctrl, stage_base, p.a_parts, p.a_box_rows, tmem_base);
+      // ---- MMA issue: D[128 weight rows][n_act] += W tile (M operand) x activations (N operand)
+      const uint32_t idesc = idesc_bf16_f32(128, p.n_act);
+      int stage = 0; uint32_t phase = 0, job_i = 0;
+      bool ok = true;
+      GemmWalk walk(p);
+      GemmJob j;
+      while (ok && walk.next(j)) {
+        const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&ctrl->acc_empty[buf]), aph ^ 1u, &ctrl->abort)) break;
+        tc_fence_after();
+        const uint32_t d = tmem_base + buf * (uint32_t)p.n_act;
+        uint32_t acc = 0;
+        for (int ks = j.kb0; ks < j.kb1; ++ks) {
+          if (!mbar_wait(smem_u32(&ctrl->full[stage]), phase, &ctrl->abort)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
+#pragma unroll
+          for (int i = 0; i < KSB; ++i) {
+            // with two boxes per stage KSB is 1 and the boxes are adjacent: n_act contiguous rows
+            const uint32_t ab = sb + (uint32_t)i * p.a_box_rows * 128;
+            const uint32_t wb = sb + a_bytes + (uint32_t)i * NT * 128;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              umma_bf16(d, smem_desc_sw128(wb + k * 32), smem_desc_sw128(ab + k * 32), idesc, acc);
+              acc = 1;
+            }
+          }
+          umma_commit(smem_u32(&ctrl->empty[stage]));          // frees the stage when the MMAs are done
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&ctrl->acc_full[buf]));
+        ++job_i;
+      }
     }
   } else {
-    pdl_wait();                                      // the partial slots may still be read by the kernel before
+    // ---- epilogue: a thread owns one output feature of the tile (its TMEM lane) and walks the
+    // activation rows (TMEM columns): hi + lo in registers, one reduction per (row, feature)
+    pdl_wait();                                      // the result matrix may still be read by the kernel before
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
-    const int row = q * 32 + lane;
-    GemmSched sched(p, NT);
+    const int feature = q * 32 + lane;
     uint32_t job_i = 0;
-    Job j;
-    while (sched.next(j, NT)) {
+    GemmWalk walk(p);
+    GemmJob j;
+    while (walk.next(j)) {
       const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
       if (!mbar_wait(smem_u32(&ctrl->acc_full[buf]), aph, &ctrl->abort)) break;
       tc_fence_after();
-      if (q * 32 < p.out_rows) {
-        // accumulator row -> result row: with hi and lo stacked in one tile the lo rows lie Rt below
-        const int orow = (p.stacked && row >= p.Rt) ? row - p.Rt : row;
-        const int grow = j.arow + orow;
-        const bool live = row < p.out_rows && grow < p.valid_rows;
-        float* dst = p.out + ((size_t)j.amap * p.Rt + grow) * p.J + j.wrow;
+      int rows = p.valid_rows - j.arow;              // live activation rows of this row tile
+      rows = rows > p.lo_col ? p.lo_col : rows;
+      float* dst = p.out + ((size_t)j.g * p.Rt + j.arow) * p.J + j.wrow + feature;
+      const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)p.n_act;
 #pragma unroll 1
-        for (int c0 = 0; c0 < NT; c0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * NT + c0, v);
-          tmem_ld_wait();
-          if (live) {
+      for (int r0 = 0; r0 < rows; r0 += 8) {
+        uint32_t hi[8], lo[8];
+        tmem_ld8(t0 + r0, hi);
+        tmem_ld8(t0 + p.lo_col + r0, lo);
+        tmem_ld_wait();
 #pragma unroll
-            for (int x = 0; x < 32; x += 4)
-              red_add_f32x4(dst + c0 + x, __uint_as_float(v[x]), __uint_as_float(v[x + 1]), __uint_as_float(v[x + 2]),
-                            __uint_as_float(v[x + 3]));
-          }
-        }
+        for (int x = 0; x < 8; ++x)
+          if (r0 + x < rows) red_add_f32(dst + (size_t)(r0 + x) * p.J, __uint_as_float(hi[x]) + __uint_as_float(lo[x]));
       }
       tc_fence_before();
       __syncwarp();
@@ -311,7 +379,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.err, 1);
-  if (warp == 2) tmem_dealloc(tmem_base, tmem_cols(NT));
+  if (warp == 2) tmem_dealloc(tmem_base, gemm_tmem_cols(p.n_act));
 }
 
 // =================================================================================================
@@ -538,11 +606,19 @@ static int pick_stages(int a_parts, int a_box_rows, int extra) {
   return s > kMaxStages ? kMaxStages : s;
 }
 
-template <int NT, int KSB, int STAGES>
+// Stages of the GEMM ring that fit beside the control block (every operand row an MMA reads is
+// loaded, so no readable padding is needed behind the ring).
+int stream_gemm_stages(int ksb, int n_act) {
+  const int stage = ksb * n_act * 128 + ksb * kGemmNT * 128;
+  const int s = (227 * 1024 - 2048) / stage;
+  return s > kMaxStages ? kMaxStages : s;
+}
+
+template <int KSB, int STAGES>
 static cudaError_t launch_gemm_t(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
-  const size_t stage = (size_t)p.a_parts * KSB * p.a_box_rows * 128 + (size_t)KSB * NT * 128;
-  const size_t smem = 1024 + 1024 + STAGES * stage + kTailPad;
-  auto kern = k_stream_gemm<NT, KSB, STAGES>;
+  const size_t stage = (size_t)KSB * p.n_act * 128 + (size_t)KSB * kGemmNT * 128;
+  const size_t smem = 1024 + 1024 + STAGES * stage;
+  auto kern = k_stream_gemm<KSB, STAGES>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   return launch_pdl(kern, dim3(grid), dim3(kThreads), smem, s, p, maps[0], maps[1], maps[2], maps[3]);
@@ -552,15 +628,18 @@ static cudaError_t launch_gemm_t(const StreamGemmParams& p, const CUtensorMap* m
 // p.ksb k-blocks per box.
 template <int KSB>
 static cudaError_t launch_stream_gemm_k(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
-  constexpr int NT = kGemmNT;
-  const int st = pick_stages<NT, KSB>(p.a_parts, p.a_box_rows, 0);
-  if (st >= 8) return launch_gemm_t<NT, KSB, 8>(p, maps, grid, s);
-  if (st >= 6) return launch_gemm_t<NT, KSB, 6>(p, maps, grid, s);
-  if (st >= 4) return launch_gemm_t<NT, KSB, 4>(p, maps, grid, s);
-  if (st >= 3) return launch_gemm_t<NT, KSB, 3>(p, maps, grid, s);
+  const int st = stream_gemm_stages(KSB, p.n_act);
+  if (st >= 8) return launch_gemm_t<KSB, 8>(p, maps, grid, s);
+  if (st >= 6) return launch_gemm_t<KSB, 6>(p, maps, grid, s);
+  if (st >= 5) return launch_gemm_t<KSB, 5>(p, maps, grid, s);
+  if (st >= 4) return launch_gemm_t<KSB, 4>(p, maps, grid, s);
+  if (st >= 3) return launch_gemm_t<KSB, 3>(p, maps, grid, s);
   return cudaErrorInvalidConfiguration;
 }
 cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
+  if (!p.out || !p.err || p.n_act != p.a_parts * p.a_box_rows || p.n_act % 16 || p.n_act < 16 || p.n_act > 256 ||
+      (p.a_parts == 2 && p.ksb != 1) || p.lo_col % 8 || p.lo_col * 2 > p.n_act)
+    return cudaErrorInvalidValue;
   if (p.ksb == 2) return launch_stream_gemm_k<2>(p, maps, grid, s);
   if (p.ksb == 1) return launch_stream_gemm_k<1>(p, maps, grid, s);
   return cudaErrorInvalidValue;

@@ -48,21 +48,25 @@ cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counte
                               LogitsPartInfo* info, Prof* prof, cudaStream_t s);
 
 // Stream-K GEMM over `groups` independent problems of identical shape (the two hyper-encoders).
-// The unit space is (group, tile, k-step); CTA c of G owns units [floor(cU/G), floor((c+1)U/G)).
-// Every maximal run of units inside one tile and one CTA is one accumulator, which the CTA adds
-// into the fp32 result matrix out[group][Rt][J] with reductions in global memory.
+// The unit space is (row tile, group, weight tile, k-step); CTA c of G owns units
+// [floor(cU/G), floor((c+1)U/G)).  Every maximal run of units inside one tile and one CTA is one
+// accumulator.  Operands are swapped with respect to the result's orientation: the 128 weight rows
+// of a tile are the MMA's M, the activation rows - hi parts and lo parts side by side - its N, so
+// that one MMA covers both parts whatever the number of rows, and a thread of the epilogue owns one
+// output feature: it adds hi and lo columns in registers and reduces the sums into the fp32
+// result matrix out[group][Rt][J] (lanes = consecutive features = consecutive addresses).
 struct StreamGemmParams {
-  int row_tiles;         // 128-row tiles of A (outermost dimension of the unit space)
+  int row_tiles;         // 128-row tiles of the activations (outermost dimension of the unit space)
   int groups, tiles_per_group, ksteps;
-  int ksb;               // 64-column k-blocks per stage and TMA box: 2 for few rows (decode), else 1
-  int a_box_rows;        // rows per TMA box of A (multiple of 8, <= 128)
-  int a_parts;           // MMA row groups per k16: 1, or 2 when hi and lo rows do not fit 128 rows
-  int a_part_row;        // first global row of part 1
-  int out_rows;          // accumulator rows that carry results
+  int ksb;               // 64-column k-blocks per stage and TMA box: 2 when the stages stay small, else 1
+  int a_box_rows;        // rows per TMA box of activations (multiple of 8)
+  int a_parts;           // boxes per stage: 1 (hi and lo rows are one contiguous box), or 2 (Rt > 128)
+  int a_part_row;        // first global row of part 1 (= Rt)
+  int n_act;             // the MMA's N: a_parts * a_box_rows, multiple of 16, <= 256
+  int lo_col;            // accumulator column of the lo part of row 0
   float* out;            // [groups][Rt][J] fp32, zero before the first add
   int J, Rt;
   int valid_rows;        // rows of the pass (results of rows beyond them are dropped)
-  int stacked;           // 1: accumulator rows [Rt, 2 Rt) are the lo parts of rows [0, Rt)
   int* err;
 };
 
@@ -109,6 +113,7 @@ cudaError_t launch_pair_gemm(const PairGemmParams& p, const void* act_hl, const 
                              cudaStream_t s);
 
 bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows);
+int stream_gemm_stages(int ksb, int n_act);
 cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s);
 cudaError_t launch_stream_logits(const StreamLogitsParams& p, const LogitMaps* maps, int grid, bool merge,
                                  Prof* prof, cudaStream_t s);

@@ -435,6 +435,24 @@ def test_tensor_core_kernels_many_rows_and_sequences():
     _decode_follow(MID_BF16, 33, zb.SELECT_ARGMAX, steps=4)
 
 
+ROWS_BF16 = si.Workload("rows_bf16", V=3000, d=256, dtype="bf16", B=2, T=220, M=3, cap=80,
+                        zipf_s=1.1, copy_p=0.4, seg_min=3, seg_max=10, steps=3, enc_layers=2,
+                        enc_heads=2, enc_dff=512)
+
+
+@pytest.mark.parametrize("w", [ROWS_BF16, ROWS_BF16.scaled(name="rows_bf16_m5", M=5, cap=45, B=3)],
+                         ids=lambda w: w.name)
+def test_weight_streaming_gemm_with_several_row_tiles(w):
+    # passes of 480 / 675 rows: below the size of the CTA-pair GEMM and above one 128-row tile, so
+    # the hi rows and the lo rows of a row tile are two operand boxes and the last tile is ragged
+    assert 128 < w.B * w.cap * w.M < 1024
+    p = Pair(w, seed=35)
+    _, worst = _prefill_both(p)
+    assert worst <= TOL
+    print(f"{w.name}: max |hyper-embedding error| = {worst:.3e}")
+    _decode_follow(w, 36, zb.SELECT_ARGMAX, steps=3)
+
+
 # ------------------------------------------------------------------------------------------------
 # Prompt-scoring logits kernel (CTA pairs, 256 x 256 tiles), forced on for small shapes:
 # several row tiles with a ragged tail, rows of several sequences inside one tile, sequences

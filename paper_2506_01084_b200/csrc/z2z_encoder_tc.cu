@@ -60,13 +60,6 @@ __device__ __forceinline__ void split_store4(bf16* hi, bf16* lo, float4 x) {
   *reinterpret_cast<uint2*>(hi) = H;
   *reinterpret_cast<uint2*>(lo) = L;
 }
-// Read 4 consecutive GEMM results and leave zeros behind.
-__device__ __forceinline__ float4 take4(float* y) {
-  const float4 v = *reinterpret_cast<const float4*>(y);
-  *reinterpret_cast<float4*>(y) = make_float4(0.f, 0.f, 0.f, 0.f);
-  return v;
-}
-
 // Base tokens of work-list entry e (0 for an unused slot): one load, so that the kernels below can
 // issue it together with their data loads instead of ahead of them.
 __device__ __forceinline__ int entry_len_tc(const CbView& cb, const EntryList& el, int e) {

@@ -435,6 +435,16 @@ def test_tensor_core_kernels_many_rows_and_sequences():
     _decode_follow(MID_BF16, 33, zb.SELECT_ARGMAX, steps=4)
 
 
+@pytest.mark.parametrize("w", [MID_BF16.scaled(name="wide_b40", d=512, enc_dff=1024, enc_heads=4, steps=3),
+                               MID_BF16.scaled(name="wide_b24", B=24, d=256, enc_dff=512, enc_heads=2, steps=3)],
+                         ids=lambda w: w.name)
+def test_weight_streaming_gemm_with_many_rows_in_one_box(w):
+    # decode passes of 120 / 72 rows: hi and lo rows side by side are more than 128 columns of one
+    # MMA (N = 240 / 144), one k-block per stage
+    assert 2 * w.B * w.M > 128
+    _decode_follow(w, 37, zb.SELECT_ARGMAX, steps=w.steps)
+
+
 ROWS_BF16 = si.Workload("rows_bf16", V=3000, d=256, dtype="bf16", B=2, T=220, M=3, cap=80,
                         zipf_s=1.1, copy_p=0.4, seg_min=3, seg_max=10, steps=3, enc_layers=2,
                         enc_heads=2, enc_dff=512)

@@ -10,8 +10,8 @@
 //
 // Layout of a hi/lo operand with Rt rows: bf16 [2 * Rt, K], hi rows first, lo rows after.
 //
-// GEMM output.  Every CTA of the stream-K GEMM adds its partial tiles (hi and lo parts alike)
-// into ONE fp32 matrix Y[group][Rt][J] with vector reductions in global memory; Y is all zero
+// GEMM output.  Every CTA of the stream-K GEMM adds its partial tiles (hi and lo parts summed
+// in registers) into ONE fp32 matrix Y[group][Rt][J] with reductions in global memory; Y is all zero
 // whenever no GEMM result is pending.  The element-wise kernel after a GEMM reads each element of
 // that GEMM's result exactly once and stores zero back ("consume and clear"), for every row of
 // the pass whether or not it belongs to a live entry, which restores the invariant for the next
@@ -20,6 +20,10 @@
 // Launches per layer: GEMM(qkv) -> [+ bias, attention] -> GEMM(o) -> [+ bias + residual,
 // LayerNorm 2] -> GEMM(1) -> [+ bias, GELU] -> GEMM(2) -> [+ bias + residual, LayerNorm 1 of the
 // next layer | mean-pool into the cache].  All are launched with programmatic serialization.
+// Between two GEMMs the weight stream stands still, so the small kernels are written for latency:
+// what a kernel needs about an entry (its length, the base token of a row) is one load from the
+// work list, and every data load is issued before the first value is used - whether a row is valid
+// only decides what is stored.
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
 #include "z2z_sm100.cuh"

@@ -1,20 +1,22 @@
 // Weight-streaming skinny GEMM on tcgen05 tensor cores, for the HBM-bound decode regime.
 //
-//   D[r, j] = sum_k A[r, k] * W[j, k]      A: <=128 activation rows (bf16, K-major)
+//   D[r, j] = sum_k A[r, k] * W[j, k]      A: activation rows (bf16, K-major), few
 //                                          W: weight rows streamed once from HBM (bf16, K-major)
 //
 // One persistent CTA per SM.  Warp 0 issues TMA loads into a ring of shared-memory stages, warp 1
-// issues tcgen05.mma (activations as the 128-row M operand, a tile of NT weight rows as the N
-// operand, fp32 accumulator in tensor memory, double buffered), warps 2-5 drain accumulators.
-// Two uses share the pipeline:
-//   * hyper-encoder linear layers: work is cut stream-K style, every CTA gets the same number of
-//     (tile, k-step) units, and each CTA stores fp32 partial tiles that the next (element-wise)
-//     kernel sums in a fixed order, so results are deterministic;
-//   * joint logits (paper Section 2.3 steps 7-9): tiles run over W_U and then over the visible
+// issues tcgen05.mma (fp32 accumulators in tensor memory, double buffered), warps 2-5 drain
+// accumulators.  Two kernels share the ring and its barriers:
+//   * hyper-encoder linear layers (k_stream_gemm): a tile of 128 weight rows is the MMA's M
+//     operand, the activation rows (hi parts | lo parts) its N operand; work is cut stream-K
+//     style, every CTA gets the same number of (tile, k-step) units and adds its accumulators
+//     into one fp32 result matrix with reductions in global memory (sums of two or three partial
+//     tiles in arrival order);
+//   * joint logits for 33 .. 2047 hidden rows (k_stream_logits; paper Section 2.3 steps 7-9):
+//     the hidden rows are the 128-row M operand, tiles run over W_U and then over the visible
 //     rows of each sequence's U_h; the epilogue keeps max / sum-exp / argmax / best perturbed
-//     score per hidden row in registers, so the logits are never written.
-// Only the rows of A that exist are loaded: the MMA also reads the shared memory behind them,
-// which only feeds accumulator rows nobody reads (rows of D depend on the same rows of A only).
+//     score per hidden row in registers, so the logits are never written.  Only the hidden rows
+//     that exist are loaded: the MMA also reads the shared memory behind them, which only feeds
+//     accumulator rows nobody reads (rows of D depend on the same rows of A only).
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
 #include "z2z_sm100.cuh"

@@ -142,14 +142,18 @@ def reduce_over_ranks(times_ms, counts, world: int, device):
 
 
 def kernel_source_digest() -> str:
-    """Digest of the sources of the streaming kernels; an ncu traffic figure only counts while it
-    matches the code that produced it."""
+    """Digest of the code of the streaming kernels (comments and blank space left out); an ncu
+    traffic figure only counts while it matches the code that produced it."""
     import hashlib
+    import re
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2506_01084_b200", "csrc")
     for f in ("z2z_stream.cu", "z2z_stream.h", "z2z_sm100.cuh", "z2z_decode_logits.cu"):
-        with open(os.path.join(d, f), "rb") as fh:
-            h.update(fh.read())
+        with open(os.path.join(d, f), "r") as fh:
+            text = fh.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update(" ".join(text.split()).encode())
     return h.hexdigest()[:12]
 
 

@@ -87,6 +87,10 @@ int32_t z2z_workspace_bytes(const z2z_config* cfg, size_t* out_bytes);
  * called again on an existing handle to start a new session.                                   */
 int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, size_t ws_bytes,
                           z2z_stream stream);
+/* (The handle also owns 64 bytes of pinned host memory, freed by z2z_codebook_destroy: the decode
+ * step's update kernel stores the session number there once every sequence's codebook is full.
+ * From then on no step can create an entry, and z2z_decode_step no longer launches the
+ * hyper-encoder pass - the weights of both encoders are not streamed for nothing.)             */
 
 /* Section 2.1 / Section 2.3 step 2: compress each prompt with LZW (greedy longest match against
  * the growing codebook; new entry = emitted phrase + next base token, only if shorter than M

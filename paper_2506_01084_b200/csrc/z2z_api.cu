@@ -17,6 +17,8 @@ struct z2z_codebook {
   int dff, heads;
   int use_tensor_cores;      // 0: CUDA cores, 1: tensor cores (kernel by shape), 2: prompt-scoring kernel always
   int prefill_strips;        // > 0: fixed number of column strips in the prompt-scoring kernel
+  int* h_frozen;             // pinned host word the decode-update kernel writes once every codebook is full
+  int epoch;                 // session number: incremented by every z2z_codebook_init
   z2z::Prof prof;
 };
 
@@ -185,6 +187,15 @@ int32_t z2z_codebook_init(z2z_codebook** cb, const z2z_config* cfg, void* d_ws, 
   h->dff = c.enc_dff; h->heads = c.enc_heads;
   h->use_tensor_cores = 1;
   h->prefill_strips = 0;
+  if (!h->h_frozen) {
+    // one word of pinned, device-visible host memory (host memory: the device workspace stays the caller's);
+    // without it the session simply never learns that its codebooks are frozen
+    void* p = nullptr;
+    if (cudaHostAlloc(&p, 64, cudaHostAllocMapped | cudaHostAllocPortable) == cudaSuccess) h->h_frozen = reinterpret_cast<int*>(p);
+    else (void)cudaGetLastError();
+  }
+  ++h->epoch;
+  if (h->h_frozen) *reinterpret_cast<volatile int*>(h->h_frozen) = 0;
   z2z::CbView& v = h->view;
   v.V = c.V; v.M = c.M; v.cap = c.cap; v.B = c.B; v.n_slots = plan.n_slots;
   v.hash = reinterpret_cast<unsigned long long*>(h->ws + plan.off_hash);
@@ -369,6 +380,7 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
     u.lpart = reinterpret_cast<const z2z::LogitPartial*>(a.lpart);
     u.part_stride = info.stride; u.part_count = info.count; u.select = select; u.forced = d_forced;
     u.next_codes = d_next_codes; u.selected = d_selected; u.lse = a.lse; u.new_entry = w_new;
+    u.frozen_flag = cb->h_frozen; u.epoch = cb->epoch;
     z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, s);
     Z2Z_CUDA(z2z::launch_decode_update(cb->view, u, el, s), "decode_step");
   } else {
@@ -391,8 +403,10 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
       Z2Z_CUDA(z2z::launch_mark_embedded(cb->view, 1, s), "decode_step");
     }
   }
-  // cache update: the at most one new entry per sequence, on both sides
-  if (cb->cfg.cap > 0) {
+  // cache update: the at most one new entry per sequence, on both sides.  Once an earlier step has
+  // reported that every codebook is full nothing can be created any more and the pass is not launched.
+  const bool frozen = cb->h_frozen && *reinterpret_cast<volatile int*>(cb->h_frozen) == cb->epoch;
+  if (cb->cfg.cap > 0 && !frozen) {
     const bool tc = cb->use_tensor_cores && z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype, cb->heads, cb->cfg.M);
     z2z::EncoderArgs g[2];
     g[0] = encoder_args(cb, d_WE, enc_E, d_Eh, d_Eh_f32, B, 0);
@@ -486,6 +500,7 @@ int32_t z2z_profile_read(z2z_codebook* cb, int32_t n_classes, double* h_ms, int6
 }
 
 int32_t z2z_codebook_destroy(z2z_codebook* cb) {
+  if (cb && cb->h_frozen) cudaFreeHost(cb->h_frozen);
   delete cb;
   return Z2Z_OK;
 }

@@ -90,7 +90,19 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
     for (int i = 0; i < cb.M; ++i) el.tok[(size_t)e * cb.M + i] = -1;
   }
   // both caches will hold every entry once the encoder pass that follows has run
-  if (tid < cb.B) { const int n = cb.n[tid]; cb.n_emb[tid] = n; cb.n_emb[cb.B + tid] = n; }
+  int full = 1;
+  if (tid < cb.B) {
+    const int n = cb.n[tid];
+    cb.n_emb[tid] = n; cb.n_emb[cb.B + tid] = n;
+    full = n >= cb.cap;
+  }
+  // Once every codebook is full no step creates an entry any more.  The host learns it through a
+  // word in its own memory and stops launching the hyper-encoder pass (the session number guards
+  // against a late store from before a reset).
+  if (a.frozen_flag && cb.B <= (int)blockDim.x) {
+    const int all_full = __syncthreads_and(full);
+    if (all_full && tid == 0) *reinterpret_cast<volatile int*>(a.frozen_flag) = a.epoch;
+  }
 }
 
 cudaError_t launch_decode_update(const CbView& cb, const DecodeUpdateArgs& a, const EntryList& el,

@@ -124,6 +124,8 @@ struct DecodeUpdateArgs {
   int select;
   const int32_t* forced;
   int32_t* next_codes; int32_t* selected; float* lse; int32_t* new_entry;
+  int* frozen_flag;   // host word mapped into the device's address space, or NULL
+  int epoch;          // written there once every codebook of the session is full
 };
 cudaError_t launch_decode_update(const CbView& cb, const DecodeUpdateArgs& a, const EntryList& el,
                                  cudaStream_t s);

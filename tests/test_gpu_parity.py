@@ -391,6 +391,36 @@ def test_decode_step_tiny_config_argmax():
     print(f"tiny: followed {followed} near-ties, worst |LSE error| {worst:.2e}")
 
 
+def test_decode_step_with_frozen_codebooks():
+    # cap reached during the prompt: no step creates an entry, the hyper-encoder GEMMs find no live
+    # entry and leave early; selections, LSE and the (unchanged) caches must still match
+    w = SMALL_BF16.scaled(name="frozen", cap=24)
+    p = Pair(w, seed=41)
+    _prefill_both(p)
+    assert all(bk.n() == w.cap for bk in p.oracle.books)
+    _decode_follow(w, 41, zb.SELECT_ARGMAX, steps=5)
+    _decode_follow(w, 42, zb.SELECT_GUMBEL, steps=4, forced_every=2)
+    # ... and once the host has seen that everything is full the encoder pass is not launched at all
+    hid = si.make_hidden(w, 4 * w.B, 43).view(4, w.B, w.d).to(p.dev)
+    nxt = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    per_step = []
+    for t in range(4):
+        zb.z2z_profile_read(p.cb)
+        zb.z2z_decode_step(p.cb, hid[t], p.g_WE, p.g_WU, p.g_encE, p.g_encU, p.E_h, p.U_h, zb.SELECT_ARGMAX, 1.0,
+                           0, t, None, nxt, None, None)
+        _, launches = zb.z2z_profile_read(p.cb)              # waits for the stream
+        per_step.append(launches)
+    assert per_step[0]["encoder_gemm"] > 0                    # the step that reports the state still runs the pass
+    assert all(s["encoder_gemm"] == 0 and s["encoder_other"] == 0 for s in per_step[1:]), per_step
+    # a new session on the same handle starts unfrozen
+    zb.z2z_codebook_init(p.cb)
+    zb.z2z_profile_read(p.cb)
+    zb.z2z_decode_step(p.cb, hid[0], p.g_WE, p.g_WU, p.g_encE, p.g_encU, p.E_h, p.U_h, zb.SELECT_ARGMAX, 1.0,
+                       0, 0, None, nxt, None, None)
+    _, launches = zb.z2z_profile_read(p.cb)
+    assert launches["encoder_gemm"] > 0
+
+
 def test_decode_step_results_written_to_pinned_host_memory():
     for w, sel in ((si.WORKLOADS["tiny"], zb.SELECT_ARGMAX), (SMALL_BF16, zb.SELECT_GUMBEL)):
         _decode_follow(w, 27, sel, steps=6, forced_every=3, host_results=True)

@@ -62,6 +62,8 @@ z2z::EntryList entry_list(z2z_codebook* cb) {
   el.idx = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_idx);
   el.len = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_len);
   el.tok = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_tok);
+  el.row_off = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_row_off);
+  el.row_src = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_row_src);
   el.off = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_off);
   el.chunk = cb->plan.enc_chunk_entries;
   return el;

@@ -384,13 +384,99 @@ __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias,
   }
 }
 
-// LayerNorm of the valid rows of X -> hi/lo (prompt-sized passes: the GEMM epilogue has already
-// added bias and residual into X).  grid (rows), one encoder.
-__global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(CbView cb, EntryList el, const float* X, const bf16* ln_w,
+// Prompt-sized passes keep their rows PACKED: entry e owns rows row_off[e] .. row_off[e] + len[e],
+// there are no padding rows inside entries, and rows at or beyond the total carry nothing.  (With
+// M = 3 or 4 a quarter to a third of the padded rows would be zeros that the GEMMs multiply anyway.)
+//
+// One block: first packed row of every entry (exclusive scan of the lengths), the total behind the
+// last entry, and the way back from a packed row to (entry, position).  E <= 1024 entries.
+__global__ void __launch_bounds__(1024) k_tc_row_map(CbView cb, EntryList el, int E) {
+  __shared__ int warp_sums[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int len = tid < E ? entry_len_tc(cb, el, tid) : 0;
+  int inc = len;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += x;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += x;
+    }
+    warp_sums[lane] = w;
+  }
+  __syncthreads();
+  const int excl = inc - len + (warp > 0 ? warp_sums[warp - 1] : 0);
+  if (tid < E) {
+    el.row_off[tid] = excl;
+    for (int i = 0; i < len; ++i) el.row_src[excl + i] = tid * cb.M + i;
+  }
+  if (tid == 0) el.row_off[E] = warp_sums[31];
+}
+
+// X = table[y] + pos for every packed row, then LN1 of layer 0 -> hi/lo.  grid (row capacity).
+__global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln_packed(CbView cb, EntryList el, const int* total,
+                                                                     const bf16* table, const bf16* pos, const bf16* ln_w,
+                                                                     const bf16* ln_b, float* X, bf16* Ahl, int d, int Rt,
+                                                                     int has_ln) {
+  __shared__ float sm[32];
+  const int r = blockIdx.x;
+  if (r >= *total) return;
+  const int src = el.row_src[r];
+  const int y = el.tok[src], i = src % cb.M;
+  float* x = X + (size_t)r * d;
+  bf16* hi = Ahl + (size_t)r * d;
+  const bf16* row = table + (size_t)y * d;
+  const bf16* pp = pos + (size_t)i * d;
+  const int nvec = d / 4;
+  float4 xv[kMaxVec4];
+  uint2 gw[kMaxVec4], gb[kMaxVec4];
+#pragma unroll
+  for (int v = 0; v < kMaxVec4; ++v) {
+    const int idx = (int)threadIdx.x + v * kRowThreads;
+    if (idx < nvec) {
+      const float4 a = load_bf16x4(row + idx * 4), b = load_bf16x4(pp + idx * 4);
+      gw[v] = reinterpret_cast<const uint2*>(ln_w)[idx];
+      gb[v] = reinterpret_cast<const uint2*>(ln_b)[idx];
+      xv[v] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+      *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
+    }
+  }
+  if (has_ln) layernorm_split_regs(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
+}
+
+// Zero-layer encoder on packed rows: cache row = mean of the entry's rows of X.  grid (entries).
+__global__ void __launch_bounds__(kRowThreads) k_tc_pool_packed(CbView cb, EntryList el, const float* X, void* cache,
+                                                                float* cache_f32, int d) {
+  const int e = blockIdx.x;
+  const int L = entry_len_tc(cb, el, e);
+  if (L <= 0) return;
+  const float* x = X + (size_t)el.row_off[e] * d;
+  const size_t dst = ((size_t)el.seq[e] * cb.cap + el.idx[e]) * d;
+  const float inv = 1.0f / (float)L;
+  bf16* out = reinterpret_cast<bf16*>(cache);
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float v = 0.f;
+    for (int i = 0; i < L; ++i) v += x[(size_t)i * d + c];
+    v *= inv;
+    out[dst + c] = __float2bfloat16_rn(v);
+    if (cache_f32) cache_f32[dst + c] = v;
+  }
+}
+
+// LayerNorm of the packed rows of X -> hi/lo (the GEMM epilogue has already added bias and
+// residual into X).  grid (row capacity), one encoder.
+__global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, const float* X, const bf16* ln_w,
                                                             const bf16* ln_b, bf16* Ahl, int d, int Rt) {
   __shared__ float sm[32];
-  const int r = blockIdx.x, e = r / cb.M, i = r - e * cb.M;
-  if (i >= entry_len_tc(cb, el, e)) return;                              // padding rows stay zero in hi/lo
+  const int r = blockIdx.x;
+  if (r >= *total) return;
   const float* x = X + (size_t)r * d;
   const int nvec = d / 4;
   float4 xv[kMaxVec4];
@@ -408,15 +494,15 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(CbView cb, EntryList
   layernorm_split_regs(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
-// Bidirectional attention inside one entry from fp32 q, k, v rows [R, 3d] (bias already added);
-// output as hi/lo.  grid (entries, heads), block (32, M), dynamic smem M * 3 * dh floats.
+// Bidirectional attention inside one entry from fp32 q, k, v of its packed rows [rows, 3d] (bias
+// already added); output as hi/lo.  grid (entries, heads), block (32, M), dynamic smem M * 3 * dh floats.
 __global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, bf16* Ohl, int d, int heads, int Rt) {
   extern __shared__ float s_qkv[];
   const int e = blockIdx.x, h = blockIdx.y, i = threadIdx.y, lane = threadIdx.x;
   const int L = entry_len_tc(cb, el, e);
   if (L <= 0) return;
   const int dh = d / heads;
-  const int r = e * cb.M + i;
+  const int r = el.row_off[e] + i;
   if (i < L) {
     const float* y = QKV + (size_t)r * 3 * d;
     for (int w = 0; w < 3; ++w)
@@ -485,12 +571,9 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
   const int d = a.d, dff = a.dff, M = cb.M;
   const int R = E * M, Rt = (R + 7) / 8 * 8;
   auto Wp = [&](int i) { return reinterpret_cast<const bf16*>(a.w[i]); };
-  Ptr2 table, pos, lw, lb; MPtr2 X, Ahl, cache, c32;
-  table.p[0] = table.p[1] = a.table; pos.p[0] = pos.p[1] = a.w[0];
-  lw.p[0] = lw.p[1] = a.layers ? a.w[1] : a.w[0]; lb.p[0] = lb.p[1] = a.layers ? a.w[2] : a.w[0];
-  X.p[0] = X.p[1] = a.X; Ahl.p[0] = Ahl.p[1] = a.Ahl; cache.p[0] = cache.p[1] = a.cache; c32.p[0] = c32.p[1] = a.cache_f32;
+  const int* total = el.row_off + E;                   // packed rows of this pass (device word)
   PairGemmParams g{};
-  g.cb = cb; g.el = el; g.R = R; g.Rt = Rt; g.err = a.err;
+  g.cb = cb; g.el = el; g.R = R; g.Rt = Rt; g.live_rows = total; g.err = a.err;
   auto gemm = [&](const bf16* act, int K, int widx, int J, int epi, float* out, bf16* out_hl) -> cudaError_t {
     PairGemmParams p = g;
     p.J = J; p.bias = a.w[widx + 1]; p.out = out; p.out_hl = out_hl;
@@ -498,9 +581,11 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
     return launch_pair_gemm(p, act, a.w[widx], K, epi, s);
   };
   {
-    ProfScope ps(prof, kProfEncOther, 1, s);
-    launch_pdl(k_tc_gather_ln, dim3(R, 1), dim3(kRowThreads), 0, s, cb, el, table, pos, lw, lb, X, Ahl, d, Rt,
-               a.layers > 0 ? 1 : 0);
+    ProfScope ps(prof, kProfEncOther, 2, s);
+    k_tc_row_map<<<1, 1024, 0, s>>>(cb, el, E);
+    k_tc_gather_ln_packed<<<R, kRowThreads, 0, s>>>(cb, el, total, reinterpret_cast<const bf16*>(a.table), Wp(0),
+                                                    a.layers ? Wp(1) : Wp(0), a.layers ? Wp(2) : Wp(0), a.X, a.Ahl, d,
+                                                    Rt, a.layers > 0 ? 1 : 0);
   }
   const int dh = d / a.heads;
   cudaError_t e;
@@ -515,17 +600,17 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
     if ((e = gemm(a.Ahl, d, o + 4, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(cb, el, a.X, Wp(o + 6), Wp(o + 7), a.Ahl, d, Rt);
+      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 6), Wp(o + 7), a.Ahl, d, Rt);
     }
     if ((e = gemm(a.Ahl, d, o + 8, dff, kEpiGelu, nullptr, a.Hhl)) != cudaSuccess) return e;
     if ((e = gemm(a.Hhl, dff, o + 10, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     if (l + 1 < a.layers) {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(cb, el, a.X, Wp(o + 12), Wp(o + 13), a.Ahl, d, Rt);
+      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 12), Wp(o + 13), a.Ahl, d, Rt);
     }
   }
   ProfScope ps(prof, kProfEncOther, 1, s);
-  launch_pdl(k_tc_pool, dim3(E, 1), dim3(kRowThreads), 0, s, cb, el, X, cache, c32, d);
+  k_tc_pool_packed<<<E, kRowThreads, 0, s>>>(cb, el, a.X, a.cache, a.cache_f32, d);
   return cudaGetLastError();
 }
 

@@ -47,6 +47,8 @@ struct EntryList {
   int32_t* idx;       // [chunk]  entry number within the sequence
   int32_t* len;       // [chunk]  base tokens of the entry, 0 for an unused slot
   int32_t* tok;       // [chunk * M]  base token of each row of the entry, -1 for padding rows
+  int32_t* row_off;   // [chunk + 1]  prompt-sized passes: first packed row of each entry, then the row total
+  int32_t* row_src;   // [chunk * M]  prompt-sized passes: packed row -> entry * M + position
   int32_t* off;       // [B + 2]  exclusive prefix sum of per-sequence counts, then the total
   int chunk;
 };

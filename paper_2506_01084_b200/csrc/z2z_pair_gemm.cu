@@ -49,7 +49,7 @@ k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, con
   const int n_clusters = gridDim.x >> 1, cluster_id = blockIdx.x >> 1;
   // only the row tiles that hold rows of live entries of this pass are computed (the host sizes
   // the launch for its upper bound of entries; the count itself is device state)
-  int live_rows = p.el.off[p.cb.B + 1] * p.cb.M;
+  int live_rows = *p.live_rows;                     // rows are packed: no padding rows inside entries
   live_rows = live_rows < p.R ? live_rows : p.R;
   const int row_tiles = (live_rows + 255) / 256;
   const int n_tiles = row_tiles * p.col_tiles;
@@ -143,15 +143,7 @@ k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, con
     for (int t = cluster_id; t < n_tiles; t += n_clusters) {
       const int rt = t % row_tiles, ct = t / row_tiles;
       const int r = rt * 256 + (int)rank * 128 + q * 32 + lane;
-      // a row carries data if it belongs to a live entry of the pass and is not padding of it
-      bool valid = false;
-      if (r < p.R) {
-        const int e = r / p.cb.M, i = r - e * p.cb.M;
-        if (e < p.el.off[p.cb.B + 1]) {
-          const int sq = p.el.seq[e];
-          valid = sq >= 0 && i < (int)p.cb.len[(size_t)sq * p.cb.cap + p.el.idx[e]];
-        }
-      }
+      const bool valid = r < live_rows;               // packed rows: every row below the total carries data
       const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
       if (!mbar_wait(smem_u32(&ctrl->acc_full[buf]), aph, &ctrl->abort)) break;
       tc_fence_after();

@@ -101,7 +101,8 @@ enum { kEpiStore = 0, kEpiResid = 1, kEpiGelu = 2 };
 struct PairGemmParams {
   CbView cb;
   EntryList el;
-  int R, Rt;             // rows of the pass; rows per hi (or lo) block of the operands
+  int R, Rt;             // row capacity of the pass; rows per hi (or lo) block of the operands
+  const int* live_rows;  // device word: packed rows that carry data (rows of live entries, no padding)
   int J;                 // output columns (a multiple of 128)
   const void* bias;      // [J] bf16
   float* out;            // kEpiStore / kEpiResid: fp32 [R, J]

@@ -495,7 +495,66 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, co
 }
 
 // Bidirectional attention inside one entry from fp32 q, k, v of its packed rows [rows, 3d] (bias
-// already added); output as hi/lo.  grid (entries, heads), block (32, M), dynamic smem M * 3 * dh floats.
+// already added); output as hi/lo.  One WARP per (entry, head): all of the item's q, k, v values
+// are loaded into registers at once (a lane holds four columns of every row), the L x L scores are
+// warp reductions, no shared memory and no block barrier.  MM = compile-time bound on the merge
+// size; dh <= 128 (larger heads take the kernel below).  grid = ceil(entries * heads / 8), block 256.
+template <int MM>
+__global__ void __launch_bounds__(256) k_tc_attention_rows_warp(CbView cb, EntryList el, const float* QKV, bf16* Ohl,
+                                                                int E, int d, int heads, int Rt) {
+  const int lane = threadIdx.x & 31;
+  const int item = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (item >= E * heads) return;
+  const int e = item / heads, h = item - e * heads;
+  const int L = entry_len_tc(cb, el, e);
+  if (L <= 0) return;
+  const int dh = d / heads, c = lane * 4;
+  const bool on = c < dh;                      // lanes beyond the head's width hold zeros
+  const size_t r0 = el.row_off[e];
+  const float* y = QKV + r0 * 3 * d + (size_t)h * dh + c;
+  float4 q[MM], k[MM], v[MM];
+#pragma unroll
+  for (int i = 0; i < MM; ++i) {
+    q[i] = k[i] = v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < L && on) {
+      const float* yi = y + (size_t)i * 3 * d;
+      q[i] = *reinterpret_cast<const float4*>(yi);
+      k[i] = *reinterpret_cast<const float4*>(yi + d);
+      v[i] = *reinterpret_cast<const float4*>(yi + 2 * d);
+    }
+  }
+  const float scale = 1.0f / sqrtf((float)dh);
+  bf16* hi = Ohl + r0 * d + (size_t)h * dh + c;
+  bf16* lo = hi + (size_t)Rt * d;
+#pragma unroll
+  for (int i = 0; i < MM; ++i) {
+    if (i >= L) break;
+    float s[MM];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < MM; ++j) {
+      float p = q[i].x * k[j].x + q[i].y * k[j].y + q[i].z * k[j].z + q[i].w * k[j].w;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) p += __shfl_xor_sync(0xffffffffu, p, off);
+      s[j] = j < L ? p * scale : -INFINITY;
+      mx = fmaxf(mx, s[j]);
+    }
+    float den = 0.f;
+#pragma unroll
+    for (int j = 0; j < MM; ++j) { s[j] = j < L ? expf(s[j] - mx) : 0.f; den += s[j]; }
+    const float inv = 1.0f / den;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < MM; ++j) {
+      const float wj = s[j] * inv;
+      o.x = fmaf(wj, v[j].x, o.x); o.y = fmaf(wj, v[j].y, o.y); o.z = fmaf(wj, v[j].z, o.z); o.w = fmaf(wj, v[j].w, o.w);
+    }
+    if (on) split_store4(hi + (size_t)i * d, lo + (size_t)i * d, o);
+  }
+}
+
+// The same for heads wider than 128 columns or merge sizes above 4: staged in shared memory.
+// grid (entries, heads), block (32, M), dynamic smem M * 3 * dh floats.
 __global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, bf16* Ohl, int d, int heads, int Rt) {
   extern __shared__ float s_qkv[];
   const int e = blockIdx.x, h = blockIdx.y, i = threadIdx.y, lane = threadIdx.x;
@@ -510,7 +569,7 @@ __global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, b
         *reinterpret_cast<float4*>(&s_qkv[(i * 3 + w) * dh + c]) = *reinterpret_cast<const float4*>(y + w * d + h * dh + c);
   }
   __syncthreads();
-  if (i >= L) return;                          // padding rows of the operand stay zero
+  if (i >= L) return;
   const float* q = s_qkv + (i * 3) * dh;
   const float scale = 1.0f / sqrtf((float)dh);
   float s[kMaxM];
@@ -594,8 +653,11 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
     if ((e = gemm(a.Ahl, d, o + 2, 3 * d, kEpiStore, a.QKV, nullptr)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_attention_rows<<<dim3(E, a.heads), dim3(32, M), (size_t)M * 3 * dh * 4, s>>>(cb, el, a.QKV, a.Ahl, d,
-                                                                                         a.heads, Rt);
+      if (dh <= 128 && M <= 4)
+        k_tc_attention_rows_warp<4><<<(E * a.heads + 7) / 8, 256, 0, s>>>(cb, el, a.QKV, a.Ahl, E, d, a.heads, Rt);
+      else
+        k_tc_attention_rows<<<dim3(E, a.heads), dim3(32, M), (size_t)M * 3 * dh * 4, s>>>(cb, el, a.QKV, a.Ahl, d,
+                                                                                           a.heads, Rt);
     }
     if ((e = gemm(a.Ahl, d, o + 4, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     {

@@ -317,6 +317,10 @@ def run_ours(args, rank: int, world: int):
     (dev_ms, e2e_ms), (bt_dev, bt_e2e) = reduce_over_ranks([dev_ms, e2e_ms], [bt_dev, bt_e2e], world, dev)
 
     pk = peaks()
+    step_input_bytes = (2 if w.dtype == "bf16" else 4) * (w.V * w.d + 2 * w.enc_layers * (4 * w.d * w.d + 2 * w.d * w.dff))
+    l2_note = ("per-step inputs (W_U and both encoders' weights) exceed the 126 MB L2" if step_input_bytes > 126e6 else
+               "per-step inputs (%.1f MB) fit the 126 MB L2 and are not flushed between steps: a small parity "
+               "configuration, not the one the metric is quoted on" % (step_input_bytes / 1e6))
     # dominant kernel class by measured time
     mean_hyper = 0.5 * (n_after + n_after2)     # hyper rows visible during the profiled pass
     classes = {"logits": logits_bytes(w, mean_hyper), "encoder_gemm": encoder_gemm_bytes(w)}
@@ -350,7 +354,7 @@ def run_ours(args, rank: int, world: int):
         "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "prompt_tokens": w.T,
                    "M": w.M, "cap": w.cap, "enc_layers": w.enc_layers, "enc_dff": w.dff,
                    "select": "argmax, free-running", "replicas": world,
-                   "l2": "per-step inputs (W_U and both encoders' weights) exceed the 126 MB L2"},
+                   "l2": l2_note},
         "steps_per_s": K / (dev_ms * 1e-3),
         "mean_phrase_len": bt_dev / (K * w.B * world),
         "new_entries_in_timed_region": int(n_after - n_before),

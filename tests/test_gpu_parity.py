@@ -493,6 +493,19 @@ def test_weight_streaming_gemm_with_several_row_tiles(w):
     _decode_follow(w, 36, zb.SELECT_ARGMAX, steps=3)
 
 
+@pytest.mark.parametrize("w", [SMALL_BF16.scaled(name="pair_m5", M=5, B=2, cap=240, T=900),
+                               SMALL_BF16.scaled(name="pair_dh256", d=512, enc_heads=2, enc_dff=1024, B=3, cap=120, T=420)],
+                         ids=lambda w: w.name)
+def test_prompt_sized_pass_with_long_entries_and_wide_heads(w):
+    # passes of >= 1024 rows (CTA-pair GEMMs, packed rows) whose attention does not fit the
+    # registers of one warp: merge size 5, or heads of 256 columns
+    assert w.B * w.cap * w.M >= 1024
+    p = Pair(w, seed=45)
+    _, worst = _prefill_both(p)
+    assert worst <= TOL
+    print(f"{w.name}: max |hyper-embedding error| = {worst:.3e}")
+
+
 # ------------------------------------------------------------------------------------------------
 # Prompt-scoring logits kernel (CTA pairs, 256 x 256 tiles), forced on for small shapes:
 # several row tiles with a ragged tail, rows of several sequences inside one tile, sequences

@@ -391,6 +391,16 @@ def test_decode_step_tiny_config_argmax():
     print(f"tiny: followed {followed} near-ties, worst |LSE error| {worst:.2e}")
 
 
+@pytest.mark.parametrize("w", [si.WORKLOADS["tiny"].scaled(name="tiny_b130", B=130, T=48, cap=24, steps=3),
+                               SMALL_BF16.scaled(name="small_b130", B=130, T=40, cap=16, d=128, enc_dff=256, enc_heads=1,
+                                                 steps=2)], ids=lambda w: w.name)
+def test_decode_step_with_more_than_128_sequences(w):
+    # beyond 128 sequences the step takes separate launches for merge, selection, LZW update and the
+    # encoder's work list instead of the single fused update kernel
+    _decode_follow(w, 47, zb.SELECT_ARGMAX, steps=w.steps)
+    _decode_follow(w, 48, zb.SELECT_GUMBEL, steps=2, forced_every=2)
+
+
 def test_decode_step_with_frozen_codebooks():
     # cap reached during the prompt: no step creates an entry, the hyper-encoder GEMMs find no live
     # entry and leave early; selections, LSE and the (unchanged) caches must still match

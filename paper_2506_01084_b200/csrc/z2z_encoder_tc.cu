@@ -37,6 +37,7 @@ using bf16 = __nv_bfloat16;
 constexpr int kNT = kGemmNT;
 constexpr int kRowThreads = 256;
 constexpr int kMaxVec4 = 8;            // float4 per thread in the row kernels: d <= 8192
+constexpr int kNarrowVec4 = 4;         // ... and for d <= 4096, where half the registers do
 constexpr int kPairPassMinRows = 1024; // passes of at least this many rows use the CTA-pair GEMM
 
 struct Ptr2 { const void* p[2]; };
@@ -91,23 +92,24 @@ __device__ __forceinline__ float block_sum(float v, float* sm) {
 // written as hi/lo bf16.  eps 1e-5, biased variance, two-pass.
 // gw / gb: gamma and beta of the thread's columns, packed 4 bf16 per uint2 and loaded by the caller
 // together with the row, so that no load waits behind the reductions.
-__device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[kMaxVec4], int nvec, const uint2 (&gw)[kMaxVec4],
-                                                     const uint2 (&gb)[kMaxVec4], bf16* hi, bf16* lo, int d, float* sm) {
+template <int NV>
+__device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[NV], int nvec, const uint2 (&gw)[NV],
+                                                     const uint2 (&gb)[NV], bf16* hi, bf16* lo, int d, float* sm) {
   float s = 0.f;
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v)
+  for (int v = 0; v < NV; ++v)
     if ((int)threadIdx.x + v * kRowThreads < nvec) s += (x[v].x + x[v].y) + (x[v].z + x[v].w);
   const float mean = block_sum(s, sm) / (float)d;
   float q = 0.f;
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v)
+  for (int v = 0; v < NV; ++v)
     if ((int)threadIdx.x + v * kRowThreads < nvec) {
       const float a = x[v].x - mean, bb = x[v].y - mean, c = x[v].z - mean, e = x[v].w - mean;
       q += (a * a + bb * bb) + (c * c + e * e);
     }
   const float rstd = 1.0f / sqrtf(block_sum(q, sm) / (float)d + kLnEps);
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
+  for (int v = 0; v < NV; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       const float4 gg = unpack_bf16x4(gw[v]), bb = unpack_bf16x4(gb[v]);
@@ -122,6 +124,7 @@ __device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[kMaxVec4]
 }
 
 // X = table[y] + pos for valid rows; then LN1 of layer 0 -> hi/lo.  grid (rows, groups).
+template <int NV>
 __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryList el, Ptr2 table, Ptr2 pos,
                                                               Ptr2 ln_w, Ptr2 ln_b, MPtr2 X, MPtr2 Ahl,
                                                               int d, int Rt, int has_ln) {
@@ -147,10 +150,10 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
   const bf16* pp = reinterpret_cast<const bf16*>(pos.p[g]) + (size_t)i * d;
   const uint2* lw = reinterpret_cast<const uint2*>(ln_w.p[g]);
   const uint2* lb = reinterpret_cast<const uint2*>(ln_b.p[g]);
-  float4 xv[kMaxVec4];
-  uint2 gw[kMaxVec4], gb[kMaxVec4];
+  float4 xv[NV];
+  uint2 gw[NV], gb[NV];
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
+  for (int v = 0; v < NV; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       const float4 a = load_bf16x4(row + idx * 4), b = load_bf16x4(pp + idx * 4);
@@ -159,12 +162,13 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
       *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
     }
   }
-  if (has_ln) layernorm_split_regs(xv, nvec, gw, gb, hi, lo, d, sm);
+  if (has_ln) layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, lo, d, sm);
 }
 
 // x = X[r] + Y[r] + bias for a valid row (Y consumed and cleared for every row); then
 // LayerNorm -> hi/lo for the next GEMM.  grid (rows, groups).  All loads (entry length, Y, X, bias,
 // gamma, beta) are issued together; whether the row is valid only decides what is stored.
+template <int NV>
 __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, EntryList el, float* Y, Ptr2 bias,
                                                                     MPtr2 X, Ptr2 ln_w, Ptr2 ln_b, MPtr2 Ahl,
                                                                     int d, int Rt) {
@@ -179,10 +183,10 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, E
   const uint2* lw = reinterpret_cast<const uint2*>(ln_w.p[g]);
   const uint2* lb = reinterpret_cast<const uint2*>(ln_b.p[g]);
   const int nvec = d / 4;
-  float4 xv[kMaxVec4], yv[kMaxVec4];
-  uint2 bv[kMaxVec4], gw[kMaxVec4], gb[kMaxVec4];
+  float4 xv[NV], yv[NV];
+  uint2 bv[NV], gw[NV], gb[NV];
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
+  for (int v = 0; v < NV; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       yv[v] = *reinterpret_cast<const float4*>(y + idx * 4);
@@ -192,7 +196,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, E
   }
   const bool valid = i < L;
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
+  for (int v = 0; v < NV; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       *reinterpret_cast<float4*>(y + idx * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -206,7 +210,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, E
   }
   if (!valid) return;                             // padding rows stay zero in X and in hi/lo
   bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)r * d;
-  layernorm_split_regs(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
+  layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
 // Last layer: x_i = X[r_i] + Y[r_i] + bias for the entry's valid rows, cache row = mean_i x_i.
@@ -421,6 +425,7 @@ __global__ void __launch_bounds__(1024) k_tc_row_map(CbView cb, EntryList el, in
 }
 
 // X = table[y] + pos for every packed row, then LN1 of layer 0 -> hi/lo.  grid (row capacity).
+template <int NV>
 __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln_packed(CbView cb, EntryList el, const int* total,
                                                                      const bf16* table, const bf16* pos, const bf16* ln_w,
                                                                      const bf16* ln_b, float* X, bf16* Ahl, int d, int Rt,
@@ -435,10 +440,10 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln_packed(CbView cb, 
   const bf16* row = table + (size_t)y * d;
   const bf16* pp = pos + (size_t)i * d;
   const int nvec = d / 4;
-  float4 xv[kMaxVec4];
-  uint2 gw[kMaxVec4], gb[kMaxVec4];
+  float4 xv[NV];
+  uint2 gw[NV], gb[NV];
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
+  for (int v = 0; v < NV; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       const float4 a = load_bf16x4(row + idx * 4), b = load_bf16x4(pp + idx * 4);
@@ -448,30 +453,38 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln_packed(CbView cb, 
       *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
     }
   }
-  if (has_ln) layernorm_split_regs(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
+  if (has_ln) layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
-// Zero-layer encoder on packed rows: cache row = mean of the entry's rows of X.  grid (entries).
+// Mean-pool on packed rows: cache row = mean of the entry's rows of X.  grid (entries,
+// ceil(d / (4 * kRowThreads))): a thread owns 4 columns and loads all rows before it adds.
 __global__ void __launch_bounds__(kRowThreads) k_tc_pool_packed(CbView cb, EntryList el, const float* X, void* cache,
                                                                 float* cache_f32, int d) {
   const int e = blockIdx.x;
+  const int col = ((int)blockIdx.y * kRowThreads + (int)threadIdx.x) * 4;
+  if (col >= d) return;
   const int L = entry_len_tc(cb, el, e);
   if (L <= 0) return;
-  const float* x = X + (size_t)el.row_off[e] * d;
-  const size_t dst = ((size_t)el.seq[e] * cb.cap + el.idx[e]) * d;
+  const float* x = X + (size_t)el.row_off[e] * d + col;
+  float4 v[kMaxM];
+#pragma unroll
+  for (int i = 0; i < kMaxM; ++i)
+    if (i < L) v[i] = *reinterpret_cast<const float4*>(x + (size_t)i * d);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < kMaxM; ++i)
+    if (i < L) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
+  const size_t dst = ((size_t)el.seq[e] * cb.cap + el.idx[e]) * d + col;
   const float inv = 1.0f / (float)L;
-  bf16* out = reinterpret_cast<bf16*>(cache);
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    float v = 0.f;
-    for (int i = 0; i < L; ++i) v += x[(size_t)i * d + c];
-    v *= inv;
-    out[dst + c] = __float2bfloat16_rn(v);
-    if (cache_f32) cache_f32[dst + c] = v;
-  }
+  const float4 m = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+  uint2 o; o.x = pack_bf16(m.x, m.y); o.y = pack_bf16(m.z, m.w);
+  *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(cache) + dst) = o;
+  if (cache_f32) *reinterpret_cast<float4*>(cache_f32 + dst) = m;
 }
 
 // LayerNorm of the packed rows of X -> hi/lo (the GEMM epilogue has already added bias and
 // residual into X).  grid (row capacity), one encoder.
+template <int NV>
 __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, const float* X, const bf16* ln_w,
                                                             const bf16* ln_b, bf16* Ahl, int d, int Rt) {
   __shared__ float sm[32];
@@ -479,10 +492,10 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, co
   if (r >= *total) return;
   const float* x = X + (size_t)r * d;
   const int nvec = d / 4;
-  float4 xv[kMaxVec4];
-  uint2 gw[kMaxVec4], gb[kMaxVec4];
+  float4 xv[NV];
+  uint2 gw[NV], gb[NV];
 #pragma unroll
-  for (int v = 0; v < kMaxVec4; ++v) {
+  for (int v = 0; v < NV; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       xv[v] = *reinterpret_cast<const float4*>(x + idx * 4);
@@ -491,7 +504,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, co
     }
   }
   bf16* hi = Ahl + (size_t)r * d;
-  layernorm_split_regs(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
+  layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
 // Bidirectional attention inside one entry from fp32 q, k, v of its packed rows [rows, 3d] (bias
@@ -631,6 +644,8 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
   const int R = E * M, Rt = (R + 7) / 8 * 8;
   auto Wp = [&](int i) { return reinterpret_cast<const bf16*>(a.w[i]); };
   const int* total = el.row_off + E;                   // packed rows of this pass (device word)
+  const bool narrow = d <= 4 * kRowThreads * kNarrowVec4;      // a row fits four float4 per thread: fewer registers, more CTAs per SM
+  auto lnk = narrow ? k_tc_ln_rows<kNarrowVec4> : k_tc_ln_rows<kMaxVec4>;
   PairGemmParams g{};
   g.cb = cb; g.el = el; g.R = R; g.Rt = Rt; g.live_rows = total; g.err = a.err;
   auto gemm = [&](const bf16* act, int K, int widx, int J, int epi, float* out, bf16* out_hl) -> cudaError_t {
@@ -642,9 +657,9 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
   {
     ProfScope ps(prof, kProfEncOther, 2, s);
     k_tc_row_map<<<1, 1024, 0, s>>>(cb, el, E);
-    k_tc_gather_ln_packed<<<R, kRowThreads, 0, s>>>(cb, el, total, reinterpret_cast<const bf16*>(a.table), Wp(0),
-                                                    a.layers ? Wp(1) : Wp(0), a.layers ? Wp(2) : Wp(0), a.X, a.Ahl, d,
-                                                    Rt, a.layers > 0 ? 1 : 0);
+    auto gk = narrow ? k_tc_gather_ln_packed<kNarrowVec4> : k_tc_gather_ln_packed<kMaxVec4>;
+    gk<<<R, kRowThreads, 0, s>>>(cb, el, total, reinterpret_cast<const bf16*>(a.table), Wp(0), a.layers ? Wp(1) : Wp(0),
+                                 a.layers ? Wp(2) : Wp(0), a.X, a.Ahl, d, Rt, a.layers > 0 ? 1 : 0);
   }
   const int dh = d / a.heads;
   cudaError_t e;
@@ -662,17 +677,18 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
     if ((e = gemm(a.Ahl, d, o + 4, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 6), Wp(o + 7), a.Ahl, d, Rt);
+      lnk<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 6), Wp(o + 7), a.Ahl, d, Rt);
     }
     if ((e = gemm(a.Ahl, d, o + 8, dff, kEpiGelu, nullptr, a.Hhl)) != cudaSuccess) return e;
     if ((e = gemm(a.Hhl, dff, o + 10, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     if (l + 1 < a.layers) {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      k_tc_ln_rows<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 12), Wp(o + 13), a.Ahl, d, Rt);
+      lnk<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 12), Wp(o + 13), a.Ahl, d, Rt);
     }
   }
   ProfScope ps(prof, kProfEncOther, 1, s);
-  k_tc_pool_packed<<<E, kRowThreads, 0, s>>>(cb, el, a.X, a.cache, a.cache_f32, d);
+  k_tc_pool_packed<<<dim3(E, (d / 4 + kRowThreads - 1) / kRowThreads), kRowThreads, 0, s>>>(cb, el, a.X, a.cache,
+                                                                                        a.cache_f32, d);
   return cudaGetLastError();
 }
 
@@ -687,6 +703,8 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   const int row_tiles = (Rt + 127) / 128;
   const bool one_box = row_tiles == 1;                 // hi and lo rows (2 Rt <= 256) are one operand box
   const int n_sm = sm_count();
+  const bool narrow = d <= 4 * kRowThreads * kNarrowVec4;      // a row fits four float4 per thread
+  auto rlk = narrow ? k_tc_reduce_resid_ln<kNarrowVec4> : k_tc_reduce_resid_ln<kMaxVec4>;
   float* Y = a0.part;                                  // GEMM results, all zero between GEMMs
   const size_t wide = (size_t)(3 * d > dff ? 3 * d : dff);
   if ((size_t)ng * Rt * wide * sizeof(float) > a0.part_bytes) return cudaErrorMemoryAllocation;
@@ -731,7 +749,7 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   cudaError_t e;
   {
     ProfScope ps(prof, kProfEncOther, 1, s);
-    launch_pdl(k_tc_gather_ln, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, table, W(0), a0.layers ? W(1) : W(0),
+    launch_pdl(narrow ? k_tc_gather_ln<kNarrowVec4> : k_tc_gather_ln<kMaxVec4>, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, table, W(0), a0.layers ? W(1) : W(0),
                a0.layers ? W(2) : W(0), X, Ahl, d, Rt, a0.layers > 0 ? 1 : 0);
   }
   if (a0.layers == 0) {
@@ -751,7 +769,7 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
     if ((e = gemm(Ahl, d, o + 4, d)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      launch_pdl(k_tc_reduce_resid_ln, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 5), X, W(o + 6),
+      launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 5), X, W(o + 6),
                  W(o + 7), Ahl, d, Rt);
     }
     if ((e = gemm(Ahl, d, o + 8, dff)) != cudaSuccess) return e;
@@ -769,7 +787,7 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
         launch_pdl(k_tc_reduce_resid_pool, dim3(E, ng, (d / 4 + kRowThreads - 1) / kRowThreads), dim3(kRowThreads), 0,
                    s, cb, el, Y, W(o + 11), X, cache, c32, d, Rt);
       else
-        launch_pdl(k_tc_reduce_resid_ln, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 11), X, W(o + 12),
+        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 11), X, W(o + 12),
                    W(o + 13), Ahl, d, Rt);
     }
   }

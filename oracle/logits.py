@@ -101,3 +101,50 @@ def select(l: np.ndarray, mode: int, temperature: float, seed: int, step: int, r
         scores = l / float(temperature) + gumbel(np.arange(l.shape[0]), row, step, seed)
     a, _, gap = top2(scores)
     return a, scores, gap
+
+
+def filter_mask(l: np.ndarray, temperature: float, top_k: int, top_p: float) -> np.ndarray:
+    """Columns that top-k and nucleus (top-p) filtering keep.  Neither is defined by the paper,
+    which only says that a token is sampled from the joint distribution (Section 2.3 step 9);
+    these are the usual definitions, with ties kept together so that the result does not depend
+    on an order among equal logits:
+      top-k: every column whose logit is >= the k-th largest logit (top_k <= 0: no filter);
+      top-p: with columns in descending order of probability softmax(l / T), the shortest prefix
+             whose probabilities sum to >= top_p, extended over ties with its last logit
+             (top_p >= 1: no filter).
+    The result is the intersection; the argmax is always kept."""
+    l = np.asarray(l, dtype=np.float64)
+    n = l.shape[0]
+    keep = np.ones(n, dtype=bool)
+    if 0 < top_k < n:
+        vk = np.sort(l)[::-1][top_k - 1]
+        keep &= l >= vk
+    if top_p < 1.0:
+        order = np.argsort(-l, kind="stable")
+        ls = l[order]
+        pr = np.exp((ls - ls[0]) / float(temperature))
+        cum = np.cumsum(pr) / pr.sum()
+        j = int(np.searchsorted(cum, top_p, side="left"))
+        j = min(j, n - 1)
+        keep &= l >= ls[j]
+    return keep
+
+
+def select_filtered(l: np.ndarray, temperature: float, top_k: int, top_p: float, seed: int, step: int, row: int):
+    """Gumbel-max sample from softmax(l / T) restricted to filter_mask (the noise of a column does
+    not depend on the filter).  Returns (choice, kept mask, gap between the two best kept scores)."""
+    keep = filter_mask(l, temperature, top_k, top_p)
+    scores = np.asarray(l, dtype=np.float64) / float(temperature) + gumbel(np.arange(l.shape[0]), row, step, seed)
+    scores = np.where(keep, scores, -np.inf)
+    a, _, gap = top2(scores)
+    return a, keep, gap
+
+
+def nucleus_margin(l: np.ndarray, temperature: float, top_p: float) -> float:
+    """How far (in probability mass) top_p is from the nearest cumulative sum of the descending
+    probabilities: parity tests skip inputs where fp32 summation could move the boundary."""
+    l = np.asarray(l, dtype=np.float64)
+    ls = np.sort(l)[::-1]
+    pr = np.exp((ls - ls[0]) / float(temperature))
+    cum = np.cumsum(pr) / pr.sum()
+    return float(np.abs(cum - top_p).min())

@@ -107,3 +107,54 @@ def test_session_step_consistency_on_tiny_workload():
             assert s.books[b].n() - n0[b] in (0, 1)               # at most one entry per step
             assert sc[b]["l"].shape[0] == w.V + n0[b]
             assert 0 <= sc[b]["choice"] < w.V + n0[b]
+
+
+# ------------------------------------------------------------------------------------------------
+# top-k / nucleus filtering (not defined by the paper; the usual definitions, ties kept together)
+# ------------------------------------------------------------------------------------------------
+def test_filter_mask_on_a_distribution_with_known_prefix_sums():
+    p = np.array([0.05, 0.5, 0.15, 0.3])                      # descending order: columns 1, 3, 2, 0
+    l = np.log(p)
+    as_set = lambda m: set(np.nonzero(m)[0].tolist())
+    assert as_set(lg.filter_mask(l, 1.0, 0, 0.49)) == {1}     # the first probability alone reaches 0.49
+    assert as_set(lg.filter_mask(l, 1.0, 0, 0.51)) == {1, 3}
+    assert as_set(lg.filter_mask(l, 1.0, 0, 0.79)) == {1, 3}
+    assert as_set(lg.filter_mask(l, 1.0, 0, 0.81)) == {1, 3, 2}
+    assert as_set(lg.filter_mask(l, 1.0, 0, 1.0)) == {0, 1, 2, 3}
+    assert as_set(lg.filter_mask(l, 1.0, 2, 1.0)) == {1, 3}
+    assert as_set(lg.filter_mask(l, 1.0, 3, 0.6)) == {1, 3}   # intersection of the two filters
+    assert as_set(lg.filter_mask(l, 1.0, 1, 0.99)) == {1}
+    # temperature reshapes the probabilities the nucleus is taken on: T = 0.5 squares them
+    q = p ** 2 / (p ** 2).sum()                               # 0.0068, 0.68, 0.061, 0.245
+    assert as_set(lg.filter_mask(l, 0.5, 0, 0.7)) == {1, 3} and q[1] < 0.7 < q[1] + q[3]
+    # ties are kept together
+    lt = np.array([1.0, 3.0, 3.0, 0.0, 3.0])
+    assert as_set(lg.filter_mask(lt, 1.0, 1, 1.0)) == {1, 2, 4}
+    assert as_set(lg.filter_mask(lt, 1.0, 0, 0.1)) == {1, 2, 4}
+
+
+def test_select_filtered_special_cases_reduce_to_argmax_and_to_plain_sampling():
+    rng = np.random.default_rng(8)
+    for t in range(20):
+        l = rng.standard_normal(200) * 2.0
+        a, keep, _ = lg.select_filtered(l, 0.8, 1, 1.0, 77, t, 3)
+        assert a == int(np.argmax(l)) and keep.sum() == 1       # k = 1: the argmax, whatever the noise
+        a2, keep2, _ = lg.select_filtered(l, 0.8, 0, 1.0, 77, t, 3)
+        assert keep2.all() and a2 == lg.select(l, 1, 0.8, 77, t, 3)[0]   # no filter: plain Gumbel-max
+        a3, keep3, _ = lg.select_filtered(l, 0.8, 7, 0.9, 77, t, 3)
+        assert keep3[a3] and keep3[int(np.argmax(l))] and keep3.sum() <= 7
+        pr = np.exp((l - l.max()) / 0.8); pr /= pr.sum()
+        kp = lg.filter_mask(l, 0.8, 0, 0.9)
+        assert pr[kp].sum() >= 0.9 and pr[kp].sum() - pr[kp].min() < 0.9   # the shortest such prefix
+
+
+def test_select_filtered_frequencies_follow_the_renormalised_distribution():
+    l = np.log(np.array([0.4, 0.25, 0.2, 0.1, 0.05]))
+    counts = np.zeros(5)
+    n = 6000
+    for t in range(n):
+        a, keep, _ = lg.select_filtered(l, 1.0, 3, 1.0, 5, t, 0)
+        counts[a] += 1
+    want = np.array([0.4, 0.25, 0.2, 0.0, 0.0]) / 0.85
+    assert counts[3] == 0 and counts[4] == 0
+    assert np.abs(counts / n - want).max() < 0.02

@@ -194,6 +194,22 @@ int32_t z2z_embed_lookup(z2z_codebook* cb, const int32_t* d_codes, int32_t N,
                          const int32_t* d_row_seq, const void* d_WE, const void* d_Eh,
                          void* d_out, z2z_stream stream);
 
+/* Top-k / nucleus (top-p) filtered sampling on stored logits (no counterpart in the paper, which
+ * only says that a token is sampled from the joint distribution: Section 2.3 step 9).  For decode
+ * batches the caller stores the joint logits once (d_logits_debug of z2z_dynamic_logits) and
+ * samples here; the applied code then goes to z2z_lzw_step and z2z_hyper_embed as usual.
+ *   d_logits [N, ld] fp32; d_n_cols [N]: columns of row r that exist (V + visible hypertokens);
+ *   top_k <= 0: no top-k filter, else every column whose logit is >= the k-th largest is kept;
+ *   top_p >= 1: no nucleus filter, else with the columns in descending order of
+ *            softmax(l / temperature) the shortest prefix with probability >= top_p is kept,
+ *            extended over ties with its last logit; the two filters intersect;
+ *   the sample is the Gumbel-max over the kept columns with the noise of the fused sampler
+ *            (seed, step; the row number in the counter is row_base + r);
+ *   d_choice [N] out (-1 for a row without columns); d_kept [N] out or NULL: columns kept.     */
+int32_t z2z_sample_filtered(const float* d_logits, int32_t N, int64_t ld, const int32_t* d_n_cols,
+                            int32_t top_k, float top_p, float temperature, uint64_t seed, uint64_t step,
+                            int32_t row_base, int32_t* d_choice, int32_t* d_kept, z2z_stream stream);
+
 /* Host -> device transfer of a small per-step input (the hidden rows of a decode step) by a kernel
  * instead of a copy-engine transfer (no counterpart in the paper; end-to-end latency aid).  The
  * kernel that follows on the stream may start its independent part - z2z_decode_step's logits

@@ -26,7 +26,7 @@ EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lz
            "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
            "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error", "z2z_profile",
            "z2z_profile_read", "z2z_set_tensor_cores", "z2z_logits_static_scratch",
-           "z2z_lzw_decode", "z2z_embed_lookup", "z2z_upload_rows"]
+           "z2z_lzw_decode", "z2z_embed_lookup", "z2z_upload_rows", "z2z_sample_filtered"]
 
 
 class Config(C.Structure):
@@ -195,6 +195,17 @@ def z2z_embed_lookup(cb: Codebook, codes: torch.Tensor, row_seq: Optional[torch.
     """codes [N] int32 -> out [N, d]: W_E rows for base tokens, cached E_h rows for hypertokens."""
     _check(lib().z2z_embed_lookup(cb.handle, _ptr(codes), C.c_int32(codes.numel()), _ptr(row_seq),
                                   _ptr(W_E), _ptr(E_h), _ptr(out), _stream()))
+
+
+def z2z_sample_filtered(logits: torch.Tensor, n_cols: torch.Tensor, top_k: int, top_p: float, temperature: float,
+                        seed: int, step: int, choice: torch.Tensor, kept: Optional[torch.Tensor] = None,
+                        row_base: int = 0):
+    """logits [N, ld] fp32 (device), n_cols [N] int32 -> choice [N] int32 (and kept [N] int32)."""
+    assert logits.dtype == torch.float32 and logits.dim() == 2
+    _check(lib().z2z_sample_filtered(_ptr(logits), C.c_int32(logits.shape[0]), C.c_int64(logits.stride(0)),
+                                     _ptr(n_cols), C.c_int32(top_k), C.c_float(top_p), C.c_float(temperature),
+                                     C.c_uint64(seed), C.c_uint64(step), C.c_int32(row_base), _ptr(choice), _ptr(kept),
+                                     _stream()))
 
 
 def z2z_upload_rows(src_pinned: torch.Tensor, dst: torch.Tensor):

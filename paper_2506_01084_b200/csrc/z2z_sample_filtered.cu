@@ -1,0 +1,201 @@
+// Top-k / nucleus (top-p) filtered sampling on stored logits (beyond the paper, which only says
+// that a token is sampled from the joint distribution over base tokens and hypertokens:
+// Section 2.3 step 9).  For decode batches the joint logits of all rows are a few megabytes, so
+// they can be stored once (z2z_dynamic_logits with its full-logit output) and filtered here; the
+// fused argmax / Gumbel-max path of the logits kernels needs no stored logits.
+//
+// One CTA per row, every pass reads the row from L2:
+//   1. m = max l,  Z = sum exp((l - m) / T);
+//   2. top-k: radix select (4 passes of 8 bits over order-preserving keys of the logits) of the
+//      k-th largest logit; everything >= it is kept (ties stay together);
+//   3. top-p: the same descent weighted by probability mass: the largest logit v with
+//      mass{l >= v} >= p Z; everything >= v is kept;
+//   4. Gumbel-max over the kept columns with the noise the fused sampler uses
+//      (Philox4x32-10 keyed by the seed, counter (column / 4, row, step), word column % 4).
+// The thresholds are found on the logits themselves, not on l / T: a positive scale preserves the
+// order, and equal logits stay exactly equal.
+#include "z2z_common.cuh"
+#include "z2z_internal.h"
+
+namespace z2z {
+
+namespace {
+
+constexpr int kSfThreads = 1024;
+
+__device__ __forceinline__ uint32_t order_key(float x) {          // larger float <-> larger key
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+struct SfShared {
+  float red_f[32];
+  int red_i[32];
+  unsigned int hist[256];
+  float mass[256];
+  float m, Z;
+  unsigned int prefix;
+  unsigned int k_left;
+  float p_left;
+};
+
+__device__ __forceinline__ float block_max(float v, SfShared* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sh->red_f[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = sh->red_f[threadIdx.x & 31];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, o));
+  return t;
+}
+__device__ __forceinline__ float block_sum_f(float v, SfShared* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sh->red_f[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = sh->red_f[threadIdx.x & 31];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  return t;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __restrict__ logits, long long ld,
+                                                                const int32_t* __restrict__ n_cols, int top_k,
+                                                                float top_p, float inv_t, uint32_t k0, uint32_t k1,
+                                                                uint32_t c2, uint32_t c3, int row_base,
+                                                                int32_t* __restrict__ choice, int32_t* __restrict__ kept) {
+  __shared__ SfShared sh;
+  const int r = blockIdx.x, tid = threadIdx.x;
+  const int C = n_cols[r];
+  const float* l = logits + (size_t)r * ld;
+  if (C <= 0) { if (tid == 0) { choice[r] = -1; if (kept) kept[r] = 0; } return; }
+  // ---- 1. max and partition sum
+  float mx = -INFINITY;
+  for (int c = tid; c < C; c += kSfThreads) mx = fmaxf(mx, l[c]);
+  mx = block_max(mx, &sh);
+  float z = 0.f;
+  for (int c = tid; c < C; c += kSfThreads) z += expf((l[c] - mx) * inv_t);
+  z = block_sum_f(z, &sh);
+  unsigned int key_k = 0u, key_p = 0u;
+  // ---- 2. k-th largest logit by radix descent on counts
+  if (top_k > 0 && top_k < C) {
+    if (tid == 0) { sh.prefix = 0u; sh.k_left = (unsigned)top_k; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) sh.hist[tid] = 0u;
+      __syncthreads();
+      const unsigned int prefix = sh.prefix;
+      for (int c = tid; c < C; c += kSfThreads) {
+        const uint32_t k = order_key(l[c]);
+        if (pass == 0 || (k >> (shift + 8)) == prefix) atomicAdd(&sh.hist[(k >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        unsigned int left = sh.k_left, d = 255u;
+        for (;; --d) {                                  // from the largest digit down
+          const unsigned int h = sh.hist[d];
+          if (h >= left || d == 0u) break;
+          left -= h;
+        }
+        sh.k_left = left;
+        sh.prefix = (prefix << 8) | d;
+      }
+      __syncthreads();
+    }
+    key_k = sh.prefix;
+  }
+  // ---- 3. nucleus threshold by radix descent on probability mass
+  if (top_p < 1.0f) {
+    __syncthreads();
+    if (tid == 0) { sh.prefix = 0u; sh.p_left = top_p * z; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) { sh.mass[tid] = 0.f; sh.hist[tid] = 0u; }
+      __syncthreads();
+      const unsigned int prefix = sh.prefix;
+      for (int c = tid; c < C; c += kSfThreads) {
+        const float x = l[c];
+        const uint32_t k = order_key(x);
+        if (pass == 0 || (k >> (shift + 8)) == prefix) {
+          atomicAdd(&sh.mass[(k >> shift) & 255u], expf((x - mx) * inv_t));
+          atomicAdd(&sh.hist[(k >> shift) & 255u], 1u);
+        }
+      }
+      __syncthreads();
+      if (tid == 0) {
+        float left = sh.p_left;
+        unsigned int d = 255u, last = 0u;
+        bool found = false;
+        for (int dd = 255; dd >= 0; --dd) {
+          if (sh.hist[dd] == 0u) continue;
+          last = (unsigned)dd;                            // the smallest occupied digit seen so far
+          if (sh.mass[dd] >= left) { d = (unsigned)dd; found = true; break; }
+          left -= sh.mass[dd];
+        }
+        if (!found) d = last;                             // rounding: the mass ran out; keep everything here
+        sh.p_left = left;
+        sh.prefix = (prefix << 8) | d;
+      }
+      __syncthreads();
+    }
+    key_p = sh.prefix;
+  }
+  const unsigned int key_t = key_k > key_p ? key_k : key_p;
+  // ---- 4. Gumbel-max over the kept columns (lowest index on ties)
+  float best = -INFINITY;
+  int best_c = 0x7fffffff, n_kept = 0;
+  for (int c = tid; c < C; c += kSfThreads) {
+    const float x = l[c];
+    if (order_key(x) < key_t) continue;
+    ++n_kept;
+    const Philox4 px = philox4x32_10((uint32_t)(c >> 2), (uint32_t)(row_base + r), c2, c3, k0, k1);
+    const float s = fmaf(x, inv_t, gumbel_from_word(philox_word(px, c & 3)));
+    if (s > best || (s == best && c < best_c)) { best = s; best_c = c; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+    n_kept += __shfl_xor_sync(0xffffffffu, n_kept, o);
+    if (ob > best || (ob == best && oc < best_c)) { best = ob; best_c = oc; }
+  }
+  __syncthreads();
+  if ((tid & 31) == 0) { sh.red_f[tid >> 5] = best; sh.red_i[tid >> 5] = best_c; sh.hist[tid >> 5] = (unsigned)n_kept; }
+  __syncthreads();
+  if (tid < 32) {
+    best = sh.red_f[tid]; best_c = sh.red_i[tid]; n_kept = (int)sh.hist[tid];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oc = __shfl_xor_sync(0xffffffffu, best_c, o);
+      n_kept += __shfl_xor_sync(0xffffffffu, n_kept, o);
+      if (ob > best || (ob == best && oc < best_c)) { best = ob; best_c = oc; }
+    }
+    if (tid == 0) { choice[r] = best_c == 0x7fffffff ? -1 : best_c; if (kept) kept[r] = n_kept; }
+  }
+}
+
+}  // namespace z2z
+
+extern "C" int32_t z2z_sample_filtered(const float* d_logits, int32_t N, int64_t ld, const int32_t* d_n_cols,
+                                       int32_t top_k, float top_p, float temperature, uint64_t seed, uint64_t step,
+                                       int32_t row_base, int32_t* d_choice, int32_t* d_kept, z2z_stream stream) {
+  auto fail = [](const char* msg) { z2z::set_last_error(msg); return (int32_t)Z2Z_ERR_INVALID_ARG; };
+  if (N < 0) return fail("N < 0");
+  if (N == 0) return Z2Z_OK;
+  if (!d_logits || !d_n_cols || !d_choice) return fail("d_logits / d_n_cols / d_choice is NULL");
+  if (!(temperature > 0.f)) return fail("sampling needs temperature > 0");
+  if (!(top_p > 0.f)) return fail("top_p must be > 0 (>= 1: no nucleus filter)");
+  if (ld < 1) return fail("ld < 1");
+  z2z::k_sample_filtered<<<N, z2z::kSfThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      d_logits, (long long)ld, d_n_cols, top_k, top_p, 1.0f / temperature, (uint32_t)seed, (uint32_t)(seed >> 32),
+      (uint32_t)step, (uint32_t)(step >> 32), row_base, d_choice, d_kept);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { z2z::set_last_error(cudaGetErrorString(e)); return Z2Z_ERR_CUDA; }
+  return Z2Z_OK;
+}

@@ -46,4 +46,6 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.z2z_embed_lookup(None, None, 0, None, None, None, None, None) == -1
     assert lib.z2z_upload_rows(None, None, ctypes.c_size_t(16), None) == -1
     assert lib.z2z_upload_rows(None, None, ctypes.c_size_t(0), None) == 0
+    assert lib.z2z_sample_filtered(None, 4, ctypes.c_int64(8), None, 0, ctypes.c_float(1.0), ctypes.c_float(1.0),
+                                   ctypes.c_uint64(0), ctypes.c_uint64(0), 0, None, None, None) == -1
     assert lib.z2z_codebook_destroy(None) == 0

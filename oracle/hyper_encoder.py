@@ -14,12 +14,17 @@ textbook pre-LayerNorm encoder layer (the reading is listed in the design notes)
         X = X + W2 gelu(W1 LN2(X) + b1) + b2             (erf GELU; LayerNorm eps 1e-5)
     h = mean_i X_i                                       over the L valid positions
 
+A layer whose feed-forward width is zero (W1 has no rows) is the attention sublayer alone: with one
+such layer this is the "1-attention-layer" variant of the appendix's architecture ablation (read
+as the first sublayer of the same pre-LN layer, residual included; the paper gives no detail).
+
 Padding positions are never used as keys and never pooled, so their values cannot matter and are
 not computed.  Everything is numpy fp64 on the exact values of the (bf16 or fp32) inputs.
 
 Pins: tests/test_oracle_encoder.py (zero layers == plain mean of the gathered rows; one and two
 layers against torch.nn.TransformerEncoderLayer(norm_first=True) with a key-padding mask;
-permutation sensitivity through ``pos``).  The absolute values under the paper's *trained*
+permutation sensitivity through ``pos``; attention-only layers against
+torch.nn.MultiheadAttention on LayerNorm'd rows, and == plain mean when Wo and bo are zero).  The absolute values under the paper's *trained*
 encoder are "parity unpinned": no weights exist offline.
 """
 from __future__ import annotations
@@ -71,6 +76,8 @@ def hyper_embed_one(constituents: Sequence[int], table: np.ndarray, enc: List[np
             P = P / P.sum(axis=1, keepdims=True)
             O[:, s] = P @ Vv[:, s]
         X = X + O @ Wo.T + bo
+        if W1.shape[0] == 0:                                      # attention-only layer
+            continue
         Hh = _gelu(_layer_norm(X, ln2_w, ln2_b) @ W1.T + b1)
         X = X + Hh @ W2.T + b2
     return X.mean(axis=0)
@@ -112,6 +119,8 @@ def hyper_embed(entries: Sequence[Sequence[int]], table: np.ndarray, enc: List[n
                 P = P / P.sum(axis=1, keepdims=True)
                 O[r, s] = P @ qkv[r, 2 * d + h * dh: 2 * d + (h + 1) * dh]
         X = X + O @ Wo.T + bo
+        if W1.shape[0] == 0:                                      # attention-only layer
+            continue
         X = X + _gelu(_layer_norm(X, ln2_w, ln2_b) @ W1.T + b1) @ W2.T + b2
     out = np.empty((len(entries), d), dtype=np.float64)
     for e in range(len(entries)):

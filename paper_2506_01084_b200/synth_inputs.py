@@ -40,6 +40,7 @@ class Workload:
     enc_heads: int = 0        # 0 -> d // 128 (tiny: 4)
     enc_dff: int = 0          # 0 -> 4 * d
     tied: int = 0
+    enc_ffn: int = 1          # 0: attention-only layers (feed-forward width 0; architecture ablation)
 
     @property
     def heads(self) -> int:
@@ -49,6 +50,8 @@ class Workload:
 
     @property
     def dff(self) -> int:
+        if not self.enc_ffn:
+            return 0
         return self.enc_dff if self.enc_dff else 4 * self.d
 
     @property

@@ -7,10 +7,10 @@ from oracle import hyper_encoder as he
 from paper_2506_01084_b200 import synth_inputs as si
 
 
-def _setup(layers, d=32, M=4, V=50, heads=4, seed=3, generic=True):
+def _setup(layers, d=32, M=4, V=50, heads=4, seed=3, generic=True, ffn=1):
     w = si.Workload("t", V=V, d=d, dtype="fp32", B=1, T=8, M=M, cap=8, zipf_s=1.0, copy_p=0.0,
                     seg_min=1, seg_max=1, steps=0, enc_layers=layers, enc_heads=heads,
-                    enc_dff=3 * d)
+                    enc_dff=3 * d, enc_ffn=ffn)
     enc = [t.double().numpy() for t in si.make_encoder(w, seed, generic=generic)]
     W, _ = si.make_tables(w, seed)
     return w, enc, W.double().numpy()
@@ -70,6 +70,50 @@ def test_against_library_encoder_layer(layers):
     many = he.hyper_embed(entries, W, enc, w.heads)
     for i, e in enumerate(entries):
         np.testing.assert_allclose(many[i], he.hyper_embed_one(e, W, enc, w.heads), atol=1e-13)
+
+
+@pytest.mark.parametrize("layers", [1, 2])
+def test_attention_only_layers_against_library_attention(layers):
+    # the "1-attention-layer" variant of the architecture ablation, read as the attention
+    # sublayer of the same pre-LN layer: X + MHA(LN1(X)), with the installed PyTorch's
+    # multi-head attention (fp64, same weights, key-padding mask) as the library routine
+    w, enc, W = _setup(layers, ffn=0)
+    d, M = w.d, w.M
+    assert enc[1 + 8].shape == (0, d) and enc[1 + 10].shape == (d, 0)
+    entries = [(3, 7), (1, 2, 3), (9, 9, 9, 4), (4, 9, 9, 9)]
+    for e in entries:
+        L = len(e)
+        x = torch.zeros(1, M, d, dtype=torch.float64)
+        x[0, :L] = torch.from_numpy(W[list(e)] + enc[0][:L])
+        x[0, L:] = -77.0
+        mask = torch.zeros(1, M, dtype=torch.bool)
+        mask[0, L:] = True
+        for l in range(layers):
+            t = [torch.from_numpy(a) for a in enc[1 + 12 * l: 13 + 12 * l]]
+            mha = torch.nn.MultiheadAttention(d, w.heads, dropout=0.0, batch_first=True, dtype=torch.float64)
+            with torch.no_grad():
+                mha.in_proj_weight.copy_(t[2]); mha.in_proj_bias.copy_(t[3])
+                mha.out_proj.weight.copy_(t[4]); mha.out_proj.bias.copy_(t[5])
+                a = torch.nn.functional.layer_norm(x, (d,), t[0], t[1], 1e-5)
+                x = x + mha(a, a, a, key_padding_mask=mask, need_weights=False)[0]
+        want = x[0, :L].mean(dim=0).numpy()
+        np.testing.assert_allclose(he.hyper_embed_one(e, W, enc, w.heads), want, rtol=0, atol=1e-12)
+    many = he.hyper_embed(entries, W, enc, w.heads)
+    for i, e in enumerate(entries):
+        np.testing.assert_allclose(many[i], he.hyper_embed_one(e, W, enc, w.heads), atol=1e-13)
+    # it is not the full layer: the feed-forward block changes the result
+    wf, encf, Wf = _setup(layers, ffn=1)
+    assert np.abs(he.hyper_embed_one((1, 2, 3), Wf, encf, w.heads) - many[1]).max() > 1e-4
+
+
+def test_attention_only_with_zero_output_projection_is_the_mean():
+    # Wo = 0, bo = 0: the sublayer adds nothing, so the result is the averaging variant
+    w, enc, W = _setup(2, ffn=0)
+    for l in range(2):
+        enc[1 + 12 * l + 4][:] = 0.0
+        enc[1 + 12 * l + 5][:] = 0.0
+    got = he.hyper_embed_one((5, 6, 7), W, enc, w.heads)
+    np.testing.assert_allclose(got, (W[[5, 6, 7]] + enc[0][:3]).mean(axis=0), atol=1e-15)
 
 
 def test_order_matters_and_padding_is_inert():

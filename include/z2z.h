@@ -64,7 +64,8 @@ typedef struct {
   int32_t dtype;        /* Z2Z_DTYPE_*: tables, encoder tensors, hidden states, caches */
   int32_t enc_layers;   /* hyper-encoder layers; 0 = the parameter-free averaging variant */
   int32_t enc_heads;    /* attention heads (d % enc_heads == 0)                     */
-  int32_t enc_dff;      /* feed-forward width                                       */
+  int32_t enc_dff;      /* feed-forward width; 0 = attention-only layers (no feed-forward block:
+                           the 1-attention-layer variant of the architecture ablation) */
   int32_t tied;         /* 1: the caller passes the same cache for both sides       */
 } z2z_config;
 
@@ -72,7 +73,8 @@ typedef struct {
  * configured dtype, as a HOST array of DEVICE pointers in this order:
  *   pos[M,d], then for each layer:
  *   ln1_w[d] ln1_b[d] Wqkv[3d,d] bqkv[3d] Wo[d,d] bo[d] ln2_w[d] ln2_b[d] W1[dff,d] b1[dff] W2[d,dff] b2[d]
- * n_tensors must be 1 + 12 * enc_layers.                                                      */
+ * n_tensors must be 1 + 12 * enc_layers.  With enc_dff == 0 the six feed-forward slots of a
+ * layer (ln2_w .. b2) are ignored and may be NULL.                                                      */
 typedef struct {
   const void* const* tensors;
   int32_t n_tensors;

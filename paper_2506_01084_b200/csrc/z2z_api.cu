@@ -51,7 +51,8 @@ int check_config(const z2z_config* c) {
   if (c->enc_layers < 0 || c->enc_layers > 16) return fail(Z2Z_ERR_INVALID_ARG, "need 0 <= enc_layers <= 16");
   if (c->enc_layers > 0) {
     if (c->enc_heads < 1 || c->d % c->enc_heads != 0) return fail(Z2Z_ERR_INVALID_ARG, "d must be a multiple of enc_heads");
-    if (c->enc_dff < 8 || c->enc_dff % 8 != 0) return fail(Z2Z_ERR_INVALID_ARG, "need enc_dff >= 8, enc_dff % 8 == 0");
+    if (c->enc_dff != 0 && (c->enc_dff < 8 || c->enc_dff % 8 != 0))
+      return fail(Z2Z_ERR_INVALID_ARG, "need enc_dff >= 8 and enc_dff % 8 == 0, or enc_dff == 0 (attention-only layers)");
   }
   return Z2Z_OK;
 }
@@ -97,8 +98,11 @@ z2z::EncoderArgs encoder_args(z2z_codebook* cb, const void* table, const z2z_enc
 int check_encoder(z2z_codebook* cb, const z2z_encoder_weights* enc) {
   if (!enc || !enc->tensors) return fail(Z2Z_ERR_INVALID_ARG, "encoder weights are NULL");
   if (enc->n_tensors != 1 + 12 * cb->cfg.enc_layers) return fail(Z2Z_ERR_INVALID_ARG, "n_tensors must be 1 + 12 * enc_layers");
-  for (int i = 0; i < enc->n_tensors; ++i)
-    if (!enc->tensors[i]) return fail(Z2Z_ERR_INVALID_ARG, "an encoder tensor is NULL");
+  for (int i = 0; i < enc->n_tensors; ++i) {
+    // attention-only layers ignore the six feed-forward slots (ln2_w .. b2), which may be NULL
+    const bool unused = cb->dff == 0 && i >= 1 && (i - 1) % 12 >= 6;
+    if (!enc->tensors[i] && !unused) return fail(Z2Z_ERR_INVALID_ARG, "an encoder tensor is NULL");
+  }
   return Z2Z_OK;
 }
 

@@ -114,7 +114,7 @@ inline WsPlan plan_workspace(const z2z_config& c) {
   p.off_new_entry = take((size_t)c.B * 4);
   p.off_sel = take((size_t)c.B * 4 * 4);
   size_t R = (size_t)p.enc_rows;
-  size_t dff = (size_t)(c.enc_dff > 0 ? c.enc_dff : 4 * c.d);
+  size_t dff = (size_t)(c.enc_dff > 0 ? c.enc_dff : 0);
   size_t wide = dff > (size_t)3 * c.d ? dff : (size_t)3 * c.d;
   // encoder scratch: one full set for prefill passes (group 0) and a decode-sized set (B entries)
   // for the second encoder of the decode step (group 1)

@@ -322,6 +322,7 @@ static cudaError_t encoder_pass_simt(const CbView& cb, const EncoderArgs& a, con
         k_enc_linear<T, 2><<<dim3((d + kTJ - 1) / kTJ, rt), blk, 0, s>>>(a.A, d, W(o + 4), d, W(o + 5),
                                                                       a.X, R, n_live, M);
       }
+      if (dff == 0) continue;                          // attention-only layer
 { ProfScope ps(prof, kProfEncOther, 1, s);
         k_enc_layernorm<T><<<R, 256, 0, s>>>(cb, el, a.X, W(o + 6), W(o + 7), a.A, d);
       }

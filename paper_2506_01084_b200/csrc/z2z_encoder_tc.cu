@@ -675,12 +675,14 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
                                                                                            a.heads, Rt);
     }
     if ((e = gemm(a.Ahl, d, o + 4, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
-    {
-      ProfScope ps(prof, kProfEncOther, 1, s);
-      lnk<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 6), Wp(o + 7), a.Ahl, d, Rt);
+    if (dff > 0) {                                     // dff == 0: attention-only layer
+      {
+        ProfScope ps(prof, kProfEncOther, 1, s);
+        lnk<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 6), Wp(o + 7), a.Ahl, d, Rt);
+      }
+      if ((e = gemm(a.Ahl, d, o + 8, dff, kEpiGelu, nullptr, a.Hhl)) != cudaSuccess) return e;
+      if ((e = gemm(a.Hhl, dff, o + 10, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     }
-    if ((e = gemm(a.Ahl, d, o + 8, dff, kEpiGelu, nullptr, a.Hhl)) != cudaSuccess) return e;
-    if ((e = gemm(a.Hhl, dff, o + 10, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     if (l + 1 < a.layers) {
       ProfScope ps(prof, kProfEncOther, 1, s);
       lnk<<<R, kRowThreads, 0, s>>>(total, a.X, Wp(o + 12), Wp(o + 13), a.Ahl, d, Rt);
@@ -767,27 +769,31 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
                  W(o + 3), Ahl, d, a0.heads, Rt);
     }
     if ((e = gemm(Ahl, d, o + 4, d)) != cudaSuccess) return e;
-    {
-      ProfScope ps(prof, kProfEncOther, 1, s);
-      launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 5), X, W(o + 6),
-                 W(o + 7), Ahl, d, Rt);
+    int last_bias = o + 5;                             // bias of the layer's last linear map
+    if (dff > 0) {                                     // dff == 0: attention-only layer
+      {
+        ProfScope ps(prof, kProfEncOther, 1, s);
+        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 5), X, W(o + 6),
+                   W(o + 7), Ahl, d, Rt);
+      }
+      if ((e = gemm(Ahl, d, o + 8, dff)) != cudaSuccess) return e;
+      {
+        ProfScope ps(prof, kProfEncOther, 1, s);
+        const long long f4 = (long long)ng * R * (dff / 4);
+        const int per_cta = kGeluThreads * kGeluPerThread;
+        launch_pdl(k_tc_reduce_gelu, dim3((unsigned)((f4 + per_cta - 1) / per_cta)), dim3(kGeluThreads), 0, s, cb, el, Y,
+                   W(o + 9), Hhl, dff, R, Rt, ng);
+      }
+      if ((e = gemm(Hhl, dff, o + 10, d)) != cudaSuccess) return e;
+      last_bias = o + 11;
     }
-    if ((e = gemm(Ahl, d, o + 8, dff)) != cudaSuccess) return e;
-    {
-      ProfScope ps(prof, kProfEncOther, 1, s);
-      const long long f4 = (long long)ng * R * (dff / 4);
-      const int per_cta = kGeluThreads * kGeluPerThread;
-      launch_pdl(k_tc_reduce_gelu, dim3((unsigned)((f4 + per_cta - 1) / per_cta)), dim3(kGeluThreads), 0, s, cb, el, Y,
-                 W(o + 9), Hhl, dff, R, Rt, ng);
-    }
-    if ((e = gemm(Hhl, dff, o + 10, d)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
       if (last)
         launch_pdl(k_tc_reduce_resid_pool, dim3(E, ng, (d / 4 + kRowThreads - 1) / kRowThreads), dim3(kRowThreads), 0,
-                   s, cb, el, Y, W(o + 11), X, cache, c32, d, Rt);
+                   s, cb, el, Y, W(last_bias), X, cache, c32, d, Rt);
       else
-        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 11), X, W(o + 12),
+        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(last_bias), X, W(o + 12),
                    W(o + 13), Ahl, d, Rt);
     }
   }

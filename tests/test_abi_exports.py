@@ -40,6 +40,12 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.z2z_workspace_bytes(ctypes.byref(bad), ctypes.byref(out)) == -1
     ok = zb.make_config(512, 64, 3, 256, 1, "fp32", 2, 4, 256)
     assert lib.z2z_workspace_bytes(ctypes.byref(ok), ctypes.byref(out)) == 0 and out.value > 0
+    full = out.value
+    # feed-forward width 0 = attention-only layers: accepted, and needs less scratch; 4 is no width
+    ok = zb.make_config(512, 64, 3, 256, 1, "fp32", 2, 4, 0)
+    assert lib.z2z_workspace_bytes(ctypes.byref(ok), ctypes.byref(out)) == 0 and 0 < out.value < full
+    bad = zb.make_config(512, 64, 3, 256, 1, "fp32", 2, 4, 4)
+    assert lib.z2z_workspace_bytes(ctypes.byref(bad), ctypes.byref(out)) == -1
     # a NULL handle is rejected, not dereferenced
     assert lib.z2z_lzw_step(None, None, None, None, None) == -1
     assert lib.z2z_lzw_decode(None, None, None, 0, 0, None, None, 0, None) == -1

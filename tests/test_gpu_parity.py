@@ -188,6 +188,8 @@ def _prefill_both(p: Pair):
 @pytest.mark.parametrize("w", [si.WORKLOADS["tiny"], SMALL_BF16, SMALL_FP32,
                                SMALL_BF16.scaled(name="avg", enc_layers=0),
                                SMALL_BF16.scaled(name="one_layer", enc_layers=1),
+                               SMALL_BF16.scaled(name="attn_only", enc_layers=1, enc_ffn=0),
+                               SMALL_FP32.scaled(name="attn_only_fp32", enc_layers=2, enc_ffn=0),
                                SMALL_BF16.scaled(name="tied", tied=1)],
                          ids=lambda w: w.name)
 def test_hyper_embed_all_prefill_entries(w):
@@ -440,7 +442,9 @@ def test_decode_step_tiny_config_sampling_and_forcing():
     _decode_follow(si.WORKLOADS["tiny"], 22, zb.SELECT_GUMBEL, forced_every=3)
 
 
-@pytest.mark.parametrize("w", [SMALL_BF16, SMALL_FP32, SMALL_BF16.scaled(name="tied", tied=1)],
+@pytest.mark.parametrize("w", [SMALL_BF16, SMALL_FP32, SMALL_BF16.scaled(name="tied", tied=1),
+                               SMALL_BF16.scaled(name="attn_only", enc_layers=1, enc_ffn=0),
+                               SMALL_BF16.scaled(name="attn_only_2", enc_layers=2, enc_ffn=0)],
                          ids=lambda w: w.name)
 def test_decode_step_small(w):
     _decode_follow(w, 23, zb.SELECT_ARGMAX, steps=w.steps)
@@ -511,6 +515,26 @@ def test_prompt_sized_pass_with_long_entries_and_wide_heads(w):
     # registers of one warp: merge size 5, or heads of 256 columns
     assert w.B * w.cap * w.M >= 1024
     p = Pair(w, seed=45)
+    _, worst = _prefill_both(p)
+    assert worst <= TOL
+    print(f"{w.name}: max |hyper-embedding error| = {worst:.3e}")
+
+
+def test_attention_only_layers_on_every_encoder_path():
+    # layers without a feed-forward block (enc_dff = 0): the CUDA-core kernels on a bf16 session,
+    # the weight-streaming GEMM with several row tiles, and a prompt-sized pass (CTA-pair GEMMs)
+    w = SMALL_BF16.scaled(name="attn_only_2", enc_layers=2, enc_ffn=0)
+    assert w.dff == 0
+    p = Pair(w, seed=5, tensor_cores=False)
+    _, worst = _prefill_both(p)
+    assert worst <= TOL
+    w = ROWS_BF16.scaled(name="rows_attn_only", enc_ffn=0)
+    p = Pair(w, seed=35)
+    _, worst = _prefill_both(p)
+    assert worst <= TOL
+    w = SMALL_BF16.scaled(name="pair_attn_only", enc_layers=2, enc_ffn=0, B=2, cap=300, T=1100)
+    assert w.B * w.cap * w.M >= 1024
+    p = Pair(w, seed=46)
     _, worst = _prefill_both(p)
     assert worst <= TOL
     print(f"{w.name}: max |hyper-embedding error| = {worst:.3e}")

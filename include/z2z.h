@@ -16,7 +16,10 @@
  *     buffer; the library allocates no device memory.  The opaque handle is host memory that
  *     stores the configuration and offsets into the caller's workspace.
  *   - All work is enqueued on the given stream and returns without synchronising (except
- *     z2z_status, which waits for the stream).
+ *     z2z_status, which waits for the stream).  The enqueueing calls may therefore be captured
+ *     into a CUDA graph (arguments passed by value, the sampling step among them, are then fixed
+ *     for every replay); capture again after z2z_codebook_init starts a new session, because
+ *     z2z_decode_step decides on the host whether the session still needs its hyper-encoder pass.
  *   - Ids are int32.  Tables are row-major [rows, d] in the configured dtype.
  *   - Hypertoken id = V + k where k is the creation order within the sequence.
  *   - Limits: V + cap < 2^24 - 1, cap <= 65535, 1 <= M <= 8, d % 8 == 0, B <= 1024.

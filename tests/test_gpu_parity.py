@@ -438,6 +438,53 @@ def test_decode_step_results_written_to_pinned_host_memory():
         _decode_follow(w, 27, sel, steps=6, forced_every=3, host_results=True)
 
 
+def test_decode_steps_replayed_from_a_cuda_graph():
+    # the step only enqueues work on the caller's stream, so a caller may capture it: six steps
+    # captured once and replayed give the session that six plain calls give (plain calls are the
+    # ones held against the oracle above); floating-point results agree to summation order
+    w, steps = SMALL_BF16, 6
+    hid = si.make_hidden(w, (steps + 1) * w.B, 78).view(steps + 1, w.B, w.d).to(DEV)
+    out = []
+    for mode in ("plain", "graph"):
+        p = Pair(w, seed=77)
+        p.gpu_encode()
+        total = w.B * w.cap
+        zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, total, p.E_h, None)
+        zb.z2z_hyper_embed(p.cb, zb.CACHE_UNEMBED, p.g_WU, p.g_encU, None, None, total, p.U_h, None)
+        nxt = torch.zeros(steps + 1, w.B, dtype=torch.int32, device=DEV)
+        new = torch.zeros(steps + 1, w.B, dtype=torch.int32, device=DEV)
+        lse = torch.zeros(steps + 1, w.B, dtype=torch.float32, device=DEV)
+
+        def step(t):
+            zb.z2z_decode_step(p.cb, hid[t], p.g_WE, p.g_WU, p.g_encE, p.g_encU, p.E_h, p.U_h,
+                               zb.SELECT_GUMBEL, 0.9, 4242, t, None, nxt[t], None, lse[t], new[t])
+        step(0)                                  # every kernel has run once before the capture
+        torch.cuda.synchronize()
+        if mode == "plain":
+            for t in range(1, steps + 1):
+                step(t)
+        else:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for t in range(1, steps + 1):
+                    step(t)
+            torch.cuda.synchronize()
+            assert int(nxt[1:].abs().sum().item()) == 0          # capturing ran nothing
+            g.replay()
+        torch.cuda.synchronize()
+        st, n = zb.z2z_status(p.cb)
+        books = [p.gpu_codebook(b)[0] for b in range(w.B)]
+        out.append((nxt.cpu(), new.cpu(), lse.cpu(), n.tolist(), st.tolist(), books, p.E_h.float().cpu(),
+                    p.U_h.float().cpu()))
+    a, b = out
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    assert a[3] == b[3] and a[4] == b[4] == [0] * w.B and a[5] == b[5]
+    assert int((a[1][1:] >= 0).sum()) > 0                        # the replayed steps created entries
+    assert float((a[2] - b[2]).abs().max()) <= 1e-3
+    for x, y in ((a[6], b[6]), (a[7], b[7])):
+        assert float((x - y).abs().max()) <= 2.0 ** -6 * max(1.0, float(x.abs().max()))
+
+
 def test_decode_step_tiny_config_sampling_and_forcing():
     _decode_follow(si.WORKLOADS["tiny"], 22, zb.SELECT_GUMBEL, forced_every=3)
 

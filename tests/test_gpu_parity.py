@@ -654,3 +654,69 @@ def test_decode_logits_kernel_fixed_shares_and_pool():
     # V = 40000: every CTA owns a fixed share of 128-row jobs and the pool holds both W_U and U_h
     _logits_case(TALL_BF16, 53, [1, 1, 1, 1, 1, 1], False, 0, debug=False)
     _logits_case(TALL_BF16, 54, [2, 3, 1, 4, 0, 2], True, 1, debug=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# Limits of the configuration: largest and smallest merge size through the encoder and the decode
+# step, the largest batch, the largest codebook
+# ------------------------------------------------------------------------------------------------
+def _periodic_tail(p: Pair, period: int, head: int):
+    """Everything after the first `head` tokens of a prompt becomes a short cycle, so that phrases
+    reach length M."""
+    w = p.w
+    t = p.tokens.copy()
+    for b in range(w.B):
+        t[b, head:] = (np.arange(w.T - head) % period) + 3 * b
+    p.tokens = t
+
+
+@pytest.mark.parametrize("w", [SMALL_BF16.scaled(name="m8_bf16", M=8, T=400, cap=200, B=2, steps=4),
+                               SMALL_FP32.scaled(name="m8_fp32", M=8, T=300, cap=120, B=2, steps=3),
+                               SMALL_BF16.scaled(name="m8_small_pass", M=8, T=120, cap=63, B=2, steps=2),
+                               SMALL_BF16.scaled(name="m2_bf16", M=2, steps=3)],
+                         ids=lambda w: w.name)
+def test_hyper_embed_at_the_merge_size_limits(w):
+    p = Pair(w, seed=51)
+    if w.name == "m8_small_pass":              # < 1024 rows per pass: the weight-streaming GEMM
+        assert w.B * w.cap * w.M < 1024
+        _periodic_tail(p, 2, 30)
+    else:
+        _periodic_tail(p, 5, w.T // 2)
+    _, worst = _prefill_both(p)
+    assert worst <= TOL
+    longest = max(len(e) for bk in p.oracle.books for e in bk.entries)
+    assert longest == w.M
+    print(f"{w.name}: max |hyper-embedding error| = {worst:.3e}, longest entry {longest}")
+
+
+@pytest.mark.parametrize("w", [SMALL_BF16.scaled(name="m8_bf16", M=8, T=400, cap=200, B=2, copy_p=0.7,
+                                                 seg_min=8, seg_max=40),
+                               SMALL_BF16.scaled(name="m1_bf16", M=1),
+                               SMALL_FP32.scaled(name="m1_fp32", M=1)],
+                         ids=lambda w: w.name)
+def test_decode_step_at_the_merge_size_limits(w):
+    # M = 1 never creates a hypertoken: the step is a plain LM-head selection and the codebooks
+    # stay empty; M = 8 is the largest merge size
+    _decode_follow(w, 53, zb.SELECT_ARGMAX, steps=4)
+    if w.M == 1:
+        p = Pair(w, seed=53)
+        p.gpu_encode()
+        assert zb.z2z_status(p.cb)[1].tolist() == [0] * w.B
+
+
+@pytest.mark.parametrize("w", [si.WORKLOADS["tiny"].scaled(name="tiny_b1024", B=1024, T=24, cap=8, steps=2),
+                               SMALL_BF16.scaled(name="bf16_b1024", B=1024, T=24, cap=8, d=128, enc_heads=1,
+                                                 enc_dff=256, steps=2)],
+                         ids=lambda w: w.name)
+def test_largest_batch(w):
+    _decode_follow(w, 55, zb.SELECT_ARGMAX, steps=w.steps)
+
+
+def test_largest_codebook():
+    # cap = 65535, the most the 16-bit entry field of a slot addresses: nearly every pair of a
+    # uniform stream over a large vocabulary is new, so the book fills and freezes
+    rng = np.random.default_rng(57)
+    tokens = rng.integers(0, 60000, size=(1, 80000)).astype(np.int32)
+    g = _compare_encode(60000, 3, 65535, tokens)
+    ents, st = g.entries(0)
+    assert len(ents) == 65535 and st & zb.ST_CAP_FROZEN

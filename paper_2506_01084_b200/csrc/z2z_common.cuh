@@ -11,14 +11,15 @@
 namespace z2z {
 
 constexpr int kMaxM = 8;                 // maximum merge size supported
-constexpr int kBucket = 32;              // hash slots probed by one warp load
+constexpr int kWindow = 32;              // consecutive hash slots one warp load looks at
 constexpr uint64_t kEmptySlot = ~0ull;
 constexpr float kLnEps = 1e-5f;
 
 // ---------------------------------------------------------------------------------------------
 // Device view of all per-sequence codebook state (lives in the caller's workspace).
 //
-// hash  [B, n_slots] u64   open addressing, key = (prefix code, next base token) -> entry number
+// hash  [B, n_slots] u64   open addressing (linear probing from an even slot), key = (prefix
+//                          code, next base token) -> entry number
 //                          slot = prefix << 40 | token << 16 | entry ; all-ones = empty
 // cons  [B, cap, M]  i32   base tokens of entry k, -1 padded  (the paper's codebook, Figure 1)
 // len   [B, cap]     u8    number of base tokens of entry k

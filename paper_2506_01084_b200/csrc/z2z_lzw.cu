@@ -1,9 +1,10 @@
 // LZW codebook kernels: session reset, prompt compression, online update.
 //
 // One warp owns one sequence.  The codebook of a sequence is an open-addressing hash table in
-// global memory keyed by (prefix code, next base token); a probe is one coalesced 256-byte load of
-// a 32-slot bucket followed by a warp ballot.  Entries are never deleted and an insert always
-// takes the first empty slot in probe order, so "an empty slot in the bucket" proves absence.
+// global memory keyed by (prefix code, next base token), probed linearly from an even slot; a warp
+// probe is one coalesced 256-byte load of 32 consecutive slots followed by a ballot.  Entries are
+// never deleted and an insert always takes the first empty slot in probe order, so an empty slot
+// proves absence.
 // The parse itself is a dependent chain (each token's lookup needs the previous match), which is
 // why the unit of parallelism is the sequence (paper Section 2.4: compression is per document).
 #include "z2z_common.cuh"
@@ -87,111 +88,122 @@ __global__ void __launch_bounds__(128) k_lzw_encode(CbView cb, const int32_t* __
 }
 
 // The same parse with the sequence's hash table held in shared memory for the duration of the
-// kernel (codebooks of up to 8192 entries: 16384 slots, 128 KB).  The parse is a dependent chain
-// of one probe per token; the bucket read comes from shared memory instead of L2, and the
-// constituents of a new entry are not copied from the table: the phrase just matched IS the last
-// `wlen` tokens of the input, so the new row is written from the token registers (the current
-// batch of 32 and the one before it).  What remains per token is the chain of warp primitives of
-// the probe itself (broadcast, hash, ballot, shuffle): about 240 ns per token against about 290
-// with the table in global memory.  One CTA per sequence: warp 0 parses, all warps move the
-// table in and out.
+// kernel (codebooks of up to 12800 entries: at most 25600 slots, 200 KB).  The parse is a
+// dependent chain of one probe per token, and a chain that a single warp executes is paced by the
+// number of instructions it issues per token (about one every four to five cycles), not by memory.
+// A warp-wide probe spends most of them on warp primitives (broadcast, ballot, shuffle: about
+// 240 ns per token with the table in shared memory, 290 with the table in global memory); here
+// ONE thread walks the probe sequence two slots (one 16-byte shared-memory load) at a time, which
+// at a load factor of at most one half ends after one or two loads: 170-200 ns per token.  The
+// rest of warp 0 stages the tokens (the batch after the one being parsed is already in flight)
+// and the other warps move the table in and out.  A new entry is the last wlen + 1 input tokens,
+// so the chain only records where the phrase starts and how long it is (one word in the first
+// constituent slot, one length byte); all threads expand the records into constituent rows from
+// the token array after the parse.
 constexpr int kEncodeSmemThreads = 128;
 constexpr size_t kEncodeSmemMaxBytes = 200 * 1024;
-
-__device__ __forceinline__ Probe warp_probe_smem(const unsigned long long* table, int n_slots, uint32_t prefix,
-                                                 uint32_t token) {
-  const int lane = threadIdx.x & 31;
-  const unsigned long long key = pack_slot(prefix, token, 0) >> 16;
-  int bucket = (int)(hash_pair(prefix, token) & (uint32_t)(n_slots - 1)) & ~(kBucket - 1);
-  Probe r{-1, -1};
-  for (int it = 0; it < n_slots / kBucket; ++it) {          // bounded: at most the whole table
-    const unsigned long long s = table[bucket + lane];
-    const unsigned hit = __ballot_sync(0xffffffffu, (s >> 16) == key && s != kEmptySlot);
-    if (hit) {
-      const unsigned long long v = __shfl_sync(0xffffffffu, s, __ffs(hit) - 1);
-      r.found = (int)(v & 0xffffu);
-      return r;
-    }
-    const unsigned empty = __ballot_sync(0xffffffffu, s == kEmptySlot);
-    if (empty) { r.slot = bucket + __ffs(empty) - 1; return r; }
-    bucket = (bucket + kBucket) & (n_slots - 1);
-  }
-  return r;
-}
 
 __global__ void __launch_bounds__(kEncodeSmemThreads) k_lzw_encode_smem(CbView cb, const int32_t* __restrict__ tokens,
                                                                         const int32_t* __restrict__ lens, int T_max,
                                                                         int32_t* __restrict__ codes,
                                                                         int32_t* __restrict__ code_lens,
                                                                         int32_t* __restrict__ entries_after) {
-  extern __shared__ unsigned long long s_table[];
+  extern __shared__ __align__(16) unsigned long long s_table[];
+  __shared__ int s_tok[64];                          // two batches of 32 tokens
+  __shared__ int s_n0, s_n1;                         // entries before / after this call
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x;
   unsigned long long* table = cb.hash + (size_t)b * cb.n_slots;
   for (int i = threadIdx.x; i < cb.n_slots; i += blockDim.x) s_table[i] = table[i];
+  int T = lens ? lens[b] : T_max;
+  T = T < 0 ? 0 : (T > T_max ? T_max : T);
+  const int32_t* x = tokens + (size_t)b * T_max;
+  int32_t* const cons = cb.cons + (size_t)b * cb.cap * cb.M;
+  uint8_t* const len = cb.len + (size_t)b * cb.cap;
   __syncthreads();
   if (threadIdx.x < 32) {
-    int T = lens ? lens[b] : T_max;
-    T = T < 0 ? 0 : (T > T_max ? T_max : T);
-    const int32_t* x = tokens + (size_t)b * T_max;
     int32_t* out = codes + (size_t)b * T_max;
     int32_t* aft = entries_after ? entries_after + (size_t)b * T_max : nullptr;
+    const int V = cb.V, M = cb.M, cap = cb.cap, mask = cb.n_slots - 1;
     int n = cb.n[b];
+    if (lane == 0) s_n0 = n;
     int st = 0;
     int w = -1, wlen = 0, n_out = 0;
-    int mine = 0, before = 0;                        // tokens [base, base + 32) and [base - 32, base)
+    int ahead = lane < T ? x[lane] : 0;              // tokens of the batch after the current one
     for (int base = 0; base < T; base += 32) {
-      before = mine;
-      mine = (base + lane < T) ? x[base + lane] : 0;
-      if ((unsigned)mine >= (unsigned)cb.V) { if (base + lane < T) st |= Z2Z_ST_BAD_TOKEN; mine = 0; }   // not a base token
-      const int cnt = T - base < 32 ? T - base : 32;
-      for (int i = 0; i < cnt; ++i) {
-        const int c = __shfl_sync(0xffffffffu, mine, i);
-        if (wlen == 0) { w = c; wlen = 1; continue; }
-        Probe p{-1, -1};
-        if (wlen < cb.M) {
-          p = warp_probe_smem(s_table, cb.n_slots, (uint32_t)w, (uint32_t)c);
-          if (p.found >= 0) { w = cb.V + p.found; ++wlen; continue; }      // match grows
-        }
-        // longest match ends: emit it, then remember (w ++ c) if allowed
-        if (lane == 0) out[n_out] = w;
-        if (wlen < cb.M && n < cb.cap) {
-          if (p.slot >= 0) {
-            if (lane == 0) s_table[p.slot] = pack_slot((uint32_t)w, (uint32_t)c, (uint32_t)n);
-            // entry n = input tokens [i - wlen, i] of this batch (negative positions: the batch before)
-            const int pos = i - wlen + lane;                               // lane j holds constituent j
-            const int from_now = __shfl_sync(0xffffffffu, mine, pos & 31);
-            const int from_before = __shfl_sync(0xffffffffu, before, pos & 31);
-            if (lane < cb.M) {
-              const int v = lane <= wlen ? (pos >= 0 ? from_now : from_before) : -1;
-              cb.cons[((size_t)b * cb.cap + n) * cb.M + lane] = v;
+      int mine = ahead;
+      ahead = base + 32 + lane < T ? x[base + 32 + lane] : 0;
+      if ((unsigned)mine >= (unsigned)V) { if (base + lane < T) st |= Z2Z_ST_BAD_TOKEN; mine = 0; }   // not a base token
+      s_tok[(base & 32) + lane] = mine;
+      __syncwarp();
+      if (lane == 0) {
+        const int cnt = T - base < 32 ? T - base : 32;
+        int c_next = s_tok[base & 63];
+        for (int i = 0; i < cnt; ++i) {
+          const int c = c_next;
+          c_next = s_tok[(base + i + 1) & 63];         // off the chain: ready before the next probe needs it
+          if (wlen == 0) { w = c; wlen = 1; continue; }
+          int slot = -1;
+          if (wlen < M) {
+            const unsigned long long key = pack_slot((uint32_t)w, (uint32_t)c, 0) >> 16;
+            int at = probe_start(cb.n_slots, (uint32_t)w, (uint32_t)c);
+            int found = -1;
+            for (int it = 0; it <= mask; it += 2) {   // bounded: at most the whole table
+              const ulonglong2 pr = *reinterpret_cast<const ulonglong2*>(&s_table[at]);
+              // (a key never equals the upper 48 bits of the empty pattern: prefix < 2^24 - 1)
+              if ((pr.x >> 16) == key) { found = (int)(pr.x & 0xffffu); break; }
+              if (pr.x == kEmptySlot) { slot = at; break; }
+              if ((pr.y >> 16) == key) { found = (int)(pr.y & 0xffffu); break; }
+              if (pr.y == kEmptySlot) { slot = at + 1; break; }
+              at = (at + 2) & mask;
             }
-            if (lane == 0) cb.len[(size_t)b * cb.cap + n] = (uint8_t)(wlen + 1);
-            ++n;
-            if (n >= cb.cap) st |= Z2Z_ST_CAP_FROZEN;
-            __syncwarp();                     // the new slot is visible to later probes
-          } else {
-            st |= Z2Z_ST_TABLE_FULL;
+            if (found >= 0) { w = V + found; ++wlen; continue; }          // match grows
           }
+          // longest match ends: emit it, then remember (w ++ c) if allowed
+          out[n_out] = w;
+          if (wlen < M && n < cap) {
+            if (slot >= 0) {
+              s_table[slot] = pack_slot((uint32_t)w, (uint32_t)c, (uint32_t)n);
+              cons[(size_t)n * M] = base + i - wlen;                       // where the phrase starts
+              len[n] = (uint8_t)(wlen + 1);
+              ++n;
+              if (n >= cap) st |= Z2Z_ST_CAP_FROZEN;
+            } else {
+              st |= Z2Z_ST_TABLE_FULL;
+            }
+          }
+          if (aft) aft[n_out] = n;
+          ++n_out;
+          w = c; wlen = 1;
         }
-        if (aft && lane == 0) aft[n_out] = n;
-        ++n_out;
-        w = c; wlen = 1;
       }
+      __syncwarp();                                  // the other half of s_tok may be rewritten
     }
-    if (wlen > 0) {                             // final flush creates no entry
-      if (lane == 0) { out[n_out] = w; if (aft) aft[n_out] = n; }
-      ++n_out;
-    }
-    st = __reduce_or_sync(0xffffffffu, st);     // BAD_TOKEN is found per lane
     if (lane == 0) {
+      if (wlen > 0) {                                // final flush creates no entry
+        out[n_out] = w;
+        if (aft) aft[n_out] = n;
+        ++n_out;
+      }
       code_lens[b] = n_out;
       cb.n[b] = n;
       if (n_out > 0) cb.prev[b] = w;
-      if (st) atomicOr(&cb.status[b], st);
+      s_n1 = n;
     }
+    st = __reduce_or_sync(0xffffffffu, st);           // BAD_TOKEN is found per lane
+    if (lane == 0 && st) atomicOr(&cb.status[b], st);
   }
   __syncthreads();
+  // constituent rows of the entries created here: tokens [start, start + len), -1 padded
+  for (int e = s_n0 + threadIdx.x; e < s_n1; e += blockDim.x) {
+    const int start = cons[(size_t)e * cb.M];
+    const int L = len[e];
+    for (int j = 0; j < cb.M; ++j) {
+      int v = -1;
+      if (j < L) { v = x[start + j]; if ((unsigned)v >= (unsigned)cb.V) v = 0; }
+      cons[(size_t)e * cb.M + j] = v;
+    }
+  }
   for (int i = threadIdx.x; i < cb.n_slots; i += blockDim.x) table[i] = s_table[i];
 }
 

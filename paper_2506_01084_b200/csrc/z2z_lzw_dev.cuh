@@ -11,15 +11,23 @@ struct Probe {
   int slot;         // if absent: first empty slot in probe order (-1: table full)
 };
 
-// All 32 lanes must call this together.
+// First slot of the probe sequence of (prefix, token): linear probing from an even slot, so that
+// a single thread can walk the sequence two slots (16 bytes) at a time and a warp can look at a
+// window of kWindow consecutive slots at once.  Entries are never deleted and an insert takes the
+// first empty slot of the sequence, so an empty slot proves that the key is absent.
+__device__ __forceinline__ int probe_start(int n_slots, uint32_t prefix, uint32_t token) {
+  return (int)(hash_pair(prefix, token) & (uint32_t)(n_slots - 1)) & ~1;
+}
+
+// All 32 lanes must call this together: lane l looks at slot (start + l) of the sequence.
 __device__ __forceinline__ Probe warp_probe(const unsigned long long* __restrict__ table,
                                             int n_slots, uint32_t prefix, uint32_t token) {
   const int lane = threadIdx.x & 31;
   const unsigned long long key = pack_slot(prefix, token, 0) >> 16;
-  int bucket = (int)(hash_pair(prefix, token) & (uint32_t)(n_slots - 1)) & ~(kBucket - 1);
+  int at = probe_start(n_slots, prefix, token);
   Probe r{-1, -1};
-  for (int it = 0; it < n_slots / kBucket; ++it) {          // bounded: at most the whole table
-    unsigned long long s = table[bucket + lane];
+  for (int it = 0; it < n_slots / kWindow; ++it) {          // bounded: at most the whole table
+    unsigned long long s = table[(at + lane) & (n_slots - 1)];
     unsigned hit = __ballot_sync(0xffffffffu, (s >> 16) == key && s != kEmptySlot);
     if (hit) {
       int src = __ffs(hit) - 1;
@@ -28,8 +36,8 @@ __device__ __forceinline__ Probe warp_probe(const unsigned long long* __restrict
       return r;
     }
     unsigned empty = __ballot_sync(0xffffffffu, s == kEmptySlot);
-    if (empty) { r.slot = bucket + __ffs(empty) - 1; return r; }
-    bucket = (bucket + kBucket) & (n_slots - 1);
+    if (empty) { r.slot = (at + __ffs(empty) - 1) & (n_slots - 1); return r; }
+    at = (at + kWindow) & (n_slots - 1);
   }
   return r;
 }

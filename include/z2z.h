@@ -56,6 +56,11 @@ enum {
 
 enum { Z2Z_DTYPE_FP32 = 0, Z2Z_DTYPE_BF16 = 1 };
 enum { Z2Z_SELECT_ARGMAX = 0, Z2Z_SELECT_GUMBEL = 1 };
+/* Markers in place of a code (batches whose sequences finish at different times):
+ *   Z2Z_CODE_NONE      no token: in d_forced the sequence sits the step out; z2z_embed_lookup
+ *                      writes a zero row for it and raises no status.
+ *   Z2Z_CODE_SELECTED  in d_forced only: apply the step's own selection to this sequence.        */
+enum { Z2Z_CODE_NONE = -1, Z2Z_CODE_SELECTED = -2 };
 enum { Z2Z_CACHE_EMBED = 0, Z2Z_CACHE_UNEMBED = 1 };
 
 typedef struct {
@@ -154,7 +159,11 @@ int32_t z2z_dynamic_logits(z2z_codebook* cb, const void* d_hidden, int32_t N,
  * hidden row b of sequence b, LZW update with the selected code, hyper-encoder on the at most
  * one new entry per sequence for both caches.
  *   d_forced [B] or NULL: codes to feed the update instead of the selection (teacher forcing;
- *            the selection is still computed and returned in d_selected).
+ *            the selection is still computed and returned in d_selected).  Z2Z_CODE_SELECTED
+ *            applies the selection after all; Z2Z_CODE_NONE makes the sequence sit the step out
+ *            (a finished sequence of the batch): its codebook, caches and status stay as they
+ *            are, d_next_codes[b] = Z2Z_CODE_NONE, d_new_entry[b] = -1, its row of d_next_embed
+ *            is zero; the row's logits results are still computed and returned.
  *   d_next_codes [B] out: the code that was applied; d_selected [B] out or NULL: argmax/sample;
  *   d_lse [B] out; d_new_entry [B] out or NULL.  These small result arrays may also be pinned host
  *            memory that is mapped into the device's address space: the kernels then store the
@@ -194,7 +203,8 @@ int32_t z2z_lzw_decode(z2z_codebook* cb, const int32_t* d_codes, const int32_t* 
  * W_E[z] for a base token z < V and the cached hyper-embedding E_h[b][z - V] otherwise, where
  * b = d_row_seq[r] (or r when d_row_seq is NULL, which needs N <= B).
  *   d_codes [N] int32; d_WE [V, d]; d_Eh [B, cap, d]; d_out [N, d]; all in the configured dtype.
- * A code outside [0, V + n_b) sets Z2Z_ST_BAD_TOKEN for that sequence and its row is zero-filled. */
+ * A code outside [0, V + n_b) sets Z2Z_ST_BAD_TOKEN for that sequence and its row is zero-filled;
+ * Z2Z_CODE_NONE gives a zero row and no status.                                                */
 int32_t z2z_embed_lookup(z2z_codebook* cb, const int32_t* d_codes, int32_t N,
                          const int32_t* d_row_seq, const void* d_WE, const void* d_Eh,
                          void* d_out, z2z_stream stream);

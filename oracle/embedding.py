@@ -21,7 +21,8 @@ def lookup(codes: Sequence[int], row_seq: Optional[Sequence[int]], W_E: np.ndarr
     """Row r of the result embeds codes[r] for sequence b = row_seq[r] (r itself if row_seq is
     None).  W_E is [V, d]; E_h is [B, cap, d]; n[b] is the number of hypertokens sequence b has.
     A code outside [0, V + n[b]) gives a zero row and is reported in the returned list ``bad``
-    (sequence numbers)."""
+    (sequence numbers); -1 stands for "no token" (a sequence that has finished): a zero row,
+    not reported."""
     V, d = W_E.shape
     out = np.zeros((len(codes), d), dtype=np.float64)
     bad = []
@@ -32,6 +33,6 @@ def lookup(codes: Sequence[int], row_seq: Optional[Sequence[int]], W_E: np.ndarr
             out[r] = W_E[z]
         elif V <= z < V + int(n[b]):
             out[r] = E_h[b, z - V]
-        else:
+        elif z != -1:
             bad.append(b)
     return out, bad

@@ -19,6 +19,7 @@ OK = 0
 ST_CAP_FROZEN, ST_BAD_TOKEN, ST_TABLE_FULL, ST_WAIT_TIMEOUT, ST_OUTPUT_TRUNCATED = 1, 2, 4, 8, 16
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 SELECT_ARGMAX, SELECT_GUMBEL = 0, 1
+CODE_NONE, CODE_SELECTED = -1, -2
 CACHE_EMBED, CACHE_UNEMBED = 0, 1
 DECODE_RESIDENT, DECODE_REPLAY = 0, 1
 

@@ -239,7 +239,7 @@ int32_t z2z_lzw_step(z2z_codebook* cb, const int32_t* d_new_codes, const uint8_t
   if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
   if (!d_new_codes) return fail(Z2Z_ERR_INVALID_ARG, "d_new_codes is NULL");
   z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, reinterpret_cast<cudaStream_t>(stream));
-  Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_new_codes, d_active, d_new_entry,
+  Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_new_codes, d_active, 0, d_new_entry,
                                 reinterpret_cast<cudaStream_t>(stream)), "lzw_step");
   return Z2Z_OK;
 }
@@ -399,7 +399,7 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
     // step 10: online LZW update
     {
       z2z::ProfScope ps(&cb->prof, z2z::kProfLzw, 1, s);
-      Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_next_codes, nullptr, w_new, s), "decode_step");
+      Z2Z_CUDA(z2z::launch_lzw_step(cb->view, d_next_codes, nullptr, d_forced ? 1 : 0, w_new, s), "decode_step");
     }
     if (cb->cfg.cap > 0) {
       z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 4, s);

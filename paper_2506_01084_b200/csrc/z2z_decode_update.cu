@@ -1,6 +1,6 @@
 // Middle of the decode step in ONE launch (paper Section 2.3, steps 8-10): finish the joint
 // softmax reductions of every sequence from the per-CTA partials of the logits kernel, select the
-// token (argmax or Gumbel-max sample, or the caller's forced code), apply the online LZW update,
+// token (argmax or Gumbel-max sample, or the caller's forced code; a sequence may sit out), apply the online LZW update,
 // and build the work list of new codebook entries for the hyper-encoder pass that follows.
 // One warp per sequence; a single block, so that the list can be compacted without a second
 // launch.
@@ -41,14 +41,16 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
     const int amax = red.idx == 0x7fffffff ? -1 : red.idx;
     const int smp = red.gidx == 0x7fffffff ? -1 : red.gidx;
     const int sel = a.select == Z2Z_SELECT_GUMBEL ? smp : amax;
-    const int code = a.forced ? a.forced[b] : sel;
+    int code = a.forced ? a.forced[b] : sel;
+    if (code == Z2Z_CODE_SELECTED) code = sel;
+    const bool sits_out = a.forced && code == Z2Z_CODE_NONE;   // a finished sequence of the batch
     if (lane == 0) {
       if (a.lse) a.lse[b] = red.m + logf(red.s);
       if (a.selected) a.selected[b] = sel;
       a.next_codes[b] = code;
     }
     // ---- online LZW update with the applied code
-    const int created = warp_lzw_step(cb, b, code, state);
+    const int created = sits_out ? -1 : warp_lzw_step(cb, b, code, state);
     if (lane == 0) {
       if (a.new_entry) a.new_entry[b] = created;
       s_cnt[b] = created >= 0 ? created + 1 : 0;         // 0: none, else entry number + 1

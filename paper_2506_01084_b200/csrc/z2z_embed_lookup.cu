@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(kLookupThreads) k_embed_lookup(
     }
     uint4* dst = out + (size_t)r * row_vecs;
     if (!src) {                                   // no such token: zero row, flag the sequence
-      if (lane == 0 && (unsigned)b < (unsigned)cb.B) atomicOr(&cb.status[b], Z2Z_ST_BAD_TOKEN);
+      if (lane == 0 && z != Z2Z_CODE_NONE && (unsigned)b < (unsigned)cb.B) atomicOr(&cb.status[b], Z2Z_ST_BAD_TOKEN);
       for (int i = lane; i < row_vecs; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
       continue;
     }

@@ -38,7 +38,7 @@ cudaError_t launch_embed_lookup(const CbView& cb, const int32_t* codes, int N,
                                 const int32_t* row_seq, const void* WE, const void* Eh, void* out,
                                 int d, int elem_bytes, cudaStream_t s);
 cudaError_t launch_lzw_step(const CbView& cb, const int32_t* new_codes, const uint8_t* active,
-                            int32_t* new_entry, cudaStream_t s);
+                            int none_sits_out, int32_t* new_entry, cudaStream_t s);
 
 // ---- z2z_encoder.cu --------------------------------------------------------------------------
 // Work list of one encoder pass: up to `chunk` entries, entry e -> (sequence, entry number).

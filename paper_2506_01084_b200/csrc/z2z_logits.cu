@@ -191,7 +191,9 @@ __global__ void k_pick_codes(int B, const int32_t* __restrict__ argmax,
   if (b >= B) return;
   const int sel = sample ? sample[b] : argmax[b];
   if (selected) selected[b] = sel;
-  next_codes[b] = forced ? forced[b] : sel;
+  int code = forced ? forced[b] : sel;
+  if (code == Z2Z_CODE_SELECTED) code = sel;
+  next_codes[b] = code;
 }
 
 cudaError_t launch_pick_codes(int B, const int32_t* argmax, const int32_t* sample,

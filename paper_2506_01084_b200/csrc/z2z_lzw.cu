@@ -208,13 +208,17 @@ __global__ void __launch_bounds__(kEncodeSmemThreads) k_lzw_encode_smem(CbView c
 }
 
 // Online update with one new code per sequence (Figure 1; Section 2.3 step 10).
+// none_sits_out: a code equal to Z2Z_CODE_NONE marks a sequence that takes no part in this step.
 __global__ void __launch_bounds__(128) k_lzw_step(CbView cb, const int32_t* __restrict__ new_codes,
-                                                  const uint8_t* __restrict__ active,
+                                                  const uint8_t* __restrict__ active, int none_sits_out,
                                                   int32_t* __restrict__ new_entry) {
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (b >= cb.B) return;
-  if (active && !active[b]) { if (lane == 0 && new_entry) new_entry[b] = -1; return; }
+  if ((active && !active[b]) || (none_sits_out && new_codes[b] == Z2Z_CODE_NONE)) {
+    if (lane == 0 && new_entry) new_entry[b] = -1;
+    return;
+  }
   const int created = warp_lzw_step(cb, b, new_codes[b]);
   if (lane == 0 && new_entry) new_entry[b] = created;
 }
@@ -247,9 +251,9 @@ cudaError_t launch_lzw_encode(const CbView& cb, const int32_t* tokens, const int
 }
 
 cudaError_t launch_lzw_step(const CbView& cb, const int32_t* new_codes, const uint8_t* active,
-                            int32_t* new_entry, cudaStream_t s) {
+                            int none_sits_out, int32_t* new_entry, cudaStream_t s) {
   int wpb = 4;
-  k_lzw_step<<<(cb.B + wpb - 1) / wpb, wpb * 32, 0, s>>>(cb, new_codes, active, new_entry);
+  k_lzw_step<<<(cb.B + wpb - 1) / wpb, wpb * 32, 0, s>>>(cb, new_codes, active, none_sits_out, new_entry);
   return cudaGetLastError();
 }
 

@@ -312,7 +312,8 @@ def test_dynamic_logits_no_hypertokens_is_plain_lm_head():
 # ------------------------------------------------------------------------------------------------
 # Whole decode step, following the GPU's selections inside the oracle's top-2 gap
 # ------------------------------------------------------------------------------------------------
-def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=True, host_results=False):
+def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=True, host_results=False,
+                   sits_out=None):
     p = Pair(w, seed=seed, tensor_cores=tensor_cores)
     _prefill_both(p)
     for b in range(w.B):
@@ -340,6 +341,9 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
             # an id equal to V + n is legal only in the special case; keep forced ids existing
             forced = [min(z, w.V + n0[b] - 1) if n0[b] else min(z, w.V - 1)
                       for b, z in enumerate(forced)]
+        if sits_out is not None:      # sequences that have finished take no part; the others run free
+            forced = [zb.CODE_SELECTED] * w.B if forced is None else forced
+            forced = [zb.CODE_NONE if sits_out(t, b) else z for b, z in enumerate(forced)]
         zb.z2z_decode_step(p.cb, g_hid[t], p.g_WE, p.g_WU, p.g_encE, p.g_encU, p.E_h, p.U_h,
                            select, 0.9, 4242, t,
                            None if forced is None else torch.tensor(forced, dtype=torch.int32,
@@ -360,10 +364,10 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
                 assert sc[b]["gap"] < GAP and s[g_sel[b]] >= s[sc[b]["choice"]] - GAP, \
                     (t, b, g_sel[b], sc[b]["choice"], sc[b]["gap"])
                 followed += 1
-            want_next = forced[b] if forced is not None else int(g_sel[b])
+            want_next = forced[b] if forced is not None and forced[b] != zb.CODE_SELECTED else int(g_sel[b])
             assert g_nxt[b] == want_next
             apply.append(want_next)
-        onew = p.oracle.advance(apply)
+        onew = p.oracle.advance(apply, active=[z != zb.CODE_NONE for z in apply])
         assert g_new.tolist() == onew, (t, g_new.tolist(), onew)
         # input embedding of the applied codes for the next model step (Figure 2a): a base token's
         # row is a copy; a hypertoken's row is the cached hyper-embedding (the row created by this
@@ -374,7 +378,7 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
         want_emb, bad = oemb.lookup(apply, None, f64(p.W_E), E_pad, [bk.n() for bk in p.oracle.books])
         assert bad == []
         for b in range(w.B):
-            if apply[b] < w.V:
+            if apply[b] < w.V:                   # (a sequence that sat out: a zero row)
                 assert np.array_equal(g_emb[b], want_emb[b])
             else:
                 assert np.abs(g_emb[b] - want_emb[b]).max() <= TOL, (t, b, apply[b])
@@ -385,6 +389,8 @@ def _decode_follow(w, seed, select, steps=None, forced_every=0, tensor_cores=Tru
         st, n = zb.z2z_status(p.cb)
         assert n.tolist() == [bk.n() for bk in p.oracle.books]
     p.check_codebooks()
+    st, _ = zb.z2z_status(p.cb)
+    assert all(int(x) & zb.ST_BAD_TOKEN == 0 for x in st)       # no step fed a code that names nothing
     return followed, worst_lse
 
 
@@ -436,6 +442,19 @@ def test_decode_step_with_frozen_codebooks():
 def test_decode_step_results_written_to_pinned_host_memory():
     for w, sel in ((si.WORKLOADS["tiny"], zb.SELECT_ARGMAX), (SMALL_BF16, zb.SELECT_GUMBEL)):
         _decode_follow(w, 27, sel, steps=6, forced_every=3, host_results=True)
+
+
+@pytest.mark.parametrize("w", [SMALL_BF16.scaled(name="small_bf16_b5", B=5),
+                               si.WORKLOADS["tiny"].scaled(name="tiny_b130", B=130, T=48, cap=24)],
+                         ids=lambda w: w.name)
+def test_decode_step_with_sequences_sitting_out(w):
+    # a batch whose sequences finish at different times: a finished sequence keeps its codebook,
+    # caches and status while the others go on (free-running and teacher-forced steps mixed);
+    # 130 sequences take the path with separate selection and update kernels
+    done_at = {b: 2 + (b % 4) for b in range(w.B)}
+    _decode_follow(w, 61, zb.SELECT_ARGMAX, steps=7, forced_every=3,
+                   sits_out=lambda t, b: b % 2 == 1 and t >= done_at[b])
+    _decode_follow(w, 62, zb.SELECT_GUMBEL, steps=5, sits_out=lambda t, b: t % 2 == 1 and b != 0)
 
 
 def test_decode_steps_replayed_from_a_cuda_graph():

@@ -197,6 +197,10 @@ def test_lookup_of_base_tokens_is_a_row_gather_and_flags_missing_hypertokens():
     out, bad = oemb.lookup([V + 1, V + 2, V], [0, 0, 1], W, E, [2, 3])
     assert bad == [0] and np.array_equal(out[0], E[0, 1]) and not out[1].any()
     assert np.array_equal(out[2], E[1, 0])
+    # -1 is "no token" (a sequence that has finished): a zero row that is not an error; any
+    # other id outside [0, V + n) is one
+    out, bad = oemb.lookup([-1, 3, -2], [0, 1, 1], W, E, [2, 3])
+    assert bad == [1] and not out[0].any() and np.array_equal(out[1], W[3]) and not out[2].any()
 
 
 def test_lookup_of_a_hypertoken_under_the_averaging_encoder_is_the_mean_of_its_base_rows():

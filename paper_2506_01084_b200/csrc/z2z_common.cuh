@@ -45,12 +45,14 @@ __host__ __device__ inline unsigned long long pack_slot(uint32_t prefix, uint32_
          (unsigned long long)entry;
 }
 
+// Multiplicative hash of the pair, upper bits (tables have at most 2^17 slots: bits 13..29).  The
+// token's part does not depend on the running match, so a parser can compute it ahead.
+__host__ __device__ inline uint32_t hash_token_part(uint32_t token) { return token * 0x85EBCA77u + 0x165667B1u; }
+__host__ __device__ inline uint32_t hash_join(uint32_t prefix, uint32_t token_part) {
+  return (prefix * 0x9E3779B1u ^ token_part) >> 13;
+}
 __host__ __device__ inline uint32_t hash_pair(uint32_t prefix, uint32_t token) {
-  uint32_t h = prefix * 0x9E3779B1u ^ (token * 0x85EBCA77u + 0x165667B1u);
-  h ^= h >> 15;
-  h *= 0x2C1B3C6Du;
-  h ^= h >> 12;
-  return h;
+  return hash_join(prefix, hash_token_part(token));
 }
 
 // CTA that owns unit u when U units are dealt to G CTAs as [floor(c U / G), floor((c+1) U / G)).

@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(128) k_lzw_encode(CbView cb, const int32_t* __
 // A warp-wide probe spends most of them on warp primitives (broadcast, ballot, shuffle: about
 // 240 ns per token with the table in shared memory, 290 with the table in global memory); here
 // ONE thread walks the probe sequence two slots (one 16-byte shared-memory load) at a time, which
-// at a load factor of at most one half ends after one or two loads: 170-200 ns per token.  The
+// at a load factor of at most one half ends after one or two loads: 165-195 ns per token.  The
 // rest of warp 0 stages the tokens (the batch after the one being parsed is already in flight)
 // and the other warps move the table in and out.  A new entry is the last wlen + 1 input tokens,
 // so the chain only records where the phrase starts and how long it is (one word in the first
@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(kEncodeSmemThreads) k_lzw_encode_smem(CbView c
                                                                         int32_t* __restrict__ code_lens,
                                                                         int32_t* __restrict__ entries_after) {
   extern __shared__ __align__(16) unsigned long long s_table[];
-  __shared__ int s_tok[64];                          // two batches of 32 tokens
+  __shared__ int4 s_tok[64];                         // two batches of 32 tokens: {c, hash part, c >> 16, c & 0xffff}
   __shared__ int s_n0, s_n1;                         // entries before / after this call
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x;
@@ -124,7 +124,10 @@ __global__ void __launch_bounds__(kEncodeSmemThreads) k_lzw_encode_smem(CbView c
   if (threadIdx.x < 32) {
     int32_t* out = codes + (size_t)b * T_max;
     int32_t* aft = entries_after ? entries_after + (size_t)b * T_max : nullptr;
-    const int V = cb.V, M = cb.M, cap = cb.cap, mask = cb.n_slots - 1;
+    const int V = cb.V, M = cb.M, cap = cb.cap;
+    const uint32_t pair_mask = (uint32_t)(cb.n_slots - 1) & ~1u;
+    // a slot as two words: hi = prefix << 8 | token >> 16, lo = token << 16 | entry (all-ones hi = empty)
+    const uint2* const slots = reinterpret_cast<const uint2*>(s_table);
     int n = cb.n[b];
     if (lane == 0) s_n0 = n;
     int st = 0;
@@ -134,28 +137,28 @@ __global__ void __launch_bounds__(kEncodeSmemThreads) k_lzw_encode_smem(CbView c
       int mine = ahead;
       ahead = base + 32 + lane < T ? x[base + 32 + lane] : 0;
       if ((unsigned)mine >= (unsigned)V) { if (base + lane < T) st |= Z2Z_ST_BAD_TOKEN; mine = 0; }   // not a base token
-      s_tok[(base & 32) + lane] = mine;
+      s_tok[(base & 32) + lane] = make_int4(mine, (int)hash_token_part((uint32_t)mine), mine >> 16, mine & 0xffff);
       __syncwarp();
       if (lane == 0) {
         const int cnt = T - base < 32 ? T - base : 32;
-        int c_next = s_tok[base & 63];
+        int4 t_next = s_tok[base & 63];
         for (int i = 0; i < cnt; ++i) {
-          const int c = c_next;
-          c_next = s_tok[(base + i + 1) & 63];         // off the chain: ready before the next probe needs it
+          const int4 t = t_next;
+          t_next = s_tok[(base + i + 1) & 63];         // off the chain: ready before the next probe needs it
+          const int c = t.x;
           if (wlen == 0) { w = c; wlen = 1; continue; }
           int slot = -1;
+          const uint32_t key_hi = ((uint32_t)w << 8) | (uint32_t)t.z;
           if (wlen < M) {
-            const unsigned long long key = pack_slot((uint32_t)w, (uint32_t)c, 0) >> 16;
-            int at = probe_start(cb.n_slots, (uint32_t)w, (uint32_t)c);
+            uint32_t at = hash_join((uint32_t)w, (uint32_t)t.y) & pair_mask;
             int found = -1;
-            for (int it = 0; it <= mask; it += 2) {   // bounded: at most the whole table
-              const ulonglong2 pr = *reinterpret_cast<const ulonglong2*>(&s_table[at]);
-              // (a key never equals the upper 48 bits of the empty pattern: prefix < 2^24 - 1)
-              if ((pr.x >> 16) == key) { found = (int)(pr.x & 0xffffu); break; }
-              if (pr.x == kEmptySlot) { slot = at; break; }
-              if ((pr.y >> 16) == key) { found = (int)(pr.y & 0xffffu); break; }
-              if (pr.y == kEmptySlot) { slot = at + 1; break; }
-              at = (at + 2) & mask;
+            for (int it = 0; it < cb.n_slots; it += 2) {   // bounded: at most the whole table
+              const uint4 pr = *reinterpret_cast<const uint4*>(&slots[at]);      // slots at, at + 1: {lo, hi, lo, hi}
+              if (pr.y == key_hi && (pr.x >> 16) == (uint32_t)t.w) { found = (int)(pr.x & 0xffffu); break; }
+              if (pr.y == 0xffffffffu) { slot = (int)at; break; }              // (no prefix is 2^24 - 1)
+              if (pr.w == key_hi && (pr.z >> 16) == (uint32_t)t.w) { found = (int)(pr.z & 0xffffu); break; }
+              if (pr.w == 0xffffffffu) { slot = (int)at + 1; break; }
+              at = (at + 2) & pair_mask;
             }
             if (found >= 0) { w = V + found; ++wlen; continue; }          // match grows
           }
@@ -163,7 +166,7 @@ __global__ void __launch_bounds__(kEncodeSmemThreads) k_lzw_encode_smem(CbView c
           out[n_out] = w;
           if (wlen < M && n < cap) {
             if (slot >= 0) {
-              s_table[slot] = pack_slot((uint32_t)w, (uint32_t)c, (uint32_t)n);
+              reinterpret_cast<uint2*>(s_table)[slot] = make_uint2(((uint32_t)t.w << 16) | (uint32_t)n, key_hi);
               cons[(size_t)n * M] = base + i - wlen;                       // where the phrase starts
               len[n] = (uint8_t)(wlen + 1);
               ++n;

@@ -141,6 +141,34 @@ def reduce_over_ranks(times_ms, counts, world: int, device):
     return tt.tolist(), cc.tolist()
 
 
+def forced_codes(zb, w, cb, dev, stream, prompt_code_lens, n_steps: int):
+    """Teacher forcing: the codes a zip2zip model would have to emit to continue each sequence
+    with the generator's own tokens.  The whole stream (prompt + continuation) is compressed in a
+    scratch session; by the online property of LZW its first k - 1 codes are the first k - 1 codes
+    of the prompt alone (k = the prompt's code count; the prompt's last code is a flush that the
+    longer stream may extend).  The session `cb` is restarted and grown from those k - 1 codes, so
+    that it is in exactly the state in which the stream's k-th, k+1-th ... codes are the next
+    ones.  Returns them as [n_steps, B] int32 on the device."""
+    cfg = zb.make_config(w.V, 8, w.M, w.cap, w.B, "fp32", 0, 1, 8)
+    scratch = zb.Codebook(cfg, dev)
+    T_full = stream.shape[1]
+    codes = torch.zeros(w.B, T_full, dtype=torch.int32, device=dev)
+    clen = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    zb.z2z_lzw_encode(scratch, torch.from_numpy(stream).to(dev), None, codes, clen, None)
+    k = (prompt_code_lens.clamp(min=1) - 1).to(torch.int32)    # codes replayed per sequence
+    if int((clen - k).min().item()) < n_steps:
+        raise SystemExit("the continuation is too short for the requested steps")
+    zb.z2z_codebook_init(cb)                                    # new session on the same handle
+    toks = torch.zeros(w.B, w.T + 8, dtype=torch.int32, device=dev)
+    tlen = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    zb.z2z_lzw_decode(cb, codes, k, zb.DECODE_REPLAY, toks, tlen)
+    idx = k.to(torch.int64)[None, :] + torch.arange(n_steps, device=dev)[:, None]      # [n_steps, B]
+    forced = torch.gather(codes.t().contiguous(), 0, idx).to(torch.int32).contiguous()
+    torch.cuda.synchronize()
+    del scratch
+    return forced
+
+
 def kernel_source_digest() -> str:
     """Digest of the code of the streaming kernels (comments and blank space left out); an ncu
     traffic figure only counts while it matches the code that produced it."""
@@ -185,7 +213,16 @@ def run_ours(args, rank: int, world: int):
         raise SystemExit("this workload has no decode steps; use tests for the prefill path")
     K, Wm = args.steps, args.warmup
     seed = replica_seed(rank)
-    tokens = si.make_tokens(w, seed)
+    forced_mode = args.decode_mode == "forced"
+    n_steps_total = Wm + 3 * K                # warm-up, device-timed, per-kernel-timed, end-to-end
+    if forced_mode:
+        # one generator stream per sequence: its first T tokens are the prompt, the rest is the
+        # continuation whose LZW codes are fed to the steps (at most M tokens per code)
+        stream = si.make_tokens(w, seed, T=w.T + n_steps_total * w.M + 64)
+        tokens = np.ascontiguousarray(stream[:, :w.T])
+    else:
+        stream = None
+        tokens = si.make_tokens(w, seed)
     W_E, W_U = si.make_tables(w, seed)
     encE_t = [t.to(dev) for t in si.make_encoder(w, seed * 3 + 1)]
     encU_t = encE_t if w.tied else [t.to(dev) for t in si.make_encoder(w, seed * 3 + 2)]
@@ -196,7 +233,6 @@ def run_ours(args, rank: int, world: int):
     encE, encU = zb.encoder_weights(encE_t), zb.encoder_weights(encU_t)
     E_h = torch.zeros(w.B, w.cap, w.d, dtype=w.torch_dtype, device=dev)
     U_h = E_h if w.tied else torch.zeros_like(E_h)
-    n_steps_total = Wm + 3 * K                # warm-up, device-timed, per-kernel-timed, end-to-end
     hidden_host = si.make_hidden(w, n_steps_total * w.B, seed).view(n_steps_total, w.B, w.d).pin_memory()
     hidden = hidden_host.to(dev)
 
@@ -214,6 +250,16 @@ def run_ours(args, rank: int, world: int):
         zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, w.B * w.T, U_h, None)
     ev[2].record()
     torch.cuda.synchronize()
+    forced_dev = None
+    if forced_mode:
+        forced_dev = forced_codes(zb, w, cb, dev, stream, clen, n_steps_total)
+        # the session now holds the codebook of the prompt's codes but the last (replayed from the
+        # stream's own codes, so that the continuation's codes name its entries): embed them again
+        E_h.zero_(); U_h.zero_()
+        zb.z2z_hyper_embed(cb, zb.CACHE_EMBED, g_WE, encE, None, None, w.B * w.T, E_h, None)
+        if not w.tied:
+            zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, w.B * w.T, U_h, None)
+        torch.cuda.synchronize()
     st, n0 = zb.z2z_status(cb)
     prefill = {"lzw_encode_ms": ev[0].elapsed_time(ev[1]), "hyper_embed_all_ms": ev[1].elapsed_time(ev[2]),
                "prompt_tokens": int(w.B * w.T), "compressed_tokens": int(clen.sum().item()),
@@ -224,7 +270,7 @@ def run_ours(args, rank: int, world: int):
 
     def step(t, hid):
         zb.z2z_decode_step(cb, hid, g_WE, g_WU, encE, encU, E_h, U_h, zb.SELECT_ARGMAX, 1.0, 0, t,
-                           None, nxt_all[t], None, lse)
+                           None if forced_dev is None else forced_dev[t], nxt_all[t], None, lse)
 
     def barrier():
         if world > 1:
@@ -278,7 +324,7 @@ def run_ours(args, rank: int, world: int):
         # the call may be host memory that is mapped into the device's address space, so the
         # device -> host transfer of the result is the kernel's own stores
         zb.z2z_decode_step(cb, hid_dev, g_WE, g_WU, encE, encU, E_h, U_h, zb.SELECT_ARGMAX, 1.0, 0, t,
-                           None, out_host, None, lse_host)
+                           None if forced_dev is None else forced_dev[t], out_host, None, lse_host)
         # the caller needs the token to go on: it watches the result land in host memory instead of
         # waiting for the whole stream (the cache update of this step is still running then, and
         # the next step's launches queue up behind it)
@@ -353,7 +399,9 @@ def run_ours(args, rank: int, world: int):
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "prompt_tokens": w.T,
                    "M": w.M, "cap": w.cap, "enc_layers": w.enc_layers, "enc_dff": w.dff,
-                   "select": "argmax, free-running", "replicas": world,
+                   "select": ("argmax computed, the update is fed the LZW codes of a generator continuation "
+                              "(teacher forcing)" if forced_mode else "argmax, free-running"),
+                   "replicas": world,
                    "l2": l2_note},
         "steps_per_s": K / (dev_ms * 1e-3),
         "mean_phrase_len": bt_dev / (K * w.B * world),
@@ -554,6 +602,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="phi3_mini_head", choices=list(si.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-mode", default="free", choices=["free", "forced"],
+                    help="free: the selected code feeds the codebook update; forced: the update is fed the "
+                         "LZW codes of a generator continuation (the selection is still computed)")
     ap.add_argument("--seqs", type=int, default=0,
                     help="prompt-scoring workloads: use this many sequences instead of the workload's B")
     args = ap.parse_args()

@@ -214,3 +214,47 @@ def test_upload_rows_copies_pinned_host_memory():
     zb.z2z_upload_rows(src2, dst2)
     zb.z2z_upload_rows(src2[1:2], dst2[0:1])                                  # a view: row 1 over row 0
     assert torch.equal(dst2.cpu()[1:], src2[1:]) and torch.equal(dst2.cpu()[0], src2[1])
+
+
+def test_teacher_forcing_codes_of_the_benchmark_continue_the_prompt():
+    """The benchmark's teacher-forced mode restarts the session from all but the last of the
+    prompt's codes and feeds the steps the codes of the generator's continuation.  Held against
+    the oracle: those codes are the oracle's codes of the whole stream at the same positions, the
+    restarted session holds the oracle's codebook at that point, and after the codes have been
+    applied one per step the session decompresses (replayed codes + forced codes) to the
+    generator's own tokens."""
+    import os
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    if root not in sys.path:
+        sys.path.insert(0, root)
+    import bench
+    w = si.WORKLOADS["tiny"].scaled(B=3, T=200, cap=256)
+    n_steps = 40
+    stream = si.make_tokens(w, 71, T=w.T + n_steps * w.M + 64)
+    prompt = np.ascontiguousarray(stream[:, :w.T])
+    s = Session(w.V, w.M, w.cap, w.B)
+    codes = torch.zeros(w.B, w.T, dtype=torch.int32, device=DEV)
+    clen = torch.zeros(w.B, dtype=torch.int32, device=DEV)
+    zb.z2z_lzw_encode(s.cb, torch.from_numpy(prompt).to(DEV), None, codes, clen, None)
+    forced = bench.forced_codes(zb, w, s.cb, torch.device(DEV), stream, clen, n_steps).cpu().numpy()
+    k = (clen.cpu().numpy() - 1).tolist()
+    full = [olzw.encode(stream[b].tolist(), w.V, w.M, w.cap) for b in range(w.B)]
+    for b in range(w.B):
+        want_codes, want_after, _ = full[b]
+        assert olzw.encode(prompt[b].tolist(), w.V, w.M, w.cap)[0][:k[b]] == want_codes[:k[b]]
+        assert forced[:, b].tolist() == want_codes[k[b]:k[b] + n_steps]
+        ents, st = s.entries(b)
+        # an encoder that has emitted k codes has created the entry that the k-th code closes; the
+        # decoder-side update creates it one code later
+        assert st == 0
+        assert len(ents) == (want_after[k[b] - 2] if k[b] >= 2 else 0)
+        assert ents == full[b][2].entries[:len(ents)]
+    new = torch.zeros(w.B, dtype=torch.int32, device=DEV)
+    for t in range(n_steps):
+        zb.z2z_lzw_step(s.cb, torch.from_numpy(forced[t]).to(DEV), None, new)
+    rows = [full[b][0][:k[b] + n_steps] for b in range(w.B)]
+    toks, st = s.decode(rows, zb.DECODE_RESIDENT, w.T + n_steps * w.M + 64)
+    for b in range(w.B):
+        assert st[b] == 0
+        assert toks[b] == stream[b, :len(toks[b])].tolist() and len(toks[b]) > w.T - w.M

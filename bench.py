@@ -594,6 +594,85 @@ def run_prompt_scoring(args, rank: int, world: int):
     return line, w
 
 
+# --------------------------------------------------------------------------------------------------
+# the calls around the hot path (decompression, embedding lookup, filtered sampling), timed alone
+# --------------------------------------------------------------------------------------------------
+def run_helpers(args):
+    """One JSON line with device times of the helper calls at the workload's sizes: prompt
+    compression, decompression (replay and resident), the mixed-stream embedding lookup and
+    top-k / nucleus sampling on stored logits.  Every figure is the best of five event-timed calls
+    after a warm-up call; tables and logits larger than L2 where the call is bound by HBM."""
+    from paper_2506_01084_b200 import binding as zb
+    zb.lib()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    w = si.WORKLOADS[args.workload]
+    if args.seqs:
+        w = w.scaled(B=args.seqs)
+    pk = peaks()
+
+    def best_ms(fn, before=None, reps=5):
+        ts = []
+        for i in range(reps + 1):
+            if before:
+                before()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            if i:
+                ts.append(e0.elapsed_time(e1))
+        return min(ts)
+
+    out = {}
+    cfg = zb.make_config(w.V, w.d, w.M, w.cap, w.B, w.dtype, 0, 1, 8)
+    cb = zb.Codebook(cfg, dev)
+    tokens = si.make_tokens(w, 1000)
+    g_tok = torch.from_numpy(tokens).to(dev)
+    codes = torch.zeros(w.B, w.T, dtype=torch.int32, device=dev)
+    clen = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    ms = best_ms(lambda: zb.z2z_lzw_encode(cb, g_tok, None, codes, clen, None), before=lambda: zb.z2z_codebook_init(cb))
+    out["lzw_encode"] = {"ms": ms, "ns_per_token_of_a_sequence": ms * 1e6 / w.T, "B": w.B, "T": w.T}
+    toks = torch.zeros(w.B, w.T, dtype=torch.int32, device=dev)
+    tlen = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    ms = best_ms(lambda: zb.z2z_lzw_decode(cb, codes, clen, zb.DECODE_RESIDENT, toks, tlen))
+    out["lzw_decode_resident"] = {"ms": ms, "round_trip_ok": bool(torch.equal(toks, g_tok))}
+    ms = best_ms(lambda: zb.z2z_lzw_decode(cb, codes, clen, zb.DECODE_REPLAY, toks, tlen),
+                 before=lambda: zb.z2z_codebook_init(cb))
+    out["lzw_decode_replay"] = {"ms": ms, "round_trip_ok": bool(torch.equal(toks, g_tok))}
+    # embedding lookup of the compressed prompts (every code of every sequence)
+    _, n_b = zb.z2z_status(cb)
+    h_len = clen.cpu().numpy()
+    flat = torch.cat([codes[b, :int(h_len[b])] for b in range(w.B)]).contiguous()
+    seq = torch.cat([torch.full((int(h_len[b]),), b, dtype=torch.int32, device=dev) for b in range(w.B)])
+    es = 2 if w.dtype == "bf16" else 4
+    W_E = torch.zeros(w.V, w.d, dtype=w.torch_dtype, device=dev)
+    E_h = torch.zeros(w.B, max(w.cap, 1), w.d, dtype=w.torch_dtype, device=dev)
+    rows = torch.empty(flat.numel(), w.d, dtype=w.torch_dtype, device=dev)
+    ms = best_ms(lambda: zb.z2z_embed_lookup(cb, flat, seq, W_E, E_h, rows))
+    by = 2.0 * flat.numel() * w.d * es
+    out["embed_lookup"] = {"ms": ms, "rows": int(flat.numel()), "algorithmic_bytes": by, "gbs": by / ms / 1e6,
+                           "frac_of_measured_hbm": by / ms / 1e6 / pk["hbm_gbs"],
+                           "note": "every output row written once and its source row read once (%.0f MB); "
+                                   "source rows of frequent tokens repeat and are then served by L2, so the "
+                                   "rate can exceed the HBM copy rate" % (by / 1e6)}
+    # top-k / nucleus sampling on stored joint logits of one decode batch
+    ld = w.V + max(w.cap, 1)
+    g = torch.Generator(device="cpu"); g.manual_seed(5)
+    logits = (torch.randn(w.B, ld, generator=g) * 3.0).to(dev)
+    n_cols = (n_b.to(torch.int32) + w.V).to(dev)
+    choice = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    kept = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    for name, k, p in (("top_k_50", 50, 1.0), ("top_p_0.9", 0, 0.9), ("top_k_50_top_p_0.9", 50, 0.9)):
+        ms = best_ms(lambda: zb.z2z_sample_filtered(logits, n_cols, k, p, 0.8, 7, 3, choice, kept))
+        out["sample_filtered_" + name] = {"us": ms * 1e3, "rows": w.B, "columns": int(n_cols.max().item()),
+                                          "kept_mean": float(kept.float().mean().item())}
+    line = {"helpers": out, "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "T": w.T, "M": w.M,
+                                       "cap": w.cap}, "data": "synthetic",
+            "peak_hbm_gbs": pk["hbm_gbs"], "peak_source": pk["source"]}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -602,6 +681,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="phi3_mini_head", choices=list(si.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--helpers", action="store_true",
+                    help="time the calls around the hot path (compression, decompression, embedding lookup, "
+                         "filtered sampling) at the workload's sizes instead of the decode step")
     ap.add_argument("--decode-mode", default="free", choices=["free", "forced"],
                     help="free: the selected code feeds the codebook update; forced: the update is fed the "
                          "LZW codes of a generator continuation (the selection is still computed)")
@@ -614,6 +696,10 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             run_reference(args)
+        return
+    if args.helpers:
+        if rank == 0:
+            run_helpers(args)
         return
     if world > 1:
         torch.distributed.init_process_group("nccl")

@@ -4,7 +4,7 @@
 // they can be stored once (z2z_dynamic_logits with its full-logit output) and filtered here; the
 // fused argmax / Gumbel-max path of the logits kernels needs no stored logits.
 //
-// One CTA per row, every pass reads the row from L2:
+// One CTA per row, every pass reads the row from L2 (16-byte loads, two in flight per thread):
 //   1. m = max l,  Z = sum exp((l - m) / T);
 //   2. top-k: radix select (4 passes of 8 bits over order-preserving keys of the logits) of the
 //      k-th largest logit; everything >= it is kept (ties stay together);
@@ -28,11 +28,19 @@ __device__ __forceinline__ uint32_t order_key(float x) {          // larger floa
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Histograms of a radix pass are kept once per lane (bin * 32 + lane): the digits of a pass are
+// far from uniform (the first digit is sign and exponent, which almost all logits share), and
+// 1024 threads adding to one shared-memory word serialise; a lane's own copy is only ever touched
+// by the same lane of other warps and sits in its own bank.
 struct SfShared {
+  union {
+    float mass[256 * 32];
+    unsigned int cnt[256 * 32];
+  } lanes;
   float red_f[32];
   int red_i[32];
-  unsigned int hist[256];
-  float mass[256];
+  unsigned int hist[256];       // per digit: count (top-k pass) or "occupied" flag (nucleus pass)
+  float mass[256];              // per digit: probability mass
   float m, Z;
   unsigned int prefix;
   unsigned int k_left;
@@ -62,6 +70,32 @@ __device__ __forceinline__ float block_sum_f(float v, SfShared* sh) {
   return t;
 }
 
+// Calls f(logit, column) for every column of a row, each thread its share.  A row is read from L2
+// seven to eleven times by one CTA, so what counts is the bytes a thread keeps in flight: 16-byte
+// loads, two per thread at a time, when the row starts on a 16-byte boundary.
+template <typename F>
+__device__ __forceinline__ void for_each_logit(const float* __restrict__ l, int C, int tid, F f) {
+  if ((reinterpret_cast<uintptr_t>(l) & 15u) == 0) {
+    const float4* l4 = reinterpret_cast<const float4*>(l);
+    const int C4 = C >> 2;
+    int i = tid;
+    for (; i + kSfThreads < C4; i += 2 * kSfThreads) {
+      const float4 a = l4[i], b = l4[i + kSfThreads];
+      const int ca = 4 * i, cb = 4 * (i + kSfThreads);
+      f(a.x, ca); f(a.y, ca + 1); f(a.z, ca + 2); f(a.w, ca + 3);
+      f(b.x, cb); f(b.y, cb + 1); f(b.z, cb + 2); f(b.w, cb + 3);
+    }
+    for (; i < C4; i += kSfThreads) {
+      const float4 a = l4[i];
+      const int ca = 4 * i;
+      f(a.x, ca); f(a.y, ca + 1); f(a.z, ca + 2); f(a.w, ca + 3);
+    }
+    for (int c = (C4 << 2) + tid; c < C; c += kSfThreads) f(l[c], c);
+  } else {
+    for (int c = tid; c < C; c += kSfThreads) f(l[c], c);
+  }
+}
+
 }  // namespace
 
 __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __restrict__ logits, long long ld,
@@ -76,10 +110,10 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
   if (C <= 0) { if (tid == 0) { choice[r] = -1; if (kept) kept[r] = 0; } return; }
   // ---- 1. max and partition sum
   float mx = -INFINITY;
-  for (int c = tid; c < C; c += kSfThreads) mx = fmaxf(mx, l[c]);
+  for_each_logit(l, C, tid, [&](float x, int) { mx = fmaxf(mx, x); });
   mx = block_max(mx, &sh);
   float z = 0.f;
-  for (int c = tid; c < C; c += kSfThreads) z += expf((l[c] - mx) * inv_t);
+  for_each_logit(l, C, tid, [&](float x, int) { z += expf((x - mx) * inv_t); });
   z = block_sum_f(z, &sh);
   unsigned int key_k = 0u, key_p = 0u;
   // ---- 2. k-th largest logit by radix descent on counts
@@ -87,23 +121,44 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
     if (tid == 0) { sh.prefix = 0u; sh.k_left = (unsigned)top_k; }
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
-      if (tid < 256) sh.hist[tid] = 0u;
+      for (int i = tid; i < 256 * 32; i += kSfThreads) sh.lanes.cnt[i] = 0u;
       __syncthreads();
       const unsigned int prefix = sh.prefix;
-      for (int c = tid; c < C; c += kSfThreads) {
-        const uint32_t k = order_key(l[c]);
-        if (pass == 0 || (k >> (shift + 8)) == prefix) atomicAdd(&sh.hist[(k >> shift) & 255u], 1u);
+      for_each_logit(l, C, tid, [&](float x, int) {
+        const uint32_t k = order_key(x);
+        if (pass == 0 || (k >> (shift + 8)) == prefix) atomicAdd(&sh.lanes.cnt[((k >> shift) & 255u) * 32 + (tid & 31)], 1u);
+      });
+      __syncthreads();
+      for (int d = tid >> 5; d < 256; d += kSfThreads / 32) {          // a warp sums the 32 copies of a digit
+        const unsigned int v = __reduce_add_sync(0xffffffffu, sh.lanes.cnt[d * 32 + (tid & 31)]);
+        if ((tid & 31) == 0) sh.hist[d] = v;
       }
       __syncthreads();
-      if (tid == 0) {
-        unsigned int left = sh.k_left, d = 255u;
-        for (;; --d) {                                  // from the largest digit down
-          const unsigned int h = sh.hist[d];
-          if (h >= left || d == 0u) break;
-          left -= h;
+      if (tid < 32) {
+        // from the largest digit down: lane L holds digits 255 - 8 L .. 248 - 8 L; the digit in which
+        // the running count reaches what is left is the next digit of the k-th largest key
+        unsigned int h[8], mine = 0u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { h[j] = sh.hist[255 - 8 * tid - j]; mine += h[j]; }
+        unsigned int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (tid >= o) incl += t;
         }
-        sh.k_left = left;
-        sh.prefix = (prefix << 8) | d;
+        const unsigned int left = sh.k_left;
+        const unsigned int cross = __ballot_sync(0xffffffffu, incl >= left);
+        const int owner = cross ? __ffs(cross) - 1 : 31;           // never reached: the smallest digit
+        if (tid == owner) {
+          unsigned int rem = left - (incl - mine), d = 248u - 8u * (unsigned)tid;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (h[j] >= rem || (owner == 31 && j == 7)) { d = 255u - 8u * (unsigned)tid - (unsigned)j; break; }
+            rem -= h[j];
+          }
+          sh.k_left = rem;
+          sh.prefix = (prefix << 8) | d;
+        }
       }
       __syncthreads();
     }
@@ -115,31 +170,63 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
     if (tid == 0) { sh.prefix = 0u; sh.p_left = top_p * z; }
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
-      if (tid < 256) { sh.mass[tid] = 0.f; sh.hist[tid] = 0u; }
+      for (int i = tid; i < 256 * 32; i += kSfThreads) sh.lanes.mass[i] = 0.f;
+      if (tid < 256) sh.hist[tid] = 0u;
       __syncthreads();
       const unsigned int prefix = sh.prefix;
-      for (int c = tid; c < C; c += kSfThreads) {
-        const float x = l[c];
+      for_each_logit(l, C, tid, [&](float x, int) {
         const uint32_t k = order_key(x);
         if (pass == 0 || (k >> (shift + 8)) == prefix) {
-          atomicAdd(&sh.mass[(k >> shift) & 255u], expf((x - mx) * inv_t));
-          atomicAdd(&sh.hist[(k >> shift) & 255u], 1u);
+          const unsigned int d = (k >> shift) & 255u;
+          atomicAdd(&sh.lanes.mass[d * 32 + (tid & 31)], expf((x - mx) * inv_t));
+          sh.hist[d] = 1u;                                         // occupied (every writer stores 1)
         }
+      });
+      __syncthreads();
+      for (int d = tid >> 5; d < 256; d += kSfThreads / 32) {          // a warp sums the 32 copies of a digit
+        float v = sh.lanes.mass[d * 32 + (tid & 31)];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if ((tid & 31) == 0) sh.mass[d] = v;
       }
       __syncthreads();
-      if (tid == 0) {
-        float left = sh.p_left;
-        unsigned int d = 255u, last = 0u;
-        bool found = false;
-        for (int dd = 255; dd >= 0; --dd) {
-          if (sh.hist[dd] == 0u) continue;
-          last = (unsigned)dd;                            // the smallest occupied digit seen so far
-          if (sh.mass[dd] >= left) { d = (unsigned)dd; found = true; break; }
-          left -= sh.mass[dd];
+      if (tid < 32) {
+        // the same descent on probability mass (unoccupied digits hold none)
+        float h[8], mine = 0.f;
+        int low = 256;                                     // smallest occupied digit of this lane
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int d = 255 - 8 * tid - j;
+          h[j] = sh.mass[d]; mine += h[j];
+          if (sh.hist[d]) low = d;
         }
-        if (!found) d = last;                             // rounding: the mass ran out; keep everything here
-        sh.p_left = left;
-        sh.prefix = (prefix << 8) | d;
+        float incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const float t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (tid >= o) incl += t;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) low = min(low, __shfl_xor_sync(0xffffffffu, low, o));
+        const float left = sh.p_left;
+        // the owner is the first lane whose running mass reaches what is left AND that finds the
+        // digit inside itself (the sums of a lane and of its digits may round differently)
+        float rem = left - (incl - mine);
+        int dsel = -1;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (dsel < 0) {
+            if (h[j] >= rem && sh.hist[255 - 8 * tid - j]) dsel = 255 - 8 * tid - j;
+            else rem -= h[j];
+          }
+        }
+        const unsigned int cross = __ballot_sync(0xffffffffu, dsel >= 0);
+        if (cross) {
+          if (tid == __ffs(cross) - 1) { sh.p_left = rem; sh.prefix = (prefix << 8) | (unsigned)dsel; }
+        } else if (tid == 31) {                            // rounding: the mass ran out; keep everything here
+          sh.p_left = rem;
+          sh.prefix = (prefix << 8) | (unsigned)(low < 256 ? low : 0);
+        }
       }
       __syncthreads();
     }
@@ -149,14 +236,13 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
   // ---- 4. Gumbel-max over the kept columns (lowest index on ties)
   float best = -INFINITY;
   int best_c = 0x7fffffff, n_kept = 0;
-  for (int c = tid; c < C; c += kSfThreads) {
-    const float x = l[c];
-    if (order_key(x) < key_t) continue;
+  for_each_logit(l, C, tid, [&](float x, int c) {
+    if (order_key(x) < key_t) return;
     ++n_kept;
     const Philox4 px = philox4x32_10((uint32_t)(c >> 2), (uint32_t)(row_base + r), c2, c3, k0, k1);
     const float s = fmaf(x, inv_t, gumbel_from_word(philox_word(px, c & 3)));
     if (s > best || (s == best && c < best_c)) { best = s; best_c = c; }
-  }
+  });
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float ob = __shfl_xor_sync(0xffffffffu, best, o);

@@ -66,6 +66,26 @@ def test_filtered_sampling_matches_oracle(top_k, top_p, T):
     assert checked == 18 and exact >= (18 if top_p >= 1.0 else 0)
 
 
+@pytest.mark.parametrize("C", [37001, 4099, 5])
+def test_filtered_sampling_rows_that_start_off_a_16_byte_boundary(C):
+    # an odd row stride: rows 1.. take the scalar loads; rows whose length is no multiple of four
+    # take the ragged tail of the vector loads
+    rng = np.random.default_rng(13)
+    N = 4
+    l32 = (rng.standard_normal((N, C)) * 2.0).astype(np.float32)
+    n_cols = [C, C - 1, max(C - 2, 1), max(C - 3, 1)]
+    for top_k, top_p in ((9, 1.0), (0, 0.8), (1, 1.0)):
+        got, kept = _run(l32, n_cols, top_k, top_p, 0.9, 5, 2)
+        for r in range(N):
+            l = l32[r, :n_cols[r]].astype(np.float64)
+            a, keep, gap = olg.select_filtered(l, 0.9, top_k, top_p, 5, 2, r)
+            band = _band(l, 0.9, top_p)
+            assert abs(int(kept[r]) - int(keep.sum())) <= int(band.sum())
+            assert keep[got[r]] or band[got[r]]
+            if got[r] != a:
+                assert gap < GAP or band[got[r]] or band[a]
+
+
 def test_filtered_sampling_small_rows_and_frequencies():
     # tiny rows, exhaustively comparable; and frequencies over many steps against the renormalised distribution
     p = np.array([0.4, 0.25, 0.2, 0.1, 0.05])

@@ -4,7 +4,10 @@
 // they can be stored once (z2z_dynamic_logits with its full-logit output) and filtered here; the
 // fused argmax / Gumbel-max path of the logits kernels needs no stored logits.
 //
-// One CTA per row, every pass reads the row from L2 (16-byte loads, two in flight per thread):
+// A cluster of 1 to 8 CTAs per row (as many as keep all rows within one wave of the SMs); every
+// pass reads the row from L2 (16-byte loads, two in flight per thread), each CTA its share of the
+// columns, and the CTAs add up their maxima, sums and digit histograms through distributed shared
+// memory between two cluster barriers:
 //   1. m = max l,  Z = sum exp((l - m) / T);
 //   2. top-k: radix select (4 passes of 8 bits over order-preserving keys of the logits) of the
 //      k-th largest logit; everything >= it is kept (ties stay together);
@@ -14,6 +17,8 @@
 //      (Philox4x32-10 keyed by the seed, counter (column / 4, row, step), word column % 4).
 // The thresholds are found on the logits themselves, not on l / T: a positive scale preserves the
 // order, and equal logits stay exactly equal.
+#include <cooperative_groups.h>
+
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
 
@@ -39,8 +44,12 @@ struct SfShared {
   } lanes;
   float red_f[32];
   int red_i[32];
-  unsigned int hist[256];       // per digit: count (top-k pass) or "occupied" flag (nucleus pass)
-  float mass[256];              // per digit: probability mass
+  unsigned int hist[256];       // per digit, this CTA's columns: count (top-k pass) or "occupied" flag (nucleus pass)
+  float mass[256];              // per digit, this CTA's columns: probability mass
+  unsigned int tot_hist[256];   // the same over all CTAs that share the row
+  float tot_mass[256];
+  float xf[3];                  // what a CTA shows the others: max, partition sum, best score
+  int xi[2];                    // best column, kept columns
   float m, Z;
   unsigned int prefix;
   unsigned int k_left;
@@ -73,26 +82,27 @@ __device__ __forceinline__ float block_sum_f(float v, SfShared* sh) {
 // Calls f(logit, column) for every column of a row, each thread its share.  A row is read from L2
 // seven to eleven times by one CTA, so what counts is the bytes a thread keeps in flight: 16-byte
 // loads, two per thread at a time, when the row starts on a 16-byte boundary.
+// `t` is the thread's index among the `nt` threads that share the row (all CTAs of the cluster).
 template <typename F>
-__device__ __forceinline__ void for_each_logit(const float* __restrict__ l, int C, int tid, F f) {
+__device__ __forceinline__ void for_each_logit(const float* __restrict__ l, int C, int t, int nt, F f) {
   if ((reinterpret_cast<uintptr_t>(l) & 15u) == 0) {
     const float4* l4 = reinterpret_cast<const float4*>(l);
     const int C4 = C >> 2;
-    int i = tid;
-    for (; i + kSfThreads < C4; i += 2 * kSfThreads) {
-      const float4 a = l4[i], b = l4[i + kSfThreads];
-      const int ca = 4 * i, cb = 4 * (i + kSfThreads);
+    int i = t;
+    for (; i + nt < C4; i += 2 * nt) {
+      const float4 a = l4[i], b = l4[i + nt];
+      const int ca = 4 * i, cb = 4 * (i + nt);
       f(a.x, ca); f(a.y, ca + 1); f(a.z, ca + 2); f(a.w, ca + 3);
       f(b.x, cb); f(b.y, cb + 1); f(b.z, cb + 2); f(b.w, cb + 3);
     }
-    for (; i < C4; i += kSfThreads) {
+    for (; i < C4; i += nt) {
       const float4 a = l4[i];
       const int ca = 4 * i;
       f(a.x, ca); f(a.y, ca + 1); f(a.z, ca + 2); f(a.w, ca + 3);
     }
-    for (int c = (C4 << 2) + tid; c < C; c += kSfThreads) f(l[c], c);
+    for (int c = (C4 << 2) + t; c < C; c += nt) f(l[c], c);
   } else {
-    for (int c = tid; c < C; c += kSfThreads) f(l[c], c);
+    for (int c = t; c < C; c += nt) f(l[c], c);
   }
 }
 
@@ -104,17 +114,28 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
                                                                 uint32_t c2, uint32_t c3, int row_base,
                                                                 int32_t* __restrict__ choice, int32_t* __restrict__ kept) {
   __shared__ SfShared sh;
-  const int r = blockIdx.x, tid = threadIdx.x;
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int G = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();     // CTAs that share the row
+  const int r = blockIdx.x / G, tid = threadIdx.x;
+  const int gt = rank * kSfThreads + tid, gnt = G * kSfThreads;
   const int C = n_cols[r];
   const float* l = logits + (size_t)r * ld;
-  if (C <= 0) { if (tid == 0) { choice[r] = -1; if (kept) kept[r] = 0; } return; }
+  if (C <= 0) { if (tid == 0 && rank == 0) { choice[r] = -1; if (kept) kept[r] = 0; } return; }   // (the whole cluster returns)
   // ---- 1. max and partition sum
   float mx = -INFINITY;
-  for_each_logit(l, C, tid, [&](float x, int) { mx = fmaxf(mx, x); });
+  for_each_logit(l, C, gt, gnt, [&](float x, int) { mx = fmaxf(mx, x); });
   mx = block_max(mx, &sh);
+  if (tid == 0) sh.xf[0] = mx;
+  cluster.sync();
+  for (int g = 0; g < G; ++g) mx = fmaxf(mx, *cluster.map_shared_rank(&sh.xf[0], g));
   float z = 0.f;
-  for_each_logit(l, C, tid, [&](float x, int) { z += expf((x - mx) * inv_t); });
+  for_each_logit(l, C, gt, gnt, [&](float x, int) { z += expf((x - mx) * inv_t); });
   z = block_sum_f(z, &sh);
+  if (tid == 0) sh.xf[1] = z;
+  cluster.sync();
+  z = 0.f;
+  for (int g = 0; g < G; ++g) z += *cluster.map_shared_rank(&sh.xf[1], g);        // same order in every CTA
   unsigned int key_k = 0u, key_p = 0u;
   // ---- 2. k-th largest logit by radix descent on counts
   if (top_k > 0 && top_k < C) {
@@ -124,7 +145,7 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
       for (int i = tid; i < 256 * 32; i += kSfThreads) sh.lanes.cnt[i] = 0u;
       __syncthreads();
       const unsigned int prefix = sh.prefix;
-      for_each_logit(l, C, tid, [&](float x, int) {
+      for_each_logit(l, C, gt, gnt, [&](float x, int) {
         const uint32_t k = order_key(x);
         if (pass == 0 || (k >> (shift + 8)) == prefix) atomicAdd(&sh.lanes.cnt[((k >> shift) & 255u) * 32 + (tid & 31)], 1u);
       });
@@ -133,13 +154,20 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
         const unsigned int v = __reduce_add_sync(0xffffffffu, sh.lanes.cnt[d * 32 + (tid & 31)]);
         if ((tid & 31) == 0) sh.hist[d] = v;
       }
-      __syncthreads();
+      cluster.sync();                                    // every CTA's digit counts are in place
+      if (tid < 256) {
+        unsigned int v = 0u;
+        for (int g = 0; g < G; ++g) v += *cluster.map_shared_rank(&sh.hist[tid], g);
+        sh.tot_hist[tid] = v;
+      }
+      cluster.sync();                                    // ... and have been read by everyone
       if (tid < 32) {
         // from the largest digit down: lane L holds digits 255 - 8 L .. 248 - 8 L; the digit in which
-        // the running count reaches what is left is the next digit of the k-th largest key
+        // the running count reaches what is left is the next digit of the k-th largest key (every
+        // CTA of the cluster takes the same decision from the same sums)
         unsigned int h[8], mine = 0u;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { h[j] = sh.hist[255 - 8 * tid - j]; mine += h[j]; }
+        for (int j = 0; j < 8; ++j) { h[j] = sh.tot_hist[255 - 8 * tid - j]; mine += h[j]; }
         unsigned int incl = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -174,7 +202,7 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
       if (tid < 256) sh.hist[tid] = 0u;
       __syncthreads();
       const unsigned int prefix = sh.prefix;
-      for_each_logit(l, C, tid, [&](float x, int) {
+      for_each_logit(l, C, gt, gnt, [&](float x, int) {
         const uint32_t k = order_key(x);
         if (pass == 0 || (k >> (shift + 8)) == prefix) {
           const unsigned int d = (k >> shift) & 255u;
@@ -189,7 +217,17 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         if ((tid & 31) == 0) sh.mass[d] = v;
       }
-      __syncthreads();
+      cluster.sync();                                    // every CTA's digit masses are in place
+      if (tid < 256) {
+        float v = 0.f;
+        unsigned int occ = 0u;
+        for (int g = 0; g < G; ++g) {
+          v += *cluster.map_shared_rank(&sh.mass[tid], g);
+          occ |= *cluster.map_shared_rank(&sh.hist[tid], g);
+        }
+        sh.tot_mass[tid] = v; sh.tot_hist[tid] = occ;
+      }
+      cluster.sync();                                    // ... and have been read by everyone
       if (tid < 32) {
         // the same descent on probability mass (unoccupied digits hold none)
         float h[8], mine = 0.f;
@@ -197,8 +235,8 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int d = 255 - 8 * tid - j;
-          h[j] = sh.mass[d]; mine += h[j];
-          if (sh.hist[d]) low = d;
+          h[j] = sh.tot_mass[d]; mine += h[j];
+          if (sh.tot_hist[d]) low = d;
         }
         float incl = mine;
 #pragma unroll
@@ -216,7 +254,7 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           if (dsel < 0) {
-            if (h[j] >= rem && sh.hist[255 - 8 * tid - j]) dsel = 255 - 8 * tid - j;
+            if (h[j] >= rem && sh.tot_hist[255 - 8 * tid - j]) dsel = 255 - 8 * tid - j;
             else rem -= h[j];
           }
         }
@@ -236,7 +274,7 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
   // ---- 4. Gumbel-max over the kept columns (lowest index on ties)
   float best = -INFINITY;
   int best_c = 0x7fffffff, n_kept = 0;
-  for_each_logit(l, C, tid, [&](float x, int c) {
+  for_each_logit(l, C, gt, gnt, [&](float x, int c) {
     if (order_key(x) < key_t) return;
     ++n_kept;
     const Philox4 px = philox4x32_10((uint32_t)(c >> 2), (uint32_t)(row_base + r), c2, c3, k0, k1);
@@ -262,8 +300,21 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
       n_kept += __shfl_xor_sync(0xffffffffu, n_kept, o);
       if (ob > best || (ob == best && oc < best_c)) { best = ob; best_c = oc; }
     }
-    if (tid == 0) { choice[r] = best_c == 0x7fffffff ? -1 : best_c; if (kept) kept[r] = n_kept; }
+    if (tid == 0) { sh.xf[2] = best; sh.xi[0] = best_c; sh.xi[1] = n_kept; }
   }
+  cluster.sync();
+  if (rank == 0 && tid == 0) {
+    best = -INFINITY; best_c = 0x7fffffff; n_kept = 0;
+    for (int g = 0; g < G; ++g) {
+      const float ob = *cluster.map_shared_rank(&sh.xf[2], g);
+      const int oc = *cluster.map_shared_rank(&sh.xi[0], g);
+      n_kept += *cluster.map_shared_rank(&sh.xi[1], g);
+      if (ob > best || (ob == best && oc < best_c)) { best = ob; best_c = oc; }
+    }
+    choice[r] = best_c == 0x7fffffff ? -1 : best_c;
+    if (kept) kept[r] = n_kept;
+  }
+  cluster.sync();                                        // no CTA leaves while its shared memory may be read
 }
 
 }  // namespace z2z
@@ -278,10 +329,24 @@ extern "C" int32_t z2z_sample_filtered(const float* d_logits, int32_t N, int64_t
   if (!(temperature > 0.f)) return fail("sampling needs temperature > 0");
   if (!(top_p > 0.f)) return fail("top_p must be > 0 (>= 1: no nucleus filter)");
   if (ld < 1) return fail("ld < 1");
-  z2z::k_sample_filtered<<<N, z2z::kSfThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      d_logits, (long long)ld, d_n_cols, top_k, top_p, 1.0f / temperature, (uint32_t)seed, (uint32_t)(seed >> 32),
-      (uint32_t)step, (uint32_t)(step >> 32), row_base, d_choice, d_kept);
-  cudaError_t e = cudaGetLastError();
+  // a decode batch has far fewer rows than the GPU has SMs, and one SM reads a row from L2 at a
+  // fraction of what the row's passes need: a cluster of G CTAs shares a row (G x N CTAs stay
+  // within one wave of the 148 SMs)
+  int G = 1;
+  while (G < 8 && (long long)N * (2 * G) <= 148) G *= 2;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((unsigned)N * (unsigned)G);
+  lc.blockDim = dim3(z2z::kSfThreads);
+  lc.dynamicSmemBytes = 0;
+  lc.stream = reinterpret_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)G; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  lc.attrs = at; lc.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&lc, z2z::k_sample_filtered, d_logits, (long long)ld, d_n_cols, top_k, top_p,
+                                     1.0f / temperature, (uint32_t)seed, (uint32_t)(seed >> 32), (uint32_t)step,
+                                     (uint32_t)(step >> 32), row_base, d_choice, d_kept);
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { z2z::set_last_error(cudaGetErrorString(e)); return Z2Z_ERR_CUDA; }
   return Z2Z_OK;
 }

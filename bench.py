@@ -667,6 +667,17 @@ def run_helpers(args):
         ms = best_ms(lambda: zb.z2z_sample_filtered(logits, n_cols, k, p, 0.8, 7, 3, choice, kept))
         out["sample_filtered_" + name] = {"us": ms * 1e3, "rows": w.B, "columns": int(n_cols.max().item()),
                                           "kept_mean": float(kept.float().mean().item())}
+    # the joint logits of one decode batch with the reductions only, and with every logit stored
+    # (what filtered sampling needs beforehand)
+    hid = si.make_hidden(w, w.B, 9).to(dev)
+    W_U = si.normal_tensor((w.V, w.d), 0.02, 10, w.torch_dtype).to(dev)
+    lse = torch.zeros(w.B, dtype=torch.float32, device=dev)
+    amax = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    mxl = torch.zeros(w.B, dtype=torch.float32, device=dev)
+    for name, store in (("logits_reductions_only", None), ("logits_stored", logits)):
+        ms = best_ms(lambda: zb.z2z_dynamic_logits(cb, hid, None, None, W_U, E_h, zb.SELECT_ARGMAX, 1.0, 0, 0, None,
+                                                   lse, amax, mxl, None, None, store))
+        out[name] = {"us": ms * 1e3, "rows": w.B}
     line = {"helpers": out, "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "T": w.T, "M": w.M,
                                        "cap": w.cap}, "data": "synthetic",
             "peak_hbm_gbs": pk["hbm_gbs"], "peak_source": pk["source"]}

@@ -86,6 +86,25 @@ def test_filtered_sampling_rows_that_start_off_a_16_byte_boundary(C):
                 assert gap < GAP or band[got[r]] or band[a]
 
 
+@pytest.mark.parametrize("N", [20, 40, 80])
+def test_filtered_sampling_with_every_cluster_size(N):
+    # the rows of a batch share the SMs: 20, 40 and 80 rows are worked on by clusters of 4, 2 and
+    # 1 CTAs per row (up to 9 rows by clusters of 8, as in the tests above)
+    rng = np.random.default_rng(17 + N)
+    C = 9001
+    l32 = (rng.standard_normal((N, C)) * 2.0).astype(np.float32)
+    n_cols = [C - (r % 7) for r in range(N)]
+    got, kept = _run(l32, n_cols, 30, 0.9, 1.1, 21, 4, row_base=3)
+    for r in range(N):
+        l = l32[r, :n_cols[r]].astype(np.float64)
+        a, keep, gap = olg.select_filtered(l, 1.1, 30, 0.9, 21, 4, 3 + r)
+        band = _band(l, 1.1, 0.9)
+        assert abs(int(kept[r]) - int(keep.sum())) <= int(band.sum())
+        assert keep[got[r]] or band[got[r]]
+        if got[r] != a:
+            assert gap < GAP or band[got[r]] or band[a]
+
+
 def test_filtered_sampling_small_rows_and_frequencies():
     # tiny rows, exhaustively comparable; and frequencies over many steps against the renormalised distribution
     p = np.array([0.4, 0.25, 0.2, 0.1, 0.05])

@@ -8,7 +8,7 @@
 // pass reads the row from L2 (16-byte loads, two in flight per thread), each CTA its share of the
 // columns, and the CTAs add up their maxima, sums and digit histograms through distributed shared
 // memory between two cluster barriers:
-//   1. m = max l,  Z = sum exp((l - m) / T);
+//   1. m = max l,  Z = sum exp((l - m) / T), in one pass and only when a nucleus is asked for;
 //   2. top-k: radix select (4 passes of 8 bits over order-preserving keys of the logits) of the
 //      k-th largest logit; everything >= it is kept (ties stay together);
 //   3. top-p: the same descent weighted by probability mass: the largest logit v with
@@ -122,20 +122,27 @@ __global__ void __launch_bounds__(kSfThreads) k_sample_filtered(const float* __r
   const int C = n_cols[r];
   const float* l = logits + (size_t)r * ld;
   if (C <= 0) { if (tid == 0 && rank == 0) { choice[r] = -1; if (kept) kept[r] = 0; } return; }   // (the whole cluster returns)
-  // ---- 1. max and partition sum
-  float mx = -INFINITY;
-  for_each_logit(l, C, gt, gnt, [&](float x, int) { mx = fmaxf(mx, x); });
-  mx = block_max(mx, &sh);
-  if (tid == 0) sh.xf[0] = mx;
-  cluster.sync();
-  for (int g = 0; g < G; ++g) mx = fmaxf(mx, *cluster.map_shared_rank(&sh.xf[0], g));
-  float z = 0.f;
-  for_each_logit(l, C, gt, gnt, [&](float x, int) { z += expf((x - mx) * inv_t); });
-  z = block_sum_f(z, &sh);
-  if (tid == 0) sh.xf[1] = z;
-  cluster.sync();
-  z = 0.f;
-  for (int g = 0; g < G; ++g) z += *cluster.map_shared_rank(&sh.xf[1], g);        // same order in every CTA
+  // ---- 1. max and partition sum in one pass (running maximum, sum rescaled when it moves); only
+  //         the nucleus filter needs them
+  float mx = 0.f, z = 0.f;
+  if (top_p < 1.0f) {
+    float m = -INFINITY, sum = 0.f;
+    for_each_logit(l, C, gt, gnt, [&](float x, int) {
+      if (x > m) { sum = sum * expf((m - x) * inv_t) + 1.f; m = x; }
+      else if (m > -INFINITY) sum += expf((x - m) * inv_t);     // (-inf logits before any finite one add nothing)
+    });
+    const float m_cta = block_max(m, &sh);
+    // (a thread, or further down a CTA, without columns has m = -inf and adds nothing)
+    const float s_cta = block_sum_f(m > -INFINITY ? sum * expf((m - m_cta) * inv_t) : 0.f, &sh);
+    if (tid == 0) { sh.xf[0] = m_cta; sh.xf[1] = s_cta; }
+    cluster.sync();
+    mx = m_cta;
+    for (int g = 0; g < G; ++g) mx = fmaxf(mx, *cluster.map_shared_rank(&sh.xf[0], g));
+    for (int g = 0; g < G; ++g) {                                                 // same order in every CTA
+      const float m_g = *cluster.map_shared_rank(&sh.xf[0], g);
+      if (m_g > -INFINITY) z += *cluster.map_shared_rank(&sh.xf[1], g) * expf((m_g - mx) * inv_t);
+    }
+  }
   unsigned int key_k = 0u, key_p = 0u;
   // ---- 2. k-th largest logit by radix descent on counts
   if (top_k > 0 && top_k < C) {

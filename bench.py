@@ -1,24 +1,36 @@
 #!/usr/bin/env python
-"""Benchmark of the dynamic-vocabulary decode step (LZW update + hyper-encoder + joint logits).
+"""Benchmark of the dynamic-vocabulary path (LZW update + hyper-encoder + joint logits).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-One "step" is one z2z_decode_step over a batch of B sequences of the workload (default: the
-Phi-3-mini-shaped head, the configuration the headline metric is quoted on): joint logits and
-selection, online LZW update with the selected code, hyper-encoder on the new entry of each
-sequence for both caches.  The prompts are compressed and their entries embedded before the timed
-region (session set-up).  Prints ONE JSON line.
+One "step" of a decode workload is one z2z_decode_step over its batch of B sequences: joint
+logits and selection, online LZW update with the selected code, hyper-encoder on the new entry of
+each sequence for both caches.  The prompts are compressed and their entries embedded before the
+timed region (session set-up).  The default workload is the Llama-3-8B-shaped head, the largest
+decode configuration that fits one GPU; with no `--workload` given on one GPU the same JSON line
+also carries a `per_workload` object with the other bf16 configurations (Phi-3-mini-shaped head,
+long context, and the prompt-scoring configuration at its full 64 prompts), each with its own step
+time, roofline figures, end-to-end figure and clocks.  Prints ONE JSON line.
+
+Timed regions.  A region is EXACTLY K steps between two CUDA events, bracketed by a barrier and a
+device synchronise.  A decode step takes a fraction of a millisecond, so when K steps cover less
+than 0.3 s the region is repeated (on fresh hidden states, the session simply goes on decoding)
+until that much time is covered; `ms_per_step` and `value` are those of the MEDIAN region, the
+spread is reported beside them, and the clock sampler runs over all of them.
 
 `--impl reference` times the CPU oracle (oracle/) as it stands on the host cores, on a bounded
-sample of the same workload.  With N > 1 ranks each rank runs an independent replica of the
-workload (the path has no exchange step); the value is the sum over ranks.
+sample of the same workload.  With `--gpus N` each of N ranks runs an independent replica of the
+workload (the path has no exchange step); times are the maximum over ranks, token counts the sum.
+When the launcher's environment (WORLD_SIZE) is absent, `--gpus N` starts the N ranks itself.
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
+import math
 import os
-import subprocess
+import socket
 import sys
 import threading
 import time
@@ -34,6 +46,10 @@ from paper_2506_01084_b200 import synth_inputs as si  # noqa: E402
 
 METRIC = "base-token-equiv decode tok/s (LZW+hyper-embed+logits)"
 UNIT = "base tokens/s"
+DEFAULT_WORKLOAD = "llama3_8b_head"
+SUB_WORKLOADS = ("phi3_mini_head", "long_context", "prefill_heavy")
+MIN_TIMED_S = 0.3            # a K-step region is repeated until this much device time is covered
+MAX_REGIONS = 200
 
 
 def peaks():
@@ -50,7 +66,7 @@ def peaks():
 class ClockSampler:
     """Samples SM clocks and clock-event (throttle) reasons through NVML, the library nvidia-smi
     itself reads, from a thread while the timed region runs (nvidia-smi's own loop cannot sample
-    faster than its start-up time, and the timed region may last only tens of milliseconds).
+    faster than its start-up time, and a timed region lasts a fraction of a second).
     Reading only: nothing is set."""
 
     def __init__(self, index: int, period_s: float = 0.004):
@@ -102,7 +118,8 @@ class ClockSampler:
                  "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
         reasons = sorted(k for k, bit in names.items() if any(r & bit for _, r, _ in self.samples))
         sm = [m for m, _, _ in self.samples if m > 0]
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": self.max_mhz,
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_mhz_min": float(min(sm)) if sm else None, "sm_max_mhz": self.max_mhz,
                 "reasons": reasons, "samples": len(sm),
                 "power_w_max": max((p for _, _, p in self.samples), default=None)}
 
@@ -110,7 +127,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # algorithmic bytes of one decode step (what the kernels must move at minimum)
 # --------------------------------------------------------------------------------------------------
-def logits_bytes(w: si.Workload, n_hyper_total: int) -> float:
+def logits_bytes(w: si.Workload, n_hyper_total: float) -> float:
     """W_U once + every visible hyper-unembedding row once + hidden rows (bf16 = 2 B)."""
     es = 2 if w.dtype == "bf16" else 4
     return es * (w.V * w.d + n_hyper_total * w.d + w.B * w.d)
@@ -139,6 +156,52 @@ def reduce_over_ranks(times_ms, counts, world: int, device):
     cc = torch.tensor(list(counts), device=device, dtype=torch.float64)
     torch.distributed.all_reduce(cc, op=torch.distributed.ReduceOp.SUM)
     return tt.tolist(), cc.tolist()
+
+
+def plan_regions(K: int, est_ms_per_step: float, steps_available: int, min_s: float = MIN_TIMED_S) -> int:
+    """Number of K-step regions: enough to cover `min_s` of device time at the estimated step
+    time, at most what the session's remaining codebook room (in steps) allows, at least one."""
+    want = int(math.ceil(min_s * 1e3 / max(K * est_ms_per_step, 1e-6)))
+    room = max(1, steps_available // max(K, 1))
+    return max(1, min(want, room, MAX_REGIONS))
+
+
+# --------------------------------------------------------------------------------------------------
+# synthetic inputs shared between the workloads of one run (same seed and shape -> same tensor)
+# --------------------------------------------------------------------------------------------------
+class Inputs:
+    """Generated weights, kept on the host and on the device and keyed by what determines their
+    values, so that workloads with the same table and encoder shapes do not draw (or upload) them
+    again: three of the configurations share V and d and differ only in the position table."""
+
+    def __init__(self, dev):
+        self.dev, self.host, self.gpu = dev, {}, {}
+
+    def tables(self, w, seed):
+        key = ("tables", w.V, w.d, w.dtype, w.tied, seed)
+        if key not in self.host:
+            self.host[key] = si.make_tables(w, seed)
+        return self.host[key]
+
+    def encoder(self, w, seed):
+        key = ("enc", w.d, w.dff, w.enc_layers, w.dtype, seed)
+        if key not in self.host:
+            self.host[key] = si.make_encoder(w, seed)             # pos belongs to this w.M
+            self.host[key + ("M",)] = w.M
+        if self.host[key + ("M",)] == w.M:
+            return self.host[key]
+        # same seed and shapes except pos[M, d]: only that tensor is drawn again (tensor i of the
+        # list depends on the seed and on i alone); kept, so that its device copy stays valid
+        pkey = key + ("pos", w.M)
+        if pkey not in self.host:
+            self.host[pkey] = si.normal_tensor((w.M, w.d), 0.02, seed * 131 + 0, w.torch_dtype)
+        return [self.host[pkey]] + list(self.host[key][1:])
+
+    def to_dev(self, t):
+        key = (t.data_ptr(), tuple(t.shape))
+        if key not in self.gpu:
+            self.gpu[key] = t.to(self.dev)
+        return self.gpu[key]
 
 
 def forced_codes(zb, w, cb, dev, stream, prompt_code_lens, n_steps: int):
@@ -200,40 +263,51 @@ def ncu_traffic(kernel_class: str, workload: str):
     return None
 
 
-# --------------------------------------------------------------------------------------------------
-# our arm
-# --------------------------------------------------------------------------------------------------
-def run_ours(args, rank: int, world: int):
-    from paper_2506_01084_b200 import binding as zb
-    zb.lib()                                  # fail loudly if the CUDA library is missing
+def _local_device():
     dev = torch.device(f"cuda:{int(os.environ.get('LOCAL_RANK', 0))}")
     torch.cuda.set_device(dev)
-    w = si.WORKLOADS[args.workload]
-    if w.steps == 0:
-        raise SystemExit("this workload has no decode steps; use tests for the prefill path")
+    return dev
+
+
+def _barrier(world):
+    if world > 1:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+
+
+# --------------------------------------------------------------------------------------------------
+# decode workloads
+# --------------------------------------------------------------------------------------------------
+def run_decode(args, w: si.Workload, inputs: Inputs, rank: int, world: int):
+    from paper_2506_01084_b200 import binding as zb
+    zb.lib()                                  # fail loudly if the CUDA library is missing
+    dev = inputs.dev
     K, Wm = args.steps, args.warmup
+    Ka = min(K, 128)                          # steps of the per-kernel, end-to-end and sampling passes
     seed = replica_seed(rank)
     forced_mode = args.decode_mode == "forced"
-    n_steps_total = Wm + 3 * K                # warm-up, device-timed, per-kernel-timed, end-to-end
+    n_probe = 8
+    # hidden states for every step that may run: regions are planned after the warm-up, bounded here
+    # (a step cannot be faster than its algorithmic bytes at 8 TB/s, which bounds the steps 0.3 s can hold)
+    floor_s = (logits_bytes(w, 0) + encoder_gemm_bytes(w)) / 8e12
+    max_steps = Wm + n_probe + 3 * Ka + min(K * MAX_REGIONS, int(MIN_TIMED_S / floor_s) + 2 * K, max(K, int(w.cap)))
     if forced_mode:
-        # one generator stream per sequence: its first T tokens are the prompt, the rest is the
-        # continuation whose LZW codes are fed to the steps (at most M tokens per code)
-        stream = si.make_tokens(w, seed, T=w.T + n_steps_total * w.M + 64)
+        stream = si.make_tokens(w, seed, T=w.T + max_steps * w.M + 64)
         tokens = np.ascontiguousarray(stream[:, :w.T])
     else:
         stream = None
         tokens = si.make_tokens(w, seed)
-    W_E, W_U = si.make_tables(w, seed)
-    encE_t = [t.to(dev) for t in si.make_encoder(w, seed * 3 + 1)]
-    encU_t = encE_t if w.tied else [t.to(dev) for t in si.make_encoder(w, seed * 3 + 2)]
-    g_WE = W_E.to(dev)
-    g_WU = g_WE if w.tied else W_U.to(dev)
+    W_E, W_U = inputs.tables(w, seed)
+    encE_t = [inputs.to_dev(t) for t in inputs.encoder(w, seed * 3 + 1)]
+    encU_t = encE_t if w.tied else [inputs.to_dev(t) for t in inputs.encoder(w, seed * 3 + 2)]
+    g_WE = inputs.to_dev(W_E)
+    g_WU = g_WE if w.tied else inputs.to_dev(W_U)
     cfg = zb.make_config(w.V, w.d, w.M, w.cap, w.B, w.dtype, w.enc_layers, w.heads, w.dff, w.tied)
     cb = zb.Codebook(cfg, dev)
     encE, encU = zb.encoder_weights(encE_t), zb.encoder_weights(encU_t)
     E_h = torch.zeros(w.B, w.cap, w.d, dtype=w.torch_dtype, device=dev)
     U_h = E_h if w.tied else torch.zeros_like(E_h)
-    hidden_host = si.make_hidden(w, n_steps_total * w.B, seed).view(n_steps_total, w.B, w.d).pin_memory()
+    hidden_host = si.make_hidden(w, max_steps * w.B, seed).view(max_steps, w.B, w.d).pin_memory()
     hidden = hidden_host.to(dev)
 
     # ---- session set-up (not timed as steps; reported separately) ----
@@ -252,7 +326,7 @@ def run_ours(args, rank: int, world: int):
     torch.cuda.synchronize()
     forced_dev = None
     if forced_mode:
-        forced_dev = forced_codes(zb, w, cb, dev, stream, clen, n_steps_total)
+        forced_dev = forced_codes(zb, w, cb, dev, stream, clen, max_steps)
         # the session now holds the codebook of the prompt's codes but the last (replayed from the
         # stream's own codes, so that the continuation's codes name its entries): embed them again
         E_h.zero_(); U_h.zero_()
@@ -265,43 +339,62 @@ def run_ours(args, rank: int, world: int):
                "prompt_tokens": int(w.B * w.T), "compressed_tokens": int(clen.sum().item()),
                "hypertokens": int(n0.sum().item())}
 
-    nxt_all = torch.zeros(n_steps_total, w.B, dtype=torch.int32, device=dev)
+    nxt_all = torch.zeros(max_steps, w.B, dtype=torch.int32, device=dev)
     lse = torch.zeros(w.B, dtype=torch.float32, device=dev)
+    cursor = [0]                               # next unused step (hidden row block, sampling step)
 
-    def step(t, hid):
-        zb.z2z_decode_step(cb, hid, g_WE, g_WU, encE, encU, E_h, U_h, zb.SELECT_ARGMAX, 1.0, 0, t,
+    def step(t, select=None):
+        zb.z2z_decode_step(cb, hidden[t], g_WE, g_WU, encE, encU, E_h, U_h,
+                           zb.SELECT_ARGMAX if select is None else select, 1.0, 0, t,
                            None if forced_dev is None else forced_dev[t], nxt_all[t], None, lse)
 
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
+    def run_steps(n, select=None):
+        t0 = cursor[0]
+        for t in range(t0, t0 + n):
+            step(t, select)
+        cursor[0] = t0 + n
+        return t0
 
-    for t in range(Wm):
-        step(t, hidden[t])
+    def timed(n, select=None):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        _barrier(world)
+        e0.record()
+        t0 = run_steps(n, select)
+        e1.record()
+        _barrier(world)
+        return e0.elapsed_time(e1), t0
+
+    run_steps(Wm)
+    est_ms, _ = timed(n_probe)
+    est_ms /= n_probe
+    # room: every step may add one entry per sequence; once all codebooks are full the encoder
+    # pass is no longer launched and a step is a different (cheaper) thing
+    _, n_now = zb.z2z_status(cb)
+    room_steps = int(w.cap - int(n_now.max().item())) - 3 * Ka - 1
+    room_steps = min(room_steps, max_steps - cursor[0] - 3 * Ka)
+    R = plan_regions(K, est_ms, room_steps)
+    if world > 1:                              # every rank runs the same number of regions
+        rr = torch.tensor([R], device=dev, dtype=torch.int64)
+        torch.distributed.all_reduce(rr, op=torch.distributed.ReduceOp.MIN)
+        R = int(rr.item())
     zb.z2z_profile_read(cb)                    # reset launch counters
 
-    # ---- device-timed region: inputs resident in HBM ----
+    # ---- device-timed regions: inputs resident in HBM ----
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
-    barrier()
     n_before = zb.z2z_status(cb)[1].sum().item()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for t in range(Wm, Wm + K):
-        step(t, hidden[t])
-    e1.record()
-    barrier()
-    dev_ms = e0.elapsed_time(e1)
+    regions = []
+    for _ in range(R):
+        ms, t0 = timed(K)
+        regions.append((ms, t0))
     clocks = sampler.stop()
     _, launches = zb.z2z_profile_read(cb)
+    launches = {k: v / R for k, v in launches.items()}          # per K-step region
     n_after = zb.z2z_status(cb)[1].sum().item()
 
-    # ---- same K steps again with per-kernel-class events (for the roofline numbers) ----
+    # ---- Ka steps again with per-kernel-class events (for the roofline numbers) ----
     zb.z2z_profile(cb, True)
-    for t in range(Wm + K, Wm + 2 * K):
-        step(t, hidden[t])
+    run_steps(Ka)
     zb.z2z_profile(cb, False)
     cls_ms, cls_launches = zb.z2z_profile_read(cb)
     n_after2 = zb.z2z_status(cb)[1].sum().item()
@@ -310,15 +403,16 @@ def run_ours(args, rank: int, world: int):
     out_host = torch.zeros(w.B, dtype=torch.int32).pin_memory()
     lse_host = torch.zeros(w.B, dtype=torch.float32).pin_memory()
     hid_dev = torch.empty(w.B, w.d, dtype=w.torch_dtype, device=dev)
-    barrier()
-    t0 = time.perf_counter()
+    _barrier(world)
+    t_start = time.perf_counter()
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record()
-    nx_e2e = np.zeros((K, w.B), dtype=np.int32)
+    nx_e2e = np.zeros((Ka, w.B), dtype=np.int32)
     out_np, lse_np = out_host.numpy(), lse_host.numpy()
     out_np[:] = -1
     lse_np[:] = np.nan
-    for i, t in enumerate(range(Wm + 2 * K, Wm + 3 * K)):
+    t_first = cursor[0]
+    for i, t in enumerate(range(t_first, t_first + Ka)):
         zb.z2z_upload_rows(hidden_host[t], hid_dev)    # host -> device by a kernel the logits kernel overlaps
         # the applied codes and the LSE go straight into pinned host memory: the result pointers of
         # the call may be host memory that is mapped into the device's address space, so the
@@ -335,10 +429,14 @@ def run_ours(args, rank: int, world: int):
         nx_e2e[i] = out_np
         out_np[:] = -1
         lse_np[:] = np.nan
+    cursor[0] = t_first + Ka
     torch.cuda.current_stream().synchronize()
     e3.record()
-    barrier()
-    e2e_ms = max(e2.elapsed_time(e3), (time.perf_counter() - t0) * 1e3)
+    _barrier(world)
+    e2e_ms = max(e2.elapsed_time(e3), (time.perf_counter() - t_start) * 1e3)
+
+    # ---- the same step with Gumbel-max sampling instead of argmax (Section 2.3 step 9) ----
+    smp_ms, smp_t0 = timed(Ka, zb.SELECT_GUMBEL)
 
     # ---- base-token equivalents of what was emitted ----
     stt, n_fin = zb.z2z_status(cb)
@@ -355,19 +453,25 @@ def run_ours(args, rank: int, world: int):
             tot += int(np.where(z < w.V, 1, lens[b][np.clip(z - w.V, 0, w.cap - 1)]).sum())
         return tot
 
-    bt_dev = base_tokens(nx[Wm:Wm + K])
+    order = sorted(range(R), key=lambda i: regions[i][0])
+    med = order[(R - 1) // 2]                                    # the median region (lower one of two)
+    dev_ms, t_med = regions[med]
+    bt_dev = base_tokens(nx[t_med:t_med + K])
     bt_e2e = base_tokens(nx_e2e)
+    bt_smp = base_tokens(nx[smp_t0:smp_t0 + Ka])
     bad = int(sum(1 for s in stt.tolist() if s & (zb.ST_BAD_TOKEN | zb.ST_TABLE_FULL | zb.ST_WAIT_TIMEOUT)))
+    all_ms = [r[0] for r in regions]
 
     # ---- reduce over ranks: max time, summed tokens ----
-    (dev_ms, e2e_ms), (bt_dev, bt_e2e) = reduce_over_ranks([dev_ms, e2e_ms], [bt_dev, bt_e2e], world, dev)
+    (dev_ms, e2e_ms, smp_ms, ms_min, ms_max), (bt_dev, bt_e2e, bt_smp) = reduce_over_ranks(
+        [dev_ms, e2e_ms, smp_ms, min(all_ms), max(all_ms)], [bt_dev, bt_e2e, bt_smp], world, dev)
 
     pk = peaks()
-    step_input_bytes = (2 if w.dtype == "bf16" else 4) * (w.V * w.d + 2 * w.enc_layers * (4 * w.d * w.d + 2 * w.d * w.dff))
+    es = 2 if w.dtype == "bf16" else 4
+    step_input_bytes = es * (w.V * w.d + 2 * w.enc_layers * (4 * w.d * w.d + 2 * w.d * w.dff))
     l2_note = ("per-step inputs (W_U and both encoders' weights) exceed the 126 MB L2" if step_input_bytes > 126e6 else
                "per-step inputs (%.1f MB) fit the 126 MB L2 and are not flushed between steps: a small parity "
-               "configuration, not the one the metric is quoted on" % (step_input_bytes / 1e6))
-    # dominant kernel class by measured time
+               "configuration, not a benchmark one" % (step_input_bytes / 1e6))
     mean_hyper = 0.5 * (n_after + n_after2)     # hyper rows visible during the profiled pass
     classes = {"logits": logits_bytes(w, mean_hyper), "encoder_gemm": encoder_gemm_bytes(w)}
     dom = max(classes, key=lambda k: cls_ms.get(k, 0.0))
@@ -375,24 +479,26 @@ def run_ours(args, rank: int, world: int):
     def class_roof(k):
         n_launch = max(cls_launches[k], 1)
         ms_launch = cls_ms[k] / n_launch                     # average launch duration
-        by_launch = classes[k] * K / n_launch                # algorithmic bytes per launch
+        by_launch = classes[k] * Ka / n_launch               # algorithmic bytes per launch
         gbs = by_launch / max(ms_launch, 1e-9) / 1e6
-        return {"algorithmic_bytes_per_launch": by_launch, "launches_per_step": n_launch / K,
-                "us_per_launch": ms_launch * 1e3, "ms_per_step": cls_ms[k] / K, "gbs": gbs,
+        return {"algorithmic_bytes_per_launch": by_launch, "launches_per_step": n_launch / Ka,
+                "us_per_launch": ms_launch * 1e3, "ms_per_step": cls_ms[k] / Ka, "gbs": gbs,
                 "frac": gbs / pk["hbm_gbs"], "traffic": ncu_traffic(k, w.name)}
 
     cr = {k: class_roof(k) for k in classes}
+    step_bytes = logits_bytes(w, 0.5 * (n_before + n_after)) + encoder_gemm_bytes(w)
     roof = {"bound": "hbm", "kernel": {"logits": "k_decode_logits", "encoder_gemm": "k_stream_gemm"}[dom],
             "achieved": cr[dom]["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
             "frac": cr[dom]["frac"], "traffic": cr[dom]["traffic"],
             "peak_source": pk["source"] + " (STREAM-style copy, burst)",
             "timing": "CUDA events around every launch of the kernel on the launching stream, in a "
-                      "second pass of K steps (the events serialise the launches, which otherwise "
+                      "separate pass of %d steps (the events serialise the launches, which otherwise "
                       "overlap their prologues with the previous kernel); achieved = algorithmic "
-                      "bytes per launch / average launch duration",
-            "per_class_ms_per_step": {k: v / K for k, v in cls_ms.items()},
-            "logits": cr["logits"], "encoder_gemm": cr["encoder_gemm"]}
-    es = 2 if w.dtype == "bf16" else 4
+                      "bytes per launch / average launch duration" % Ka,
+            "per_class_ms_per_step": {k: v / Ka for k, v in cls_ms.items()},
+            "logits": cr["logits"], "encoder_gemm": cr["encoder_gemm"],
+            "whole_step": {"algorithmic_bytes": step_bytes, "gbs": step_bytes / (dev_ms / K) / 1e6,
+                           "frac": step_bytes / (dev_ms / K) / 1e6 / pk["hbm_gbs"]}}
     line = {
         "metric": METRIC, "value": bt_dev / (dev_ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": Wm, "ms_per_step": dev_ms / K, "higher_is_better": True,
@@ -403,25 +509,34 @@ def run_ours(args, rank: int, world: int):
                               "(teacher forcing)" if forced_mode else "argmax, free-running"),
                    "replicas": world,
                    "l2": l2_note},
+        "regions": {"count": R, "steps_each": K, "timed_s": sum(all_ms) * 1e-3,
+                    "ms_per_step_median": dev_ms / K, "ms_per_step_min": ms_min / K,
+                    "ms_per_step_max": ms_max / K,
+                    "note": "value and ms_per_step are those of the median region"},
         "steps_per_s": K / (dev_ms * 1e-3),
         "mean_phrase_len": bt_dev / (K * w.B * world),
-        "new_entries_in_timed_region": int(n_after - n_before),
+        "new_entries_in_timed_regions": int(n_after - n_before),
         "status_errors": bad,
         "prefill": prefill,
-        "e2e": {"value": bt_e2e / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / K,
+        "e2e": {"value": bt_e2e / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / Ka, "steps": Ka,
                 "h2d_bytes_per_step": int(w.B * w.d * es), "d2h_bytes_per_step": int(w.B * 8)},
-        "gpu_launches": int(sum(launches.values())),
+        "select_gumbel": {"value": bt_smp / (smp_ms * 1e-3), "unit": UNIT, "ms_per_step": smp_ms / Ka,
+                          "steps": Ka, "temperature": 1.0,
+                          "vs_argmax_step": (smp_ms / Ka) / (dev_ms / K)},
+        "gpu_launches": int(round(sum(launches.values()))),
         "gpu_launches_by_class": launches,
         "clocks": clocks,
         "roofline": roof,
     }
-    return line, w
+    del cb, E_h, U_h, hidden, nxt_all
+    return line
 
 
 # --------------------------------------------------------------------------------------------------
 # oracle on the host cores (cpu_baseline of our arm, and the whole `--impl reference` arm)
 # --------------------------------------------------------------------------------------------------
-def oracle_sample(w: si.Workload, n_steps: int, seed: int = 1000, prompt_tokens: int = 256):
+def oracle_sample(w: si.Workload, n_steps: int, seed: int = 1000, prompt_tokens: int | None = None,
+                  inputs: Inputs | None = None):
     """Times `n_steps` decode steps of the oracle session on the workload's shapes.
 
     Bounded sample: prompts are cut to `prompt_tokens` tokens so that embedding their entries in
@@ -430,12 +545,19 @@ def oracle_sample(w: si.Workload, n_steps: int, seed: int = 1000, prompt_tokens:
     """
     from oracle import decode_step as ods
     torch.set_num_threads(os.cpu_count() or 1)
+    if prompt_tokens is None:
+        prompt_tokens = 256 if w.d * w.B <= 3072 * 8 else 64
     T = min(w.T, prompt_tokens)
     tokens = si.make_tokens(w, seed, T=T)
-    W_E, W_U = si.make_tables(w, seed)
+    if inputs is None:
+        W_E, W_U = si.make_tables(w, seed)
+        eE, eU = si.make_encoder(w, seed * 3 + 1), (None if w.tied else si.make_encoder(w, seed * 3 + 2))
+    else:
+        W_E, W_U = inputs.tables(w, seed)
+        eE, eU = inputs.encoder(w, seed * 3 + 1), (None if w.tied else inputs.encoder(w, seed * 3 + 2))
     f = lambda t: t.double().numpy()
-    encE = [f(t) for t in si.make_encoder(w, seed * 3 + 1)]
-    encU = encE if w.tied else [f(t) for t in si.make_encoder(w, seed * 3 + 2)]
+    encE = [f(t) for t in eE]
+    encU = encE if w.tied else [f(t) for t in eU]
     s = ods.Session(w.V, w.M, w.cap, w.B, w.heads, w.dtype, f(W_E), f(W_E) if w.tied else f(W_U),
                     encE, encU)
     t0 = time.perf_counter()
@@ -450,23 +572,29 @@ def oracle_sample(w: si.Workload, n_steps: int, seed: int = 1000, prompt_tokens:
     dt = time.perf_counter() - t0
     return {"value": base / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
             "threads": torch.get_num_threads(),
-            "sample": f"{n_steps} decode steps of the full-shape workload (V, d, B, M, encoder as "
-                      f"configured) after prompts cut to {T} tokens; oracle prefill took "
-                      f"{t_prefill:.1f} s",
+            "sample": f"{n_steps} decode steps of the full-shape workload {w.name} (V, d, B, M, encoder as "
+                      f"configured) after prompts CUT to {T} of {w.T} tokens (a smaller codebook state than the "
+                      f"GPU arm's); oracle prefill took {t_prefill:.1f} s; numpy fp64, "
+                      f"{torch.get_num_threads()} threads",
             "seconds": dt, "ms_per_step": dt / n_steps * 1e3}
 
 
 def run_reference(args):
-    w = si.WORKLOADS[args.workload]
+    w = si.WORKLOADS[args.workload or DEFAULT_WORKLOAD]
+    if w.steps == 0:
+        print(json.dumps({"impl": "reference", "unavailable": "the oracle arm times decode steps; "
+                          "this workload has none"}))
+        return
     K = max(1, args.steps)
     per_step = 1 if w.d >= 2048 else 4
-    res = oracle_sample(w, n_steps=max(1, min(K, 6)) * per_step)
+    n = max(1, min(K, 6 if w.d * w.B <= 3072 * 8 else 2)) * per_step
+    res = oracle_sample(w, n_steps=n)
     line = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT,
             "n_gpus": args.gpus, "steps": K, "warmup": args.warmup,
             "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "M": w.M, "cap": w.cap},
-            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "threads", "kind", "sample")},
             "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
                     "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -475,24 +603,21 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------------
 # prompt-scoring workloads (no decode steps): encode + embed every entry + logits at every position
 # --------------------------------------------------------------------------------------------------
-def run_prompt_scoring(args, rank: int, world: int):
+def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: int, K: int, Wm: int):
     """One step = the whole prompt pass of the workload: LZW encode of every prompt, hyper-encoder
     over every codebook entry for both caches, joint logits + LSE / argmax at every compressed
     position (all n_b hypertokens of the sequence visible, the paper's training convention)."""
     from paper_2506_01084_b200 import binding as zb
     zb.lib()
-    dev = torch.device(f"cuda:{int(os.environ.get('LOCAL_RANK', 0))}")
-    torch.cuda.set_device(dev)
-    w = si.WORKLOADS[args.workload]
+    dev = inputs.dev
     if args.seqs:
         w = w.scaled(B=args.seqs)
-    K, Wm = args.steps, args.warmup
     seed = replica_seed(rank)
     tokens = si.make_tokens(w, seed)
-    W_E, W_U = si.make_tables(w, seed)
-    encE_t = [t.to(dev) for t in si.make_encoder(w, seed * 3 + 1)]
-    encU_t = [t.to(dev) for t in si.make_encoder(w, seed * 3 + 2)]
-    g_WE, g_WU = W_E.to(dev), W_U.to(dev)
+    W_E, W_U = inputs.tables(w, seed)
+    encE_t = [inputs.to_dev(t) for t in inputs.encoder(w, seed * 3 + 1)]
+    encU_t = [inputs.to_dev(t) for t in inputs.encoder(w, seed * 3 + 2)]
+    g_WE, g_WU = inputs.to_dev(W_E), inputs.to_dev(W_U)
     cfg = zb.make_config(w.V, w.d, w.M, w.cap, w.B, w.dtype, w.enc_layers, w.heads, w.dff, 0)
     cb = zb.Codebook(cfg, dev)
     encE, encU = zb.encoder_weights(encE_t), zb.encoder_weights(encU_t)
@@ -522,39 +647,36 @@ def run_prompt_scoring(args, rank: int, world: int):
         zb.z2z_dynamic_logits(cb, hid_dev, row_seq, None, g_WU, U_h, zb.SELECT_ARGMAX, 1.0, 0, 0, None,
                               lse, am, mx)
 
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-
     for _ in range(Wm):
         step(g_tok, hidden)
     zb.z2z_profile_read(cb)
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+    _barrier(world)
     e0.record()
     for _ in range(K):
         step(g_tok, hidden)
     e1.record()
-    barrier()
+    _barrier(world)
     dev_ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
     _, launches = zb.z2z_profile_read(cb)
     st, n_fin = zb.z2z_status(cb)
-    # per-class pass
+    # per-class pass (one step: its launches run for milliseconds, the events cost nothing beside them)
+    Kc = 1
     zb.z2z_profile(cb, True)
-    for _ in range(K):
+    for _ in range(Kc):
         step(g_tok, hidden)
     zb.z2z_profile(cb, False)
     cls_ms, cls_launches = zb.z2z_profile_read(cb)
     # end to end: prompts and hidden rows from pinned host memory, LSE back to the host
+    Ke = 1
     tok_dev = torch.empty_like(g_tok)
     hid_dev = torch.empty_like(hidden)
-    barrier()
+    _barrier(world)
     t0 = time.perf_counter()
-    for _ in range(K):
+    for _ in range(Ke):
         tok_dev.copy_(tok_host, non_blocking=True)
         hid_dev.copy_(hid_host, non_blocking=True)
         step(tok_dev, hid_dev)
@@ -566,7 +688,15 @@ def run_prompt_scoring(args, rank: int, world: int):
     n_rows = torch.bincount(row_seq.cpu().to(torch.int64), minlength=w.B).numpy()
     flops = 2.0 * w.d * float(sum(int(n_rows[b]) * (w.V + int(n_fin[b])) for b in range(w.B)))
     n_logit = max(cls_launches["logits"], 1)
-    tfs = flops * K / n_logit / max(cls_ms["logits"] / n_logit, 1e-9) / 1e9
+    tfs = flops * Kc / n_logit / max(cls_ms["logits"] / n_logit, 1e-9) / 1e9
+    # hyper-encoder linear layers: flop per row that carries data (rows = base tokens of all entries),
+    # both encoders; the kernel executes twice that (hi and lo parts of the activations)
+    enc_rows = 0
+    for b in range(w.B):
+        _, ln = zb.z2z_codebook_read(cb, b)
+        enc_rows += int(ln.numpy()[:int(n_fin[b])].sum())
+    enc_flops = 2.0 * enc_rows * w.enc_layers * 2.0 * (4 * w.d * w.d + 2 * w.d * w.dff)
+    enc_tfs = enc_flops * Kc / max(cls_ms["encoder_gemm"], 1e-9) / 1e9
     prompt_tokens = w.B * w.T * world
     bad = int(sum(1 for x in st.tolist() if x & (zb.ST_BAD_TOKEN | zb.ST_TABLE_FULL | zb.ST_WAIT_TIMEOUT)))
     es = 2
@@ -580,18 +710,25 @@ def run_prompt_scoring(args, rank: int, world: int):
                    "compressed_positions": N, "hypertokens": int(n_fin.sum()), "replicas": world,
                    "l2": "W_U, the caches and the hidden rows exceed the 126 MB L2"},
         "status_errors": bad,
-        "per_class_ms_per_step": {k: v / K for k, v in cls_ms.items()},
-        "e2e": {"value": prompt_tokens * K / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / K,
+        "per_class_ms_per_step": {k: v / Kc for k, v in cls_ms.items()},
+        "e2e": {"value": prompt_tokens * Ke / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms / Ke, "steps": Ke,
                 "h2d_bytes_per_step": int(tok_host.numel() * 4 + hid_host.numel() * es),
                 "d2h_bytes_per_step": int(N * 4)},
         "gpu_launches": int(sum(launches.values())), "gpu_launches_by_class": launches, "clocks": clocks,
         "roofline": {"bound": "tensor", "kernel": "k_prefill_logits", "achieved": tfs,
                      "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": tfs / pk["bf16_tflops_sustained"],
                      "traffic": None, "peak_source": pk["source"] + " (cuBLAS bf16, sustained)",
-                     "flops_per_launch": flops * K / n_logit, "us_per_launch": cls_ms["logits"] / n_logit * 1e3,
-                     "frac_of_burst_peak": tfs / pk["bf16_tflops"], "frac_of_nominal_2250": tfs / 2250.0},
+                     "flops_per_launch": flops * Kc / n_logit, "us_per_launch": cls_ms["logits"] / n_logit * 1e3,
+                     "frac_of_burst_peak": tfs / pk["bf16_tflops"], "frac_of_nominal_2250": tfs / 2250.0,
+                     "encoder_gemm": {"kernel": "k_pair_gemm", "rows": enc_rows,
+                                      "algorithmic_tflops": enc_tfs, "executed_tflops": 2.0 * enc_tfs,
+                                      "ms_per_step": cls_ms["encoder_gemm"] / Kc,
+                                      "frac_executed_of_sustained_peak": 2.0 * enc_tfs / pk["bf16_tflops_sustained"],
+                                      "note": "activations enter as bf16 hi + lo parts: two MMAs per k-step, so the "
+                                              "tensor pipe executes twice the algorithmic flop"}},
     }
-    return line, w
+    del cb, E_h, U_h, hidden, hid_host, lse, am, mx
+    return line
 
 
 # --------------------------------------------------------------------------------------------------
@@ -606,7 +743,7 @@ def run_helpers(args):
     zb.lib()
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
-    w = si.WORKLOADS[args.workload]
+    w = si.WORKLOADS[args.workload or DEFAULT_WORKLOAD]
     if args.seqs:
         w = w.scaled(B=args.seqs)
     pk = peaks()
@@ -684,13 +821,49 @@ def run_helpers(args):
     print(json.dumps(line))
 
 
-def main():
+# --------------------------------------------------------------------------------------------------
+# replicas: `--gpus N` without a launcher's environment starts the N ranks itself
+# --------------------------------------------------------------------------------------------------
+def free_port() -> int:
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_replicas(n: int, argv) -> int:
+    """Runs this script as `n` local ranks (one process per GPU) through torch.distributed.run
+    with a rendezvous on 127.0.0.1 and returns the launcher's exit code.  Rank 0 prints the line."""
+    from torch.distributed.run import main as torchrun
+    cmd = ["--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1", "--master-port",
+           str(free_port()), os.path.abspath(__file__)] + list(argv)
+    try:
+        torchrun(cmd)
+    except SystemExit as e:
+        return int(e.code or 0)
+    return 0
+
+
+def run_stub(rank: int, world: int):
+    """Launcher self-test (`--stub`): no kernel runs; every rank contributes fixed per-rank numbers
+    so that a CPU test can check the launch, the rendezvous, the reduction and the single line."""
+    dev = torch.device("cpu")
+    (ms,), (tok,) = reduce_over_ranks([10.0 + rank], [1000.0 * (rank + 1)], world, dev)
+    return {"metric": METRIC, "value": tok / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": 1, "warmup": 0,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "stub": True,
+            "config": {"workload": "stub", "replicas": world, "replica_seeds": [replica_seed(r) for r in range(world)]}}
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else list(argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="phi3_mini_head", choices=list(si.WORKLOADS))
+    ap.add_argument("--workload", default=None, choices=list(si.WORKLOADS),
+                    help="default: %s, with the other bf16 configurations as sub-records" % DEFAULT_WORKLOAD)
+    ap.add_argument("--sub-workloads", default="auto", choices=["auto", "on", "off"],
+                    help="auto: add the per_workload sub-records when no --workload is given and one GPU runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--helpers", action="store_true",
                     help="time the calls around the hot path (compression, decompression, embedding lookup, "
@@ -700,8 +873,13 @@ def main():
                          "LZW codes of a generator continuation (the selection is still computed)")
     ap.add_argument("--seqs", type=int, default=0,
                     help="prompt-scoring workloads: use this many sequences instead of the workload's B")
-    args = ap.parse_args()
+    ap.add_argument("--prompt-steps", type=int, default=2,
+                    help="timed steps of a prompt-scoring workload (one step is a whole prompt batch)")
+    ap.add_argument("--stub", action="store_true", help="launcher self-test: ranks report fixed numbers, no GPU work")
+    args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3)
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_replicas(args.gpus, argv))
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":
@@ -713,13 +891,38 @@ def main():
             run_helpers(args)
         return
     if world > 1:
-        torch.distributed.init_process_group("nccl")
-    prompt_mode = si.WORKLOADS[args.workload].steps == 0
-    line, w = run_prompt_scoring(args, rank, world) if prompt_mode else run_ours(args, rank, world)
+        torch.distributed.init_process_group("gloo" if args.stub else "nccl")
+    if args.stub:
+        line = run_stub(rank, world)
+    else:
+        inputs = Inputs(_local_device())
+        w = si.WORKLOADS[args.workload or DEFAULT_WORKLOAD]
+        prompt_mode = w.steps == 0
+        if prompt_mode:
+            line = run_prompt_scoring(args, w, inputs, rank, world, max(1, args.prompt_steps), 3)
+        else:
+            line = run_decode(args, w, inputs, rank, world)
+        subs = args.sub_workloads == "on" or (args.sub_workloads == "auto" and args.workload is None and world == 1)
+        if subs:
+            per = {}
+            for name in SUB_WORKLOADS:
+                if name == w.name:
+                    continue
+                gc.collect()
+                torch.cuda.empty_cache()
+                sw = si.WORKLOADS[name]
+                if sw.steps == 0:
+                    per[name] = run_prompt_scoring(args, sw, inputs, rank, world, max(1, args.prompt_steps), 3)
+                else:
+                    per[name] = run_decode(args, sw, inputs, rank, world)
+                for k in ("metric", "unit", "higher_is_better", "scaling", "vs_baseline", "data", "n_gpus"):
+                    if k != "metric" or sw.steps > 0:
+                        per[name].pop(k, None)
+            line["per_workload"] = per
+        if rank == 0 and world == 1 and not args.no_cpu_baseline and not prompt_mode:
+            res = oracle_sample(w, n_steps=2 if w.d >= 2048 else 16, inputs=inputs)
+            line["cpu_baseline"] = {k: res[k] for k in ("value", "unit", "cores", "threads", "kind", "sample")}
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline and not prompt_mode:
-            res = oracle_sample(w, n_steps=2 if w.d >= 2048 else 16)
-            line["cpu_baseline"] = {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()

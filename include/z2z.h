@@ -274,7 +274,8 @@ int32_t z2z_profile_read(z2z_codebook* cb, int32_t n_classes, double* h_ms, int6
  * nothing in this call.
  *   d_hidden [N, d], d_row_seq [N] or NULL (row r belongs to sequence r), d_WU [V, d],
  *   d_Uh [B, cap, d], all in `dtype`; d_n_hyper [B] DEVICE array: visible hypertokens of each
- *   sequence; d_lse / d_argmax / d_max_logit [N] out, each may be NULL.
+ *   sequence, 0 <= d_n_hyper[b] <= cap (a larger count is read as cap: no row beyond a sequence's
+ *   cap rows is touched); d_lse / d_argmax / d_max_logit [N] out, each may be NULL.
  * Limits: N <= 1024 rows per call (larger N returns Z2Z_ERR_INVALID_ARG and z2z_last_error says
  * so); the other limits are those of z2z_config.  Same arithmetic as the CUDA-core path of
  * z2z_dynamic_logits (fp32 accumulation).

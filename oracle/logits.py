@@ -138,13 +138,3 @@ def select_filtered(l: np.ndarray, temperature: float, top_k: int, top_p: float,
     scores = np.where(keep, scores, -np.inf)
     a, _, gap = top2(scores)
     return a, keep, gap
-
-
-def nucleus_margin(l: np.ndarray, temperature: float, top_p: float) -> float:
-    """How far (in probability mass) top_p is from the nearest cumulative sum of the descending
-    probabilities: parity tests skip inputs where fp32 summation could move the boundary."""
-    l = np.asarray(l, dtype=np.float64)
-    ls = np.sort(l)[::-1]
-    pr = np.exp((ls - ls[0]) / float(temperature))
-    cum = np.cumsum(pr) / pr.sum()
-    return float(np.abs(cum - top_p).min())

@@ -377,6 +377,10 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
   a.sample = select == Z2Z_SELECT_GUMBEL ? w_sample : nullptr;
   a.lpart = cb->ws + cb->plan.off_lpart; a.lpart_bytes = cb->plan.lpart_bytes;
   const bool fused = B <= 128;                 // one launch for merge + select + LZW update + work list
+  // The frozen-session word is sampled BEFORE this step's update kernel is enqueued, and that kernel
+  // only reports codebooks that were already full when it started: a step whose update can still
+  // create an entry therefore always runs its hyper-encoder pass, however fast the device is.
+  const bool frozen = cb->h_frozen && *reinterpret_cast<volatile int*>(cb->h_frozen) == cb->epoch;
   z2z::EntryList el = entry_list(cb);
   if (fused) {
     z2z::LogitsPartInfo info{0, 0};
@@ -411,7 +415,6 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
   }
   // cache update: the at most one new entry per sequence, on both sides.  Once an earlier step has
   // reported that every codebook is full nothing can be created any more and the pass is not launched.
-  const bool frozen = cb->h_frozen && *reinterpret_cast<volatile int*>(cb->h_frozen) == cb->epoch;
   if (cb->cfg.cap > 0 && !frozen) {
     const bool tc = cb->use_tensor_cores && z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype, cb->heads, cb->cfg.M);
     z2z::EncoderArgs g[2];
@@ -459,15 +462,19 @@ int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t*
   if (h_cons)
     Z2Z_CUDA(cudaMemcpyAsync(h_cons, cb->view.cons + (size_t)b * cap * M, (size_t)cap * M * 4,
                              cudaMemcpyDeviceToHost, s), "codebook_read");
-  Z2Z_CUDA(cudaStreamSynchronize(s), "codebook_read");
-  if (h_len) {
-    uint8_t* tmp = new (std::nothrow) uint8_t[cap];
+  uint8_t* tmp = nullptr;
+  if (h_len) {                                     // lengths are bytes on the device, int32 for the caller
+    tmp = new (std::nothrow) uint8_t[cap];
     if (!tmp) return fail(Z2Z_ERR_INVALID_ARG, "out of host memory");
-    cudaError_t e = cudaMemcpy(tmp, cb->view.len + (size_t)b * cap, cap, cudaMemcpyDeviceToHost);
-    for (int i = 0; i < cap; ++i) h_len[i] = tmp[i];
-    delete[] tmp;
-    if (e != cudaSuccess) return fail_cuda(e, "codebook_read");
+    cudaError_t e = cudaMemcpyAsync(tmp, cb->view.len + (size_t)b * cap, cap, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) { delete[] tmp; return fail_cuda(e, "codebook_read"); }
   }
+  cudaError_t e = cudaStreamSynchronize(s);
+  if (tmp) {
+    if (e == cudaSuccess) for (int i = 0; i < cap; ++i) h_len[i] = tmp[i];
+    delete[] tmp;
+  }
+  if (e != cudaSuccess) return fail_cuda(e, "codebook_read");
   return Z2Z_OK;
 }
 

@@ -32,7 +32,11 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kThreads = 192;
+// Threads per CTA: producer warp, MMA warp, then the epilogue warps.  Up to 16 hidden rows one
+// epilogue thread keeps the reductions of every row of its vocabulary row in registers (4 warps, one
+// per tensor-memory lane quarter); 17-32 rows are split between two warps per quarter, 16 rows each.
+__host__ __device__ constexpr int decode_epi_warps(int nb) { return nb > 16 ? 8 : 4; }
+__host__ __device__ constexpr int decode_threads(int nb) { return 64 + 32 * decode_epi_warps(nb); }
 constexpr int kGran = 64;                // pool unit / scheduling granule, in weight rows
 constexpr int kJobRing = 32;             // published jobs kept (> stages + accumulators in flight)
 constexpr int kDecodeMaxStages = 12;
@@ -97,10 +101,12 @@ __device__ __forceinline__ bool pool_job(const DecodeLogitsParams& p, const int*
 }
 
 template <int NB, bool GENERIC, bool RESIDENT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(decode_threads(NB), 1)
 k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitMaps tm) {
   constexpr int NT = 128;
   constexpr int NBP = NB < 16 ? 16 : NB;            // the MMA's N (a multiple of 16 for M = 128)
+  constexpr int EW = decode_epi_warps(NB);          // epilogue warps
+  constexpr int RW = NB > 16 ? 16 : NB;             // hidden rows one epilogue thread reduces
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   DecodeCtrl* ctrl = reinterpret_cast<DecodeCtrl*>(sm);
@@ -122,7 +128,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&ctrl->acc_full[b]), 1);
-      mbar_init(smem_u32(&ctrl->acc_empty[b]), 4);
+      mbar_init(smem_u32(&ctrl->acc_empty[b]), EW);
     }
     for (int i = 0; i < kJobRing; ++i) mbar_init(smem_u32(&ctrl->job_ready[i]), 1);
     mbar_init(smem_u32(&ctrl->hid_full), 1);
@@ -255,7 +261,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
       ds->seq[r] = sq; ds->nvis[r] = nv; ds->tgt[r] = tg;
     }
     tc_fence_before();
-    asm volatile("bar.sync 2, 160;" ::: "memory");   // warps 1-5: tensor memory address and row table are set
+    asm volatile("bar.sync 2, %0;" ::"n"(32 + 32 * EW) : "memory");   // all but the producer warp: tensor memory address and row table are set
     tc_fence_after();
   }
   if (warp == 1) {
@@ -303,16 +309,17 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
     // ---------------- epilogue: thread = vocabulary row of the job ------------------------------------
     const uint32_t tmem_base = ctrl->tmem_base;
     const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
+    const int h0 = ((warp - 2) >> 2) * RW;            // first hidden row of this warp's share
     const int row_in_job = q * 32 + lane;
     const uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
     const uint32_t c2 = (uint32_t)a.step, c3 = (uint32_t)(a.step >> 32);
     const size_t ldbg = (size_t)p.cb.V + p.cb.cap;
-    float m[NB], s[NB]; int idx[NB];
-    float gm[GENERIC ? NB : 1]; int gidx[GENERIC ? NB : 1];
+    float m[RW], s[RW]; int idx[RW];
+    float gm[GENERIC ? RW : 1]; int gidx[GENERIC ? RW : 1];
 #pragma unroll
-    for (int bb = 0; bb < NB; ++bb) { m[bb] = -INFINITY; s[bb] = 0.f; idx[bb] = 0x7fffffff; }
+    for (int bb = 0; bb < RW; ++bb) { m[bb] = -INFINITY; s[bb] = 0.f; idx[bb] = 0x7fffffff; }
 #pragma unroll
-    for (int bb = 0; bb < (GENERIC ? NB : 1); ++bb) { gm[bb] = -INFINITY; gidx[bb] = 0x7fffffff; }
+    for (int bb = 0; bb < (GENERIC ? RW : 1); ++bb) { gm[bb] = -INFINITY; gidx[bb] = 0x7fffffff; }
     uint32_t job_i = 0;
     while (true) {
       const uint32_t slot = job_i % kJobRing;
@@ -323,28 +330,29 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
       if (!mbar_wait(smem_u32(&ctrl->acc_full[buf]), aph, &ctrl->abort)) break;
       tc_fence_after();
       if (q * 32 < j.nvalid) {                       // warp-uniform: some weight row of this quarter exists
-        uint32_t v[NB];
-        TmemRow<NB>::ld(tmem_base + ((uint32_t)(q * 32) << 16) + buf * NBP, v);
+        uint32_t v[RW];
+        TmemRow<RW>::ld(tmem_base + ((uint32_t)(q * 32) << 16) + buf * NBP + h0, v);
         tmem_ld_wait();
         if (row_in_job < j.nvalid) {
           const int col = j.col0 + row_in_job;
           const int krow = j.k0 + row_in_job;        // entry number, for hypertoken rows
 #pragma unroll
-          for (int bb = 0; bb < NB; ++bb) {
-            const int sq = ds->seq[bb];
-            const bool vis = sq >= 0 && (j.owner < 0 || (sq == j.owner && krow < ds->nvis[bb]));
+          for (int bb = 0; bb < RW; ++bb) {
+            const int hr = h0 + bb;                    // hidden row of the batch
+            const int sq = ds->seq[hr];
+            const bool vis = sq >= 0 && (j.owner < 0 || (sq == j.owner && krow < ds->nvis[hr]));
             if (vis) {
               const float l = __uint_as_float(v[bb]);
               if (l > m[bb]) { s[bb] = s[bb] * __expf(m[bb] - l) + 1.f; m[bb] = l; idx[bb] = col; }
               else { s[bb] += __expf(l - m[bb]); if (l == m[bb] && col < idx[bb]) idx[bb] = col; }
               if (GENERIC) {
                 if (a.select == Z2Z_SELECT_GUMBEL) {
-                  const Philox4 px = philox4x32_10((uint32_t)(col >> 2), (uint32_t)(a.row_base + bb), c2, c3, k0, k1);
+                  const Philox4 px = philox4x32_10((uint32_t)(col >> 2), (uint32_t)(a.row_base + hr), c2, c3, k0, k1);
                   const float sc = fmaf(l, a.inv_temperature, gumbel_from_word(philox_word(px, col & 3)));
                   if (sc > gm[bb] || (sc == gm[bb] && col < gidx[bb])) { gm[bb] = sc; gidx[bb] = col; }
                 }
-                if (a.logits_debug) a.logits_debug[(size_t)bb * ldbg + col] = l;
-                if (col == ds->tgt[bb] && a.target_logit) a.target_logit[bb] = l;
+                if (a.logits_debug) a.logits_debug[(size_t)hr * ldbg + col] = l;
+                if (col == ds->tgt[hr] && a.target_logit) a.target_logit[hr] = l;
               }
             }
           }
@@ -358,7 +366,7 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
     // merge the 128 threads' reductions of every hidden row: the warp's maximum first, then every
     // lane's sum rescaled to it, then the lowest index among the lanes that hold the maximum
 #pragma unroll
-    for (int bb = 0; bb < NB; ++bb) {
+    for (int bb = 0; bb < RW; ++bb) {
       const float mm = key_float(__reduce_max_sync(0xffffffffu, float_key(m[bb])));
       float ss = m[bb] == -INFINITY ? 0.f : s[bb] * __expf(m[bb] - mm);
 #pragma unroll
@@ -369,9 +377,9 @@ k_decode_logits(const DecodeLogitsParams p, const __grid_constant__ DecodeLogitM
         gg = key_float(__reduce_max_sync(0xffffffffu, float_key(gm[bb])));
         gi = __reduce_min_sync(0xffffffffu, gm[bb] == gg ? gidx[bb] : 0x7fffffff);
       }
-      if (lane == 0) { RowRed r; r.m = mm; r.s = ss; r.idx = ii; r.gm = gg; r.gidx = gi; ds->part[q][bb] = r; }
+      if (lane == 0) { RowRed r; r.m = mm; r.s = ss; r.idx = ii; r.gm = gg; r.gidx = gi; ds->part[q][h0 + bb] = r; }
     }
-    asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps only
+    asm volatile("bar.sync 1, %0;" ::"n"(32 * EW) : "memory");   // the epilogue warps only
     const int t = (warp - 2) * 32 + lane;
     if (t < NB && t < a.N) {
       RowRed red = ds->part[0][t];
@@ -427,11 +435,9 @@ __global__ void k_decode_fill_nan(float* p, int n) {
 
 }  // namespace
 
-// Decode batches: N <= 16 rows with any outputs, N <= 32 rows when only the plain reductions are
-// wanted (the sampling state of 32 rows does not fit the register file); d a multiple of 256.
+// Decode batches: at most 32 hidden rows, with any outputs; d a multiple of 256.
 bool decode_logits_applies(const LogitsArgs& a) {
-  const bool generic = a.select == Z2Z_SELECT_GUMBEL || a.logits_debug || a.target_logit;
-  return a.dtype == Z2Z_DTYPE_BF16 && a.d % 256 == 0 && (a.N <= 16 || (a.N <= 32 && !generic));
+  return a.dtype == Z2Z_DTYPE_BF16 && a.d % 256 == 0 && a.N <= 32;
 }
 
 template <int NB, bool GENERIC>
@@ -451,7 +457,7 @@ static cudaError_t launch_decode(DecodeLogitsParams p, const DecodeLogitMaps& ma
   auto kern = resident ? k_decode_logits<NB, GENERIC, true> : k_decode_logits<NB, GENERIC, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(kern, dim3(grid), dim3(kThreads), smem, s, p, maps);
+  return launch_pdl(kern, dim3(grid), dim3(decode_threads(NB)), smem, s, p, maps);
 }
 
 cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counters, int* err_word,
@@ -500,7 +506,7 @@ cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counte
     ProfScope ps(prof, kProfLogits, 1, s);
     if (a.N <= 8) e = generic ? launch_decode<8, true>(p, maps, grid, resident, s) : launch_decode<8, false>(p, maps, grid, resident, s);
     else if (a.N <= 16) e = generic ? launch_decode<16, true>(p, maps, grid, resident, s) : launch_decode<16, false>(p, maps, grid, resident, s);
-    else e = launch_decode<32, false>(p, maps, grid, resident, s);
+    else e = generic ? launch_decode<32, true>(p, maps, grid, resident, s) : launch_decode<32, false>(p, maps, grid, resident, s);
   }
   if (e != cudaSuccess || info) return e;
   ProfScope ps(prof, kProfLogitsMerge, 1, s);

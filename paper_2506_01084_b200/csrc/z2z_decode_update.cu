@@ -96,11 +96,13 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
   if (tid < cb.B) {
     const int n = cb.n[tid];
     cb.n_emb[tid] = n; cb.n_emb[cb.B + tid] = n;
-    full = n >= cb.cap;
+    full = n >= cb.cap && mine == 0;             // full already when this step began: it created nothing
   }
   // Once every codebook is full no step creates an entry any more.  The host learns it through a
   // word in its own memory and stops launching the hyper-encoder pass (the session number guards
-  // against a late store from before a reset).
+  // against a late store from before a reset).  The word is only written by a step that found every
+  // codebook full on entry: the step that creates the last entry still needs its encoder pass, and
+  // the host may read the word at any time after this kernel was enqueued.
   if (a.frozen_flag && cb.B <= (int)blockDim.x) {
     const int all_full = __syncthreads_and(full);
     if (all_full && tid == 0) *reinterpret_cast<volatile int*>(a.frozen_flag) = a.epoch;

@@ -27,7 +27,7 @@ __device__ __forceinline__ TileDesc logits_tile(const CbView& cb, int t, int n_s
     td.owner = u / tiles_per_seq;
     td.k0 = (u - td.owner * tiles_per_seq) * kTJ;
     td.col0 = cb.V + td.k0;
-    const int n = cb.n[td.owner];
+    const int n = min(cb.n[td.owner], cb.cap);      // a count beyond the cache's rows reads no further than them
     td.nvalid = n - td.k0 < kTJ ? n - td.k0 : kTJ;
     td.base = reinterpret_cast<const char*>(Uh) + ((size_t)td.owner * cb.cap + td.k0) * d * esz;
   }
@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(256) k_logits_simt(CbView cb, LogitsArgs a, in
     if (r < a.N) {
       sq = a.row_seq ? a.row_seq[r] : r;
       if (sq < 0 || sq >= cb.B) sq = -1;
-      if (sq >= 0) { nv = cb.n[sq]; if (a.row_nvis) { int q = a.row_nvis[r]; nv = q < nv ? (q < 0 ? 0 : q) : nv; } }
+      if (sq >= 0) { nv = min(cb.n[sq], cb.cap); if (a.row_nvis) { int q = a.row_nvis[r]; nv = q < nv ? (q < 0 ? 0 : q) : nv; } }
       if (a.targets) tg = a.targets[r];
     }
     s_seq[t] = sq; s_nvis[t] = nv; s_tgt[t] = tg;
@@ -162,7 +162,14 @@ cudaError_t run_logits_simt(const CbView& cb, const LogitsArgs& a, LogitsPartInf
   const int tiles_per_seq = (cb.cap + kTJ - 1) / kTJ;
   const int n_tiles = n_static + cb.B * tiles_per_seq;
   const int row_tiles = (a.N + kTR - 1) / kTR;
-  int G = (148 * 4 + row_tiles - 1) / row_tiles;
+  static int n_sm = 0;
+  if (!n_sm) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (n_sm <= 0) n_sm = 148;
+  }
+  int G = (n_sm * 4 + row_tiles - 1) / row_tiles;
   if (G > n_tiles) G = n_tiles;
   while (G > 1 && (size_t)a.N * G * sizeof(LogitPartial) > a.lpart_bytes) --G;
   if ((size_t)a.N * G * sizeof(LogitPartial) > a.lpart_bytes) return cudaErrorInvalidValue;

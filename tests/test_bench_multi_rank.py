@@ -1,7 +1,9 @@
 """Host-side logic of the multi-GPU benchmark path, on CPU with two `gloo` ranks: the path has no
 data-path collective (ranks run independent replicas of the workload), so what has to be right is
 that replicas differ, that the reported time is the maximum over ranks and that counts are summed."""
+import json
 import os
+import subprocess
 import sys
 
 import numpy as np
@@ -47,3 +49,29 @@ def test_single_rank_reduction_is_identity():
     import bench
     assert bench.reduce_over_ranks([1.5, 2.5], [3.0], 1, torch.device("cpu")) == ([1.5, 2.5], [3.0])
     assert bench.replica_seed(0) != bench.replica_seed(1)
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    # `bench.py --gpus 2` without a launcher's environment must start two ranks, rendezvous on
+    # 127.0.0.1, reduce over them and print one line from rank 0.  --stub replaces the GPU work by
+    # fixed per-rank numbers (rank r: 10 + r ms, 1000 (r + 1) tokens) so this runs on CPU with gloo.
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--stub"], env=env,
+                       stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["stub"] is True
+    assert line["ms_per_step"] == 11.0                       # max over ranks
+    assert abs(line["value"] - 3000.0 / 0.011) < 1e-6        # summed tokens / max time
+    assert line["config"]["replica_seeds"] == [1000, 1001]
+
+
+def test_region_planning():
+    import bench
+    assert bench.plan_regions(20, 0.25, 10 ** 6) == 60       # 0.3 s / (20 x 0.25 ms)
+    assert bench.plan_regions(20, 0.25, 100) == 5            # bounded by the codebook room in steps
+    assert bench.plan_regions(256, 2.0, 10 ** 6) == 1        # one region already covers 0.3 s
+    assert bench.plan_regions(20, 0.25, -5) == 1

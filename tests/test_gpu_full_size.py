@@ -136,18 +136,56 @@ def test_full_size_decode_steps_sampled(name, steps, sample_seqs):
     print(f"{name}: worst |LSE error| {worst_lse:.2e}, worst |hyper-embedding error| {worst_emb:.2e}")
 
 
+def _oracle_logits_rows(H64, W_U, block=16384):
+    """Static part of the joint logits of several hidden rows at once: the oracle's joint_logits
+    applied to the rows as columns of one matrix, W_U converted to fp64 block by block.
+    Returns [V, rows]."""
+    parts = [olg.joint_logits(H64.T, _f64(W_U[i:i + block]), None) for i in range(0, W_U.shape[0], block)]
+    return np.concatenate(parts, axis=0)
+
+
 def test_full_size_prompt_scoring_sampled():
-    """prefill_heavy: every compressed position scored against V + n_b columns (CTA-pair kernel),
-    causal visibility from the encoder's entries_after; a sample of entries embedded and checked."""
+    """prefill_heavy at its full size (64 prompts of 8192 tokens): every compressed position scored
+    against V + n_vis columns by the CTA-pair kernel with causal visibility from the encoder's
+    entries_after.  The oracle scores a sample of positions chosen where an indexing mistake would
+    show: the first and last row of 256-row tiles, rows on both sides of sequence boundaries that
+    fall inside a tile, rows that see no hypertoken and rows that see all of them, plus random rows.
+    Then both hyper-encoders run prompt-sized passes (all entries of two sequences, a few of every
+    other) and a sample of entries, entries of length M among them, is held against the oracle."""
     w = si.WORKLOADS["prefill_heavy"]
     s = FullSession(w, seed=73)
     clen = s.clen.cpu().numpy()
     N = int(clen.sum())
+    offs = np.concatenate([[0], np.cumsum(clen)]).astype(np.int64)
     row_seq = torch.repeat_interleave(torch.arange(w.B, dtype=torch.int32, device=DEV), s.clen.to(torch.int64))
     # visible hypertokens at compressed position i of sequence b: those that exist once code i is out
     mask = torch.arange(w.T, device=DEV)[None, :] < s.clen[:, None]
     row_nvis = s.after[mask].contiguous()
     assert row_seq.numel() == N and row_nvis.numel() == N
+    st, n_gpu = zb.z2z_status(s.cb)
+    rng = np.random.default_rng(75)
+    n_tiles = (N + 255) // 256
+    rows = set()
+    for t in [0, 1, n_tiles // 3, n_tiles // 2, n_tiles - 2, n_tiles - 1]:
+        rows.update([t * 256, min(t * 256 + 255, N - 1)])                 # tile edges (the last tile is ragged)
+    inner = [b for b in range(1, w.B) if offs[b] % 256 not in (0, 255)]  # boundaries inside a tile
+    for b in inner[:6] + inner[-2:]:
+        rows.update([int(offs[b]) - 1, int(offs[b])])
+    none_rows = [int(offs[b]) + int(rng.integers(1, clen[b])) for b in (2, 31, w.B - 1)]
+    all_rows = [int(offs[b]) + int(rng.integers(0, clen[b] - 1)) for b in (0, 17, 40, w.B - 2)]
+    rows.update(none_rows + all_rows)
+    while len(rows) < 72:
+        rows.add(int(rng.integers(0, N)))
+    rows = sorted(rows)
+    seq_of = np.searchsorted(offs, np.asarray(rows), side="right") - 1
+    # two overrides of the causal limit (any value in [0, n_b] is a legal input): no hypertoken
+    # visible, and every hypertoken of the sequence visible
+    nvis_host = row_nvis.cpu().numpy().copy()
+    for r in none_rows:
+        nvis_host[r] = 0
+    for r in all_rows:
+        nvis_host[r] = s.book(int(np.searchsorted(offs, r, side="right") - 1)).n()
+    row_nvis = torch.from_numpy(nvis_host).to(DEV)
     hid = si.make_hidden(w, 16384, 74)[torch.arange(N) % 16384]     # 16384 distinct rows, repeated
     g_hid = hid.to(DEV)
     lse = torch.zeros(N, dtype=torch.float32, device=DEV)
@@ -156,34 +194,63 @@ def test_full_size_prompt_scoring_sampled():
     zb.z2z_dynamic_logits(s.cb, g_hid, row_seq, row_nvis, s.g_WU, s.U_h, zb.SELECT_ARGMAX, 1.0, 0, 0, None,
                           lse, am, mx)
     g_lse, g_am, g_mx = lse.cpu().numpy(), am.cpu().numpy(), mx.cpu().numpy()
-    offs = np.concatenate([[0], np.cumsum(clen)])
-    rng = np.random.default_rng(75)
-    samples = [(0, 0), (0, int(clen[0]) - 1), (w.B - 1, int(clen[-1]) - 1)]
-    samples += [(int(b), int(rng.integers(0, clen[b]))) for b in rng.integers(0, w.B, size=5)]
+    H64 = _f64(hid[rows])
+    static = _oracle_logits_rows(H64, s.W_U)                        # [V, len(rows)]
+    enc_cache = {}
     worst = 0.0
-    for b, i in samples:
-        r = int(offs[b]) + i
-        codes_b, after_b, _ = olzw.encode(s.tokens[b].tolist(), w.V, w.M, w.cap)
-        assert len(codes_b) == clen[b]
-        nv = after_b[i]
-        l = _oracle_logits(_f64(hid[r]), s.W_U, _f64(s.U_syn[b, :nv]))
-        worst = max(worst, abs(g_lse[r] - olg.lse(l)))
-        assert abs(g_lse[r] - olg.lse(l)) <= TOL, (b, i, g_lse[r], olg.lse(l))
+    for x, r in enumerate(rows):
+        b = int(seq_of[x]); i = r - int(offs[b])
+        if b not in enc_cache:
+            enc_cache[b] = olzw.encode(s.tokens[b].tolist(), w.V, w.M, w.cap)
+        codes_b, after_b, ob = enc_cache[b]
+        assert len(codes_b) == clen[b] and ob.n() == int(n_gpu[b])
+        nv = 0 if r in none_rows else (ob.n() if r in all_rows else after_b[i])
+        assert nv == nvis_host[r]
+        l = static[:, x]
+        if nv > 0:
+            l = np.concatenate([l, _f64(s.U_syn[b, :nv]) @ H64[x]])
+        want = olg.lse(l)
+        worst = max(worst, abs(g_lse[r] - want))
+        assert abs(g_lse[r] - want) <= TOL, (b, i, r, g_lse[r], want)
         a, best, gap = olg.top2(l)
-        assert abs(g_mx[r] - best) <= TOL
+        assert abs(g_mx[r] - best) <= TOL, (b, i, r)
+        assert 0 <= g_am[r] < w.V + nv, (b, i, r, g_am[r], nv)
         if g_am[r] != a:
-            assert gap < GAP and l[g_am[r]] >= best - GAP
-    print(f"prefill_heavy: {N} rows scored, worst sampled |LSE error| {worst:.2e}")
-    # hyper-embedding of a sample of entries of every sequence (explicit ranges)
-    first = torch.tensor([int(rng.integers(0, 1000)) for _ in range(w.B)], dtype=torch.int32, device=DEV)
-    count = torch.full((w.B,), 4, dtype=torch.int32, device=DEV)
+            assert gap < GAP and l[g_am[r]] >= best - GAP, (b, i, r)
+    print(f"prefill_heavy: {N} rows scored, {len(rows)} sampled, worst sampled |LSE error| {worst:.2e}")
+    del g_hid, lse, am, mx, static
+    # ---- hyper-embedding at prompt size, both sides (CTA-pair GEMM passes)
+    full = [5, 50]                                   # every entry of these sequences; four of every other
+    nb = [s.book(b).n() if b in full else 0 for b in range(w.B)]
+    first_h = [0 if b in full else int(rng.integers(0, 1000)) for b in range(w.B)]
+    count_h = [nb[b] if b in full else 4 for b in range(w.B)]
+    first = torch.tensor(first_h, dtype=torch.int32, device=DEV)
+    count = torch.tensor(count_h, dtype=torch.int32, device=DEV)
     E32 = torch.zeros(w.B, w.cap, w.d, dtype=torch.float32, device=DEV)
-    zb.z2z_hyper_embed(s.cb, zb.CACHE_EMBED, s.g_WE, s.g_encE, first, count, 4 * w.B, s.E_h, E32)
-    encE64 = [_f64(t) for t in s.enc_E]
-    for b in (0, 33, w.B - 1):
-        ob = s.book(b)
-        k = int(first[b].item()) + 2
-        want = _oracle_embed(ob.entries[k], s.W_E, encE64, w.heads)
-        err = np.abs(E32[b, k].cpu().double().numpy() - want).max()
-        assert err <= TOL, (b, k, err)
-        assert torch.equal(s.E_h[b, k].cpu(), E32[b, k].cpu().to(w.torch_dtype))
+    U_out = torch.zeros(w.B, w.cap, w.d, dtype=w.torch_dtype, device=DEV)
+    zb.z2z_hyper_embed(s.cb, zb.CACHE_EMBED, s.g_WE, s.g_encE, first, count, sum(count_h), s.E_h, E32)
+    picks = []
+    for b in full:
+        ents = s.book(b).entries
+        longest = [k for k in range(len(ents)) if len(ents[k]) == w.M]
+        assert longest
+        ks = {0, len(ents) - 1, longest[0], longest[-1], longest[len(longest) // 2]}
+        while len(ks) < 12:
+            ks.add(int(rng.integers(0, len(ents))))
+        picks += [(b, k) for k in sorted(ks)]
+    picks += [(b, first_h[b] + j) for b, j in ((0, 0), (1, 3), (33, 2), (w.B - 1, 1), (20, 0), (41, 3), (63, 0), (12, 2))]
+    assert len(picks) >= 32
+    worst_e = 0.0
+    for side, table, enc_t, cache, out32 in (("E", s.W_E, s.enc_E, s.E_h, E32), ("U", s.W_U, s.enc_U, U_out, None)):
+        if side == "U":
+            E32.zero_()                               # the one fp32 side buffer serves both sides in turn
+            zb.z2z_hyper_embed(s.cb, zb.CACHE_UNEMBED, s.g_WU, s.g_encU, first, count, sum(count_h), U_out, E32)
+        enc64 = [_f64(t) for t in enc_t]
+        for b, k in picks:
+            want = _oracle_embed(s.book(b).entries[k], table, enc64, w.heads)
+            err = np.abs(E32[b, k].cpu().double().numpy() - want).max()
+            worst_e = max(worst_e, err)
+            assert err <= TOL, (side, b, k, err)
+            assert torch.equal(cache[b, k].cpu(), E32[b, k].cpu().to(w.torch_dtype))
+        del enc64
+    print(f"prefill_heavy: {len(picks)} entries per side, worst |hyper-embedding error| {worst_e:.2e}")

@@ -439,6 +439,45 @@ def test_decode_step_with_frozen_codebooks():
     assert launches["encoder_gemm"] > 0
 
 
+def test_decode_step_codebooks_fill_up_during_decode():
+    # The cap is reached in the middle of decoding.  The step that creates a sequence's last entry
+    # must still embed it on both sides (its rows are held against the oracle inside _decode_follow),
+    # and the hyper-encoder pass runs in every step that can still create an entry, never afterwards:
+    # the host samples the "all full" word before it enqueues a step, and a step only reports
+    # codebooks that were already full when it began.
+    base = SMALL_BF16
+    seed = 44
+    tokens = si.make_tokens(base, seed)
+    n_prompt = [olzw.encode(tokens[b].tolist(), base.V, base.M, 10 ** 6)[2].n() for b in range(base.B)]
+    w = base.scaled(name="fills_up", cap=min(n_prompt) + 2)
+    _decode_follow(w, seed, zb.SELECT_ARGMAX, steps=10)            # checks every created row, the last one included
+    p = Pair(w, seed=seed)
+    _prefill_both(p)
+    assert min(bk.n() for bk in p.oracle.books) == w.cap - 2
+    hid = si.make_hidden(w, 16 * w.B, seed + 1).view(16, w.B, w.d).to(p.dev)
+    nxt = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    new = torch.zeros(w.B, dtype=torch.int32, device=p.dev)
+    passes, full_before = [], []
+    for t in range(16):
+        _, n = zb.z2z_status(p.cb)
+        full_before.append(bool((n >= w.cap).all()))
+        zb.z2z_profile_read(p.cb)
+        zb.z2z_decode_step(p.cb, hid[t], p.g_WE, p.g_WU, p.g_encE, p.g_encU, p.E_h, p.U_h, zb.SELECT_ARGMAX, 1.0,
+                           0, t, None, nxt, None, None, new, p.E_f32, p.U_f32)
+        _, launches = zb.z2z_profile_read(p.cb)                 # waits for the stream
+        passes.append(launches["encoder_gemm"] > 0)
+        for b in range(w.B):                                    # a created row was written on both sides
+            k = int(new[b].item())
+            if k >= 0:
+                assert float(p.E_f32[b, k].abs().max().item()) > 0 and float(p.U_f32[b, k].abs().max().item()) > 0
+    assert full_before[-1] and not full_before[0]               # the codebooks filled up on the way
+    first_full = full_before.index(True)
+    # not full before the step -> the pass ran; the first step that starts full reports it (and may
+    # still run the pass); every later step launches none
+    assert all(passes[:first_full]), (passes, full_before)
+    assert not any(passes[first_full + 1:]), (passes, full_before)
+
+
 def test_decode_step_results_written_to_pinned_host_memory():
     for w, sel in ((si.WORKLOADS["tiny"], zb.SELECT_ARGMAX), (SMALL_BF16, zb.SELECT_GUMBEL)):
         _decode_follow(w, 27, sel, steps=6, forced_every=3, host_results=True)
@@ -553,6 +592,7 @@ def test_weight_streaming_gemm_with_many_rows_in_one_box(w):
     # MMA (N = 240 / 144), one k-block per stage
     assert 2 * w.B * w.M > 128
     _decode_follow(w, 37, zb.SELECT_ARGMAX, steps=w.steps)
+    _decode_follow(w, 38, zb.SELECT_GUMBEL, steps=2)      # 24 rows: sampled on the decode-batch logits kernel
 
 
 ROWS_BF16 = si.Workload("rows_bf16", V=3000, d=256, dtype="bf16", B=2, T=220, M=3, cap=80,
@@ -657,6 +697,9 @@ TALL_BF16 = si.Workload("tall_bf16", V=40000, d=256, dtype="bf16", B=6, T=900, M
     ([16, 0, 0, 0, 0], True, 0, True),       # one sequence owns every row
     ([7, 7, 5, 5, 5], False, 0, False),      # 29 rows -> 32-row class
     ([6, 6, 6, 7, 7], True, 0, False),       # 32 rows, causal
+    ([7, 7, 5, 5, 5], True, 1, True),        # 29 rows: sampling and every output, two warps per lane quarter
+    ([6, 6, 6, 7, 7], False, 1, True),       # 32 rows, sampling and every output
+    ([0, 17, 0, 0, 0], True, 1, False),      # 17 rows of one sequence, sampling without the debug outputs
 ])
 def test_decode_logits_kernel_batches(rows, causal, select, debug):
     worst = _logits_case(PAIR_BF16, 51, rows, causal, select, debug=debug)
@@ -673,6 +716,7 @@ def test_decode_logits_kernel_fixed_shares_and_pool():
     # V = 40000: every CTA owns a fixed share of 128-row jobs and the pool holds both W_U and U_h
     _logits_case(TALL_BF16, 53, [1, 1, 1, 1, 1, 1], False, 0, debug=False)
     _logits_case(TALL_BF16, 54, [2, 3, 1, 4, 0, 2], True, 1, debug=True)
+    _logits_case(TALL_BF16, 55, [5, 6, 4, 7, 3, 6], True, 1, debug=True)        # 31 rows, sampled
 
 
 # ------------------------------------------------------------------------------------------------

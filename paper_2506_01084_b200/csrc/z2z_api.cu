@@ -65,6 +65,7 @@ z2z::EntryList entry_list(z2z_codebook* cb) {
   el.tok = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_tok);
   el.row_off = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_row_off);
   el.row_src = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_row_src);
+  el.row_tok = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_row_tok);
   el.off = reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_entry_off);
   el.chunk = cb->plan.enc_chunk_entries;
   return el;
@@ -304,7 +305,7 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
       z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
       Z2Z_CUDA(z2z::launch_entry_fill(cb->view, which, d_first, nullptr, el, c, s), "hyper_embed");
     }
-    if (tc) Z2Z_CUDA(z2z::run_encoder_pass_tc(cb->view, &a, 1, el, &cb->prof, s), "hyper_embed (tensor cores)");
+    if (tc) Z2Z_CUDA(z2z::run_encoder_pass_tc(cb->view, &a, 1, el, false, &cb->prof, s), "hyper_embed (tensor cores)");
     else Z2Z_CUDA(z2z::run_encoder_pass(cb->view, a, el, false, &cb->prof, s), "hyper_embed");
   }
   if (!d_first) {
@@ -421,7 +422,7 @@ int32_t z2z_decode_step(z2z_codebook* cb, const void* d_hidden, const void* d_WE
     g[0] = encoder_args(cb, d_WE, enc_E, d_Eh, d_Eh_f32, B, 0);
     if (!tied) g[1] = encoder_args(cb, d_WU, enc_U, d_Uh, d_Uh_f32, B, 1);
     if (tc) {
-      Z2Z_CUDA(z2z::run_encoder_pass_tc(cb->view, g, tied ? 1 : 2, el, &cb->prof, s), "decode_step (tensor cores)");
+      Z2Z_CUDA(z2z::run_encoder_pass_tc(cb->view, g, tied ? 1 : 2, el, fused, &cb->prof, s), "decode_step (tensor cores)");
     } else {
       Z2Z_CUDA(z2z::run_encoder_pass(cb->view, g[0], el, false, &cb->prof, s), "decode_step");
       if (!tied) {

@@ -68,7 +68,7 @@ struct WsPlan {
   int enc_chunk_entries;      // entries the encoder processes per pass
   int enc_rows;               // = enc_chunk_entries * M (rows padded to M per entry)
   size_t off_hash, off_cons, off_len, off_n, off_prev, off_status, off_n_emb, state_end;
-  size_t off_entry_seq, off_entry_idx, off_entry_len, off_entry_tok, off_row_off, off_row_src, off_entry_off, off_new_entry, off_sel;
+  size_t off_entry_seq, off_entry_idx, off_entry_len, off_entry_tok, off_row_off, off_row_src, off_row_tok, off_entry_off, off_new_entry, off_sel;
   size_t off_X, off_A, off_QKV, off_H;            // fp32 encoder activations
   size_t off_Ahl, off_Hhl;                        // bf16 hi/lo activations (tensor-core path)
   size_t off_g1_X, off_g1_QKV, off_g1_Ahl, off_g1_Hhl;   // second encoder of the decode step
@@ -113,6 +113,7 @@ inline WsPlan plan_workspace(const z2z_config& c) {
   p.off_entry_tok = take((size_t)chunk * c.M * 4);
   p.off_row_off = take((size_t)(chunk + 1) * 4);
   p.off_row_src = take((size_t)chunk * c.M * 4);
+  p.off_row_tok = take((size_t)chunk * c.M * 4);
   p.off_entry_off = take((size_t)(c.B + 2) * 4);
   p.off_new_entry = take((size_t)c.B * 4);
   p.off_sel = take((size_t)c.B * 4 * 4);

@@ -57,10 +57,15 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
     }
   }
   __syncthreads();
-  // ---- compact the new entries into the encoder's work list (exclusive scan over sequences)
+  // ---- compact the new entries into the encoder's work list (exclusive scan over sequences): an
+  // entry's slot in the list, and the first of the PACKED rows that its base tokens take (the
+  // tensor-core pass keeps no padding rows).  Both sums travel in one word: entries in the low
+  // half, rows in the high half (at most 1024 entries of at most 8 rows).
   const int mine = tid < cb.B ? s_cnt[tid] : 0;
   const int flag = mine > 0 ? 1 : 0;
-  int incl = flag;
+  const int my_len = flag ? (int)cb.len[(size_t)tid * cb.cap + (mine - 1)] : 0;     // written above by this block
+  const int val = flag | (my_len << 16);
+  int incl = val;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const int x = __shfl_up_sync(0xffffffffu, incl, o);
@@ -78,17 +83,26 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
     s_warp[lane] = w;
   }
   __syncthreads();
-  const int excl = incl - flag + (warp > 0 ? s_warp[warp - 1] : 0);
-  const int total = s_warp[31];
+  const int excl_both = incl - val + (warp > 0 ? s_warp[warp - 1] : 0);
+  const int excl = excl_both & 0xffff, row0 = excl_both >> 16;
+  const int total = s_warp[31] & 0xffff, total_rows = s_warp[31] >> 16;
   if (tid < cb.B) el.off[tid] = excl;
-  if (tid == 0) { el.off[cb.B] = total; el.off[cb.B + 1] = total < el.chunk ? total : el.chunk; }
+  if (tid == 0) {
+    el.off[cb.B] = total; el.off[cb.B + 1] = total < el.chunk ? total : el.chunk;
+    el.row_off[cb.B] = total_rows;                 // the pass that follows is sized for B entries
+  }
   if (flag && excl < el.chunk) {
     el.seq[excl] = tid; el.idx[excl] = mine - 1;
-    el.len[excl] = (int)cb.len[(size_t)tid * cb.cap + (mine - 1)];     // written above by this block
-    for (int i = 0; i < cb.M; ++i) el.tok[(size_t)excl * cb.M + i] = cb.cons[((size_t)tid * cb.cap + (mine - 1)) * cb.M + i];
+    el.len[excl] = my_len;
+    el.row_off[excl] = row0;
+    for (int i = 0; i < cb.M; ++i) {
+      const int tok = cb.cons[((size_t)tid * cb.cap + (mine - 1)) * cb.M + i];
+      el.tok[(size_t)excl * cb.M + i] = tok;
+      if (i < my_len) { el.row_src[row0 + i] = excl * cb.M + i; el.row_tok[row0 + i] = tok; }
+    }
   }
   for (int e = total + tid; e < el.chunk && e < cb.B; e += blockDim.x) {
-    el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0;
+    el.seq[e] = -1; el.idx[e] = 0; el.len[e] = 0; el.row_off[e] = total_rows;
     for (int i = 0; i < cb.M; ++i) el.tok[(size_t)e * cb.M + i] = -1;
   }
   // both caches will hold every entry once the encoder pass that follows has run

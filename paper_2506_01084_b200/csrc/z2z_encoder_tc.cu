@@ -8,14 +8,20 @@
 // and lo*w are exact in fp32, so A.W^T = hi.W^T + lo.W^T with fp32 accumulation.  Rounding the
 // activations to a single bf16 would leave the hyper-embeddings outside the 2e-2 tolerance.
 //
-// Layout of a hi/lo operand with Rt rows: bf16 [2 * Rt, K], hi rows first, lo rows after.
+// Rows are PACKED in both kinds of pass: entry e owns the rows row_off[e] .. row_off[e] + len[e],
+// there are no padding rows, and only the device knows how many rows a pass has (the word behind
+// the last entry slot of row_off).
+// Layout of a hi/lo operand: decode-sized passes (stream-K GEMM) keep the two parts of packed
+// row r in operand rows 2r and 2r + 1 of a bf16 [2 * Rt, K] matrix, so that the live rows are one
+// contiguous range whatever their number; prompt-sized passes (CTA-pair GEMM) keep hi rows
+// [0, Rt) first and lo rows [Rt, 2 Rt) after them.
 //
 // GEMM output.  Every CTA of the stream-K GEMM adds its partial tiles (hi and lo parts summed
 // in registers) into ONE fp32 matrix Y[group][Rt][J] with reductions in global memory; Y is all zero
 // whenever no GEMM result is pending.  The element-wise kernel after a GEMM reads each element of
-// that GEMM's result exactly once and stores zero back ("consume and clear"), for every row of
-// the pass whether or not it belongs to a live entry, which restores the invariant for the next
-// GEMM.  The session start clears Y once.
+// that GEMM's result exactly once and stores zero back ("consume and clear"), for every live row
+// of the pass (the GEMM adds nothing to rows beyond them), which restores the invariant for the
+// next GEMM.  The session start clears Y once.
 //
 // Launches per layer: GEMM(qkv) -> [+ bias, attention] -> GEMM(o) -> [+ bias + residual,
 // LayerNorm 2] -> GEMM(1) -> [+ bias, GELU] -> GEMM(2) -> [+ bias + residual, LayerNorm 1 of the
@@ -123,29 +129,23 @@ __device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[NV], int 
   }
 }
 
-// X = table[y] + pos for valid rows; then LN1 of layer 0 -> hi/lo.  grid (rows, groups).
+// X = table[y] + pos for every live packed row; then LN1 of layer 0 -> hi/lo.  grid (rows, groups).
 template <int NV>
-__global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryList el, Ptr2 table, Ptr2 pos,
-                                                              Ptr2 ln_w, Ptr2 ln_b, MPtr2 X, MPtr2 Ahl,
-                                                              int d, int Rt, int has_ln) {
+__global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryList el, const int* total, Ptr2 table,
+                                                              Ptr2 pos, Ptr2 ln_w, Ptr2 ln_b, MPtr2 X, MPtr2 Ahl,
+                                                              int d, int has_ln) {
   __shared__ float sm[32];
   sm100::pdl_trigger();            // the next kernel may start its prologue and weight prefetch
   sm100::pdl_wait();               // everything read or written below depends on earlier kernels
-  const int r = blockIdx.x, g = blockIdx.y, e = r / cb.M, i = r - e * cb.M;
-  const int y = el.tok[r];                        // the row's base token; loaded together with the count
-  if (e >= el.off[cb.B + 1]) return;
+  const int r = blockIdx.x, g = blockIdx.y;
+  const int y = el.row_tok[r];                    // the row's base token, its place in the entry and the
+  const int src = el.row_src[r];                  // row count: three independent loads
+  if (r >= *total) return;
+  const int i = src % cb.M;
   float* x = reinterpret_cast<float*>(X.p[g]) + (size_t)r * d;
-  bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)r * d;
-  bf16* lo = hi + (size_t)Rt * d;
+  bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)2 * r * d;
+  bf16* lo = hi + d;
   const int nvec = d / 4;
-  if (y < 0) {                                    // padding row: zero everywhere
-    for (int idx = threadIdx.x; idx < nvec; idx += kRowThreads) {
-      *reinterpret_cast<float4*>(x + idx * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-      *reinterpret_cast<uint2*>(hi + idx * 4) = make_uint2(0u, 0u);
-      *reinterpret_cast<uint2*>(lo + idx * 4) = make_uint2(0u, 0u);
-    }
-    return;
-  }
   const bf16* row = reinterpret_cast<const bf16*>(table.p[g]) + (size_t)y * d;
   const bf16* pp = reinterpret_cast<const bf16*>(pos.p[g]) + (size_t)i * d;
   const uint2* lw = reinterpret_cast<const uint2*>(ln_w.p[g]);
@@ -165,18 +165,18 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln(CbView cb, EntryLi
   if (has_ln) layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, lo, d, sm);
 }
 
-// x = X[r] + Y[r] + bias for a valid row (Y consumed and cleared for every row); then
-// LayerNorm -> hi/lo for the next GEMM.  grid (rows, groups).  All loads (entry length, Y, X, bias,
-// gamma, beta) are issued together; whether the row is valid only decides what is stored.
+// x = X[r] + Y[r] + bias for a live packed row (Y consumed and cleared); then LayerNorm -> hi/lo
+// for the next GEMM.  grid (rows, groups).  All loads (row count, Y, X, bias, gamma, beta) are
+// issued together; whether the row is live only decides what is stored.
 template <int NV>
-__global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, EntryList el, float* Y, Ptr2 bias,
+__global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(const int* total, float* Y, Ptr2 bias,
                                                                     MPtr2 X, Ptr2 ln_w, Ptr2 ln_b, MPtr2 Ahl,
                                                                     int d, int Rt) {
   __shared__ float sm[32];
   sm100::pdl_trigger();
   sm100::pdl_wait();
-  const int r = blockIdx.x, g = blockIdx.y, e = r / cb.M, i = r - e * cb.M;
-  const int L = entry_len_tc(cb, el, e);
+  const int r = blockIdx.x, g = blockIdx.y;
+  const int live = *total;
   float* y = Y + ((size_t)g * Rt + r) * d;
   float* x = reinterpret_cast<float*>(X.p[g]) + (size_t)r * d;
   const uint2* bs = reinterpret_cast<const uint2*>(bias.p[g]);
@@ -194,26 +194,23 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_ln(CbView cb, E
       bv[v] = bs[idx]; gw[v] = lw[idx]; gb[v] = lb[idx];
     }
   }
-  const bool valid = i < L;
+  if (r >= live) return;                          // nothing was added to this row of Y: it is still zero
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
     const int idx = (int)threadIdx.x + v * kRowThreads;
     if (idx < nvec) {
       *reinterpret_cast<float4*>(y + idx * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (valid) {
-        const float4 b = unpack_bf16x4(bv[v]);
-        xv[v] = make_float4(xv[v].x + yv[v].x + b.x, xv[v].y + yv[v].y + b.y, xv[v].z + yv[v].z + b.z,
-                            xv[v].w + yv[v].w + b.w);
-        *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
-      }
+      const float4 b = unpack_bf16x4(bv[v]);
+      xv[v] = make_float4(xv[v].x + yv[v].x + b.x, xv[v].y + yv[v].y + b.y, xv[v].z + yv[v].z + b.z,
+                          xv[v].w + yv[v].w + b.w);
+      *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
     }
   }
-  if (!valid) return;                             // padding rows stay zero in X and in hi/lo
-  bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)r * d;
-  layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
+  bf16* hi = reinterpret_cast<bf16*>(Ahl.p[g]) + (size_t)2 * r * d;
+  layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, hi + d, d, sm);
 }
 
-// Last layer: x_i = X[r_i] + Y[r_i] + bias for the entry's valid rows, cache row = mean_i x_i.
+// Last layer: x_i = X[r_i] + Y[r_i] + bias for the entry's rows, cache row = mean_i x_i.
 // grid (entries, groups, ceil(d / (4 * kRowThreads))): a thread owns 4 columns of the entry and
 // issues the loads of all its rows before it adds.
 __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb, EntryList el, float* Y, Ptr2 bias,
@@ -225,28 +222,27 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb,
   const int col = ((int)blockIdx.z * kRowThreads + (int)threadIdx.x) * 4;
   if (col >= d) return;
   const int L = entry_len_tc(cb, el, e);
+  const int r0 = el.row_off[e];
   const int seq = el.seq[e], idx = el.idx[e];
   const float4 b = load_bf16x4(reinterpret_cast<const bf16*>(bias.p[g]) + col);
+  if (L <= 0) return;
   float4 yv[kMaxM], xv[kMaxM];
 #pragma unroll
   for (int i = 0; i < kMaxM; ++i)
-    if (i < cb.M) {
-      const size_t r = (size_t)e * cb.M + i;
+    if (i < L) {
+      const size_t r = (size_t)r0 + i;
       yv[i] = *reinterpret_cast<const float4*>(Y + ((size_t)g * Rt + r) * d + col);
       xv[i] = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X.p[g]) + r * d + col);
     }
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
   for (int i = 0; i < kMaxM; ++i)
-    if (i < cb.M) {
-      const size_t r = (size_t)e * cb.M + i;
+    if (i < L) {
+      const size_t r = (size_t)r0 + i;
       *reinterpret_cast<float4*>(Y + ((size_t)g * Rt + r) * d + col) = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (i < L) {
-        acc.x += xv[i].x + yv[i].x + b.x; acc.y += xv[i].y + yv[i].y + b.y;
-        acc.z += xv[i].z + yv[i].z + b.z; acc.w += xv[i].w + yv[i].w + b.w;
-      }
+      acc.x += xv[i].x + yv[i].x + b.x; acc.y += xv[i].y + yv[i].y + b.y;
+      acc.z += xv[i].z + yv[i].z + b.z; acc.w += xv[i].w + yv[i].w + b.w;
     }
-  if (L <= 0) return;
   const size_t dst = ((size_t)seq * cb.cap + idx) * d + col;
   const float inv = 1.0f / (float)L;
   const float4 m = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
@@ -256,7 +252,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_reduce_resid_pool(CbView cb,
   if (out32) *reinterpret_cast<float4*>(out32 + dst) = m;
 }
 
-// Zero-layer encoder (the parameter-free averaging variant): cache row = mean of X rows.
+// Zero-layer encoder (the parameter-free averaging variant): cache row = mean of the entry's X rows.
 __global__ void __launch_bounds__(kRowThreads) k_tc_pool(CbView cb, EntryList el, MPtr2 X, MPtr2 cache,
                                                          MPtr2 cache_f32, int d) {
   sm100::pdl_trigger();
@@ -264,33 +260,35 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_pool(CbView cb, EntryList el
   const int e = blockIdx.x, g = blockIdx.y;
   const int L = entry_len_tc(cb, el, e);
   if (L <= 0) return;
-  const float* x = reinterpret_cast<const float*>(X.p[g]);
+  const float* x = reinterpret_cast<const float*>(X.p[g]) + (size_t)el.row_off[e] * d;
   const size_t dst = ((size_t)el.seq[e] * cb.cap + el.idx[e]) * d;
   const float inv = 1.0f / (float)L;
   bf16* out = reinterpret_cast<bf16*>(cache.p[g]);
   float* out32 = reinterpret_cast<float*>(cache_f32.p[g]);
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
     float v = 0.f;
-    for (int i = 0; i < L; ++i) v += x[((size_t)e * cb.M + i) * d + c];
+    for (int i = 0; i < L; ++i) v += x[(size_t)i * d + c];
     v *= inv;
     out[dst + c] = __float2bfloat16_rn(v);
     if (out32) out32[dst + c] = v;
   }
 }
 
-// H = GELU(Y + bias) -> hi/lo (Y consumed and cleared).  The [groups * R, J] results are one flat
-// range of float4; every thread takes kGeluPerThread of them, kGeluThreads apart, and issues all of
-// its loads before it computes.  grid = ceil(groups * R * J / 4 / (kGeluThreads * kGeluPerThread)).
+// H = GELU(Y + bias) -> hi/lo (Y consumed and cleared) for the live packed rows.  The
+// [groups * R, J] results are one flat range of float4; every thread takes kGeluPerThread of them,
+// kGeluThreads apart, and issues all of its loads before it computes.
+// grid = ceil(groups * R * J / 4 / (kGeluThreads * kGeluPerThread)), R = row capacity of the pass.
 constexpr int kGeluThreads = 256, kGeluPerThread = 4;
-__global__ void __launch_bounds__(kGeluThreads) k_tc_reduce_gelu(CbView cb, EntryList el, float* Y, Ptr2 bias, MPtr2 Hhl,
+__global__ void __launch_bounds__(kGeluThreads) k_tc_reduce_gelu(const int* total_rows, float* Y, Ptr2 bias, MPtr2 Hhl,
                                                                  int J, int R, int Rt, int ng) {
   sm100::pdl_trigger();
   sm100::pdl_wait();
   const int J4 = J / 4;
   const long long total = (long long)ng * R * J4;
   const long long base = (long long)blockIdx.x * (kGeluThreads * kGeluPerThread) + threadIdx.x;
+  const int live = *total_rows;
   float4 q[kGeluPerThread], bs[kGeluPerThread];
-  int row[kGeluPerThread], jj[kGeluPerThread], len[kGeluPerThread];
+  int row[kGeluPerThread], jj[kGeluPerThread];
 #pragma unroll
   for (int k = 0; k < kGeluPerThread; ++k) {
     const long long f = base + (long long)k * kGeluThreads;
@@ -301,27 +299,26 @@ __global__ void __launch_bounds__(kGeluThreads) k_tc_reduce_gelu(CbView cb, Entr
       const int g = row[k] / R, r = row[k] - g * R;
       q[k] = *reinterpret_cast<const float4*>(Y + ((size_t)g * Rt + r) * J + jj[k]);
       bs[k] = load_bf16x4(reinterpret_cast<const bf16*>(bias.p[g]) + jj[k]);
-      len[k] = entry_len_tc(cb, el, r / cb.M);
     }
   }
 #pragma unroll
   for (int k = 0; k < kGeluPerThread; ++k) {
     if (row[k] < 0) continue;
     const int g = row[k] / R, r = row[k] - g * R;
+    if (r >= live) continue;                       // no row there: Y is still zero, nothing reads the operand row
     *reinterpret_cast<float4*>(Y + ((size_t)g * Rt + r) * J + jj[k]) = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (len[k] <= 0) continue;                     // unused slot: nothing reads its rows
     float4 v = make_float4(q[k].x + bs[k].x, q[k].y + bs[k].y, q[k].z + bs[k].z, q[k].w + bs[k].w);
     v.x = 0.5f * v.x * (1.0f + erff(v.x * 0.70710678118654752440f));
     v.y = 0.5f * v.y * (1.0f + erff(v.y * 0.70710678118654752440f));
     v.z = 0.5f * v.z * (1.0f + erff(v.z * 0.70710678118654752440f));
     v.w = 0.5f * v.w * (1.0f + erff(v.w * 0.70710678118654752440f));
-    bf16* hi = reinterpret_cast<bf16*>(Hhl.p[g]) + (size_t)r * J + jj[k];
-    split_store4(hi, hi + (size_t)Rt * J, v);
+    bf16* hi = reinterpret_cast<bf16*>(Hhl.p[g]) + (size_t)2 * r * J + jj[k];
+    split_store4(hi, hi + J, v);
   }
 }
 
 // q, k, v = Y + bias for one head of one entry (consumed, cleared, staged in shared memory), then
-// bidirectional attention over the entry's valid rows; output as hi/lo.
+// bidirectional attention over the entry's rows; output as hi/lo.
 // grid (entries, heads, groups), block (32, M), dynamic smem M * 3 * dh floats; dh % 4 == 0.
 __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias, MPtr2 Ohl, int d, int heads,
                                    int Rt) {
@@ -330,15 +327,15 @@ __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias,
   sm100::pdl_wait();
   const int e = blockIdx.x, h = blockIdx.y, g = blockIdx.z, i = threadIdx.y, lane = threadIdx.x;
   const int L = entry_len_tc(cb, el, e);
+  const int r = el.row_off[e] + i;               // packed row of position i (only used while i < L)
   const int dh = d / heads;
-  const int r = e * cb.M + i;
-  {
+  if (i < L) {
     const bf16* bs = reinterpret_cast<const bf16*>(bias.p[g]);
     float* y = Y + ((size_t)g * Rt + r) * 3 * d;
     for (int c = lane * 4; c < dh; c += 128) {
       float4 p[3], b[3];
 #pragma unroll
-      for (int w = 0; w < 3; ++w) {                // the six loads are independent of one another and of L
+      for (int w = 0; w < 3; ++w) {                // the six loads are independent of one another
         const int col = w * d + h * dh + c;
         p[w] = *reinterpret_cast<const float4*>(y + col);
         b[w] = load_bf16x4(bs + col);
@@ -346,14 +343,13 @@ __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias,
 #pragma unroll
       for (int w = 0; w < 3; ++w) {
         *reinterpret_cast<float4*>(y + w * d + h * dh + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (i < L)
-          *reinterpret_cast<float4*>(&s_qkv[(i * 3 + w) * dh + c]) =
-              make_float4(p[w].x + b[w].x, p[w].y + b[w].y, p[w].z + b[w].z, p[w].w + b[w].w);
+        *reinterpret_cast<float4*>(&s_qkv[(i * 3 + w) * dh + c]) =
+            make_float4(p[w].x + b[w].x, p[w].y + b[w].y, p[w].z + b[w].z, p[w].w + b[w].w);
       }
     }
   }
   __syncthreads();
-  if (i >= L) return;                          // padding rows of the operand stay zero
+  if (i >= L) return;
   const float* q = s_qkv + (i * 3) * dh;
   const float scale = 1.0f / sqrtf((float)dh);
   float s[kMaxM];
@@ -375,8 +371,8 @@ __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias,
 #pragma unroll
   for (int j = 0; j < kMaxM; ++j) { s[j] = j < L ? expf(s[j] - mx) : 0.f; den += s[j]; }
   const float inv = 1.0f / den;
-  bf16* hi = reinterpret_cast<bf16*>(Ohl.p[g]) + (size_t)r * d + (size_t)h * dh;
-  bf16* lo = hi + (size_t)Rt * d;
+  bf16* hi = reinterpret_cast<bf16*>(Ohl.p[g]) + (size_t)2 * r * d + (size_t)h * dh;
+  bf16* lo = hi + d;
   for (int c = lane; c < dh; c += 32) {
     float v = 0.f;
 #pragma unroll
@@ -388,12 +384,13 @@ __global__ void k_tc_qkv_attention(CbView cb, EntryList el, float* Y, Ptr2 bias,
   }
 }
 
-// Prompt-sized passes keep their rows PACKED: entry e owns rows row_off[e] .. row_off[e] + len[e],
-// there are no padding rows inside entries, and rows at or beyond the total carry nothing.  (With
-// M = 3 or 4 a quarter to a third of the padded rows would be zeros that the GEMMs multiply anyway.)
+// Packed rows: entry e owns rows row_off[e] .. row_off[e] + len[e], there are no padding rows
+// inside entries, and rows at or beyond the total carry nothing.  (With M = 3 or 4 a quarter to a
+// third of padded rows would be zeros that the GEMMs load and multiply anyway.)
 //
 // One block: first packed row of every entry (exclusive scan of the lengths), the total behind the
-// last entry, and the way back from a packed row to (entry, position).  E <= 1024 entries.
+// last entry slot, the way back from a packed row to (entry, position) and the row's base token.
+// E <= 1024 entries.  (The decode step's update kernel writes the same map itself.)
 __global__ void __launch_bounds__(1024) k_tc_row_map(CbView cb, EntryList el, int E) {
   __shared__ int warp_sums[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -419,7 +416,10 @@ __global__ void __launch_bounds__(1024) k_tc_row_map(CbView cb, EntryList el, in
   const int excl = inc - len + (warp > 0 ? warp_sums[warp - 1] : 0);
   if (tid < E) {
     el.row_off[tid] = excl;
-    for (int i = 0; i < len; ++i) el.row_src[excl + i] = tid * cb.M + i;
+    for (int i = 0; i < len; ++i) {
+      el.row_src[excl + i] = tid * cb.M + i;
+      el.row_tok[excl + i] = el.tok[tid * cb.M + i];
+    }
   }
   if (tid == 0) el.row_off[E] = warp_sums[31];
 }
@@ -695,15 +695,15 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
 }
 
 cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng, const EntryList& el,
-                                Prof* prof, cudaStream_t s) {
+                                bool rows_mapped, Prof* prof, cudaStream_t s) {
   const EncoderArgs& a0 = grp[0];
   const int d = a0.d, dff = a0.dff, M = cb.M;
   const int E = a0.entries < el.chunk ? a0.entries : el.chunk;
-  const int R = E * M;                                 // rows of this pass
+  const int R = E * M;                                 // row capacity of this pass
   if (ng == 1 && R >= kPairPassMinRows) return run_encoder_pass_pair(cb, a0, el, E, prof, s);
-  const int Rt = (R + 7) / 8 * 8;                      // rows per hi (or lo) block
+  const int Rt = (R + 7) / 8 * 8;                      // rows of the result matrix per group
   const int row_tiles = (Rt + 127) / 128;
-  const bool one_box = row_tiles == 1;                 // hi and lo rows (2 Rt <= 256) are one operand box
+  const int* total = el.row_off + E;                   // packed rows of this pass (device word)
   const int n_sm = sm_count();
   const bool narrow = d <= 4 * kRowThreads * kNarrowVec4;      // a row fits four float4 per thread
   auto rlk = narrow ? k_tc_reduce_resid_ln<kNarrowVec4> : k_tc_reduce_resid_ln<kMaxVec4>;
@@ -720,21 +720,16 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
   const MPtr2 c32 = M2([](const EncoderArgs& a) { return (void*)a.cache_f32; });
   const Ptr2 table = P2([](const EncoderArgs& a) { return a.table; });
 
-  // one GEMM: activations (hi/lo, K columns) x weight [J, K], added into Y[group][Rt][J]
+  // one GEMM: activations (hi/lo of packed row r in operand rows 2r, 2r + 1; K columns) x weight
+  // [J, K], added into Y[group][Rt][J]
   auto gemm = [&](const MPtr2& act, int K, int widx, int J) -> cudaError_t {
     StreamGemmParams p{};
     p.row_tiles = row_tiles; p.groups = ng; p.tiles_per_group = J / kNT;
-    // hi rows [0, Rt) and lo rows [Rt, 2 Rt) of the operand are one contiguous box while they fit
-    // the MMA's N (256); beyond that a row tile takes its 128 hi rows and its 128 lo rows as two boxes
-    p.a_parts = one_box ? 1 : 2;
-    p.a_box_rows = one_box ? 2 * Rt : 128;
-    p.a_part_row = Rt;
-    p.n_act = p.a_parts * p.a_box_rows;
-    p.lo_col = one_box ? Rt : 128;
+    p.a_box_rows = row_tiles == 1 ? 2 * Rt : 256;      // one box per stage: all operand rows of a row tile
     // two k-blocks per stage (fewer TMA operations per byte) while at least four stages still fit
-    p.ksb = (one_box && K % 128 == 0 && stream_gemm_stages(2, p.n_act) >= 4) ? 2 : 1;
+    p.ksb = (K % 128 == 0 && stream_gemm_stages(2, p.a_box_rows) >= 4) ? 2 : 1;
     p.ksteps = (K / 64 + p.ksb - 1) / p.ksb;
-    p.out = Y; p.J = J; p.Rt = Rt; p.valid_rows = R;
+    p.out = Y; p.J = J; p.Rt = Rt; p.rows_dev = total;
     p.err = a0.err;
     const long long tiles = (long long)row_tiles * ng * p.tiles_per_group;
     const int G = tiles * p.ksteps < n_sm ? (int)(tiles * p.ksteps) : n_sm;     // every CTA owns >= 1 unit
@@ -748,11 +743,15 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
     return launch_stream_gemm(p, maps, G, s);
   };
 
+  if (!rows_mapped) {
+    ProfScope ps(prof, kProfEncOther, 1, s);
+    k_tc_row_map<<<1, 1024, 0, s>>>(cb, el, E);
+  }
   cudaError_t e;
   {
     ProfScope ps(prof, kProfEncOther, 1, s);
-    launch_pdl(narrow ? k_tc_gather_ln<kNarrowVec4> : k_tc_gather_ln<kMaxVec4>, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, table, W(0), a0.layers ? W(1) : W(0),
-               a0.layers ? W(2) : W(0), X, Ahl, d, Rt, a0.layers > 0 ? 1 : 0);
+    launch_pdl(narrow ? k_tc_gather_ln<kNarrowVec4> : k_tc_gather_ln<kMaxVec4>, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, total, table, W(0), a0.layers ? W(1) : W(0),
+               a0.layers ? W(2) : W(0), X, Ahl, d, a0.layers > 0 ? 1 : 0);
   }
   if (a0.layers == 0) {
     ProfScope ps(prof, kProfEncOther, 1, s);
@@ -773,7 +772,7 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
     if (dff > 0) {                                     // dff == 0: attention-only layer
       {
         ProfScope ps(prof, kProfEncOther, 1, s);
-        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(o + 5), X, W(o + 6),
+        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, total, Y, W(o + 5), X, W(o + 6),
                    W(o + 7), Ahl, d, Rt);
       }
       if ((e = gemm(Ahl, d, o + 8, dff)) != cudaSuccess) return e;
@@ -781,7 +780,7 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
         ProfScope ps(prof, kProfEncOther, 1, s);
         const long long f4 = (long long)ng * R * (dff / 4);
         const int per_cta = kGeluThreads * kGeluPerThread;
-        launch_pdl(k_tc_reduce_gelu, dim3((unsigned)((f4 + per_cta - 1) / per_cta)), dim3(kGeluThreads), 0, s, cb, el, Y,
+        launch_pdl(k_tc_reduce_gelu, dim3((unsigned)((f4 + per_cta - 1) / per_cta)), dim3(kGeluThreads), 0, s, total, Y,
                    W(o + 9), Hhl, dff, R, Rt, ng);
       }
       if ((e = gemm(Hhl, dff, o + 10, d)) != cudaSuccess) return e;
@@ -793,7 +792,7 @@ cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* grp, int ng
         launch_pdl(k_tc_reduce_resid_pool, dim3(E, ng, (d / 4 + kRowThreads - 1) / kRowThreads), dim3(kRowThreads), 0,
                    s, cb, el, Y, W(last_bias), X, cache, c32, d, Rt);
       else
-        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, cb, el, Y, W(last_bias), X, W(o + 12),
+        launch_pdl(rlk, dim3(R, ng), dim3(kRowThreads), 0, s, total, Y, W(last_bias), X, W(o + 12),
                    W(o + 13), Ahl, d, Rt);
     }
   }

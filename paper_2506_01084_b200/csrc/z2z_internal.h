@@ -47,8 +47,10 @@ struct EntryList {
   int32_t* idx;       // [chunk]  entry number within the sequence
   int32_t* len;       // [chunk]  base tokens of the entry, 0 for an unused slot
   int32_t* tok;       // [chunk * M]  base token of each row of the entry, -1 for padding rows
-  int32_t* row_off;   // [chunk + 1]  prompt-sized passes: first packed row of each entry, then the row total
-  int32_t* row_src;   // [chunk * M]  prompt-sized passes: packed row -> entry * M + position
+  int32_t* row_off;   // [chunk + 1]  tensor-core passes: first packed row of each entry; the row total sits
+                      //              behind the last entry slot of the pass
+  int32_t* row_src;   // [chunk * M]  tensor-core passes: packed row -> entry * M + position
+  int32_t* row_tok;   // [chunk * M]  tensor-core passes: base token of each packed row
   int32_t* off;       // [B + 2]  exclusive prefix sum of per-sequence counts, then the total
   int chunk;
 };
@@ -69,8 +71,9 @@ struct EncoderArgs {
 bool encoder_tc_supported(int d, int dff, int dtype, int heads, int M);
 bool logits_tc_supported(int d, int dtype);
 // Two encoders (embedding side, unembedding side) run through the same launches.
+// rows_mapped: the packed-row map of the work list (row_off, row_src, row_tok) is already there.
 cudaError_t run_encoder_pass_tc(const CbView& cb, const EncoderArgs* groups, int n_groups,
-                                const EntryList& el, Prof* prof, cudaStream_t s);
+                                const EntryList& el, bool rows_mapped, Prof* prof, cudaStream_t s);
 // Per-sequence ranges from (first, count) arrays, or "everything since the last call" when NULL.
 cudaError_t launch_entry_offsets(const CbView& cb, int which, const int32_t* first,
                                  const int32_t* count, const EntryList& el, cudaStream_t s);

@@ -17,6 +17,9 @@
 //     score per hidden row in registers, so the logits are never written.  Only the hidden rows
 //     that exist are loaded: the MMA also reads the shared memory behind them, which only feeds
 //     accumulator rows nobody reads (rows of D depend on the same rows of A only).
+#include <mutex>
+#include <unordered_map>
+
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
 #include "z2z_sm100.cuh"
@@ -242,6 +245,15 @@ __host__ __device__ constexpr uint32_t gemm_tmem_cols(int n_act) {
   return 2 * n_act <= 32 ? 32u : (2 * n_act <= 64 ? 64u : (2 * n_act <= 128 ? 128u : (2 * n_act <= 256 ? 256u : 512u)));
 }
 
+// Live packed rows of row tile `arow / 128`, rounded up to 8 (at least 8, at most half a box).
+__device__ __forceinline__ int gemm_tile_rows8(const StreamGemmParams& p, int live, int arow) {
+  int rows = live - arow;
+  rows = rows < 1 ? 1 : rows;
+  rows = (rows + 7) & ~7;
+  const int cap = p.a_box_rows / 2;
+  return rows > cap ? cap : rows;
+}
+
 template <int KSB, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0,
@@ -253,14 +265,14 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(sm);
   const uint32_t stage_base = smem_u32(sm + 1024);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t a_part_bytes = (uint32_t)KSB * p.a_box_rows * 128;
-  const uint32_t a_bytes = p.a_parts * a_part_bytes;
+  const uint32_t a_bytes = (uint32_t)KSB * p.a_box_rows * 128;
   const uint32_t stage_bytes = a_bytes + (uint32_t)KSB * NT * 128;
+  const bool shifted = p.row_tiles == 1;           // one row tile: the box is shifted so that only live rows are read
   pdl_trigger();                                   // the next kernel may get resident behind this one
   setup_barriers<STAGES>(ctrl);
   if (warp == 0 && lane == 0) { prefetch_tmap(&tmA0); prefetch_tmap(&tmW0); if (p.groups > 1) { prefetch_tmap(&tmA1); prefetch_tmap(&tmW1); } }
   __syncthreads();
-  if (warp == 2) { tmem_alloc(smem_u32(&ctrl->tmem_base), gemm_tmem_cols(p.n_act)); tmem_relinquish(); }
+  if (warp == 2) { tmem_alloc(smem_u32(&ctrl->tmem_base), gemm_tmem_cols(p.a_box_rows)); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -271,18 +283,25 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
       // ---- TMA producer.  The weight tiles depend on no earlier kernel, the activation tiles do:
       // during the first pass over the ring only the weight boxes are issued and the activation
       // boxes are noted; once the ring is full (or the work ends) the producer waits for the
-      // preceding kernel and issues them.  With an ordinary launch the wait returns at once.
+      // preceding kernel, learns how many rows are live and issues them.  With an ordinary launch
+      // the wait returns at once.
       const CUtensorMap* amaps[2] = {&tmA0, &tmA1};
       const CUtensorMap* wmaps[2] = {&tmW0, &tmW1};
       const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
-      struct Deferred { uint32_t dst, bar; int map, row, kb; };
-      Deferred def[kMaxStages * 2];
-      int n_def = 0, issued = 0;
+      struct Deferred { uint32_t dst, bar; int map, arow, kb; };
+      Deferred def[kMaxStages];
+      int n_def = 0, issued = 0, live = 0;
       bool deps = false, ok = true;
+      // first operand row of the box of the row tile that starts at packed row `arow`
+      auto box_row = [&](int arow) {
+        return shifted ? 2 * gemm_tile_rows8(p, live, arow) - p.a_box_rows : 2 * arow;
+      };
       auto need_deps = [&]() {
         if (deps) return;
         pdl_wait();
-        for (int i = 0; i < n_def; ++i) tma_load_3d(def[i].dst, amaps[def[i].map], 0, def[i].row, def[i].kb, def[i].bar, pol_a);
+        live = *p.rows_dev;
+        for (int i = 0; i < n_def; ++i)
+          tma_load_3d(def[i].dst, amaps[def[i].map], 0, box_row(def[i].arow), def[i].kb, def[i].bar, pol_a);
         deps = true;
       };
       int stage = 0; uint32_t phase = 0;
@@ -293,15 +312,11 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
           if (issued == STAGES) need_deps();
           if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctrl->full[stage]);
-          mbar_expect_tx(full, stage_bytes);
+          mbar_expect_tx(full, stage_bytes);        // rows of a box outside the tensor are zero-filled and counted
           const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
           tma_load_3d(sb + a_bytes, wmaps[j.g], 0, j.wrow, ks * KSB, full, pol_w);
-          for (int part = 0; part < p.a_parts; ++part) {
-            const uint32_t dst = sb + part * a_part_bytes;
-            const int row = j.arow + part * p.a_part_row;
-            if (deps) tma_load_3d(dst, amaps[j.g], 0, row, ks * KSB, full, pol_a);
-            else { def[n_def].dst = dst; def[n_def].bar = full; def[n_def].map = j.g; def[n_def].row = row; def[n_def].kb = ks * KSB; ++n_def; }
-          }
+          if (deps) tma_load_3d(sb, amaps[j.g], 0, box_row(j.arow), ks * KSB, full, pol_a);
+          else { def[n_def].dst = sb; def[n_def].bar = full; def[n_def].map = j.g; def[n_def].arow = j.arow; def[n_def].kb = ks * KSB; ++n_def; }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -310,8 +325,9 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      // ---- MMA issue: D[128 weight rows][n_act] += W tile (M operand) x activations (N operand)
-      const uint32_t idesc = idesc_bf16_f32(128, p.n_act);
+      // ---- MMA issue: D[128 weight rows][n] += W tile (M operand) x live activation rows (N operand)
+      pdl_wait();                                      // the live-row count comes from an earlier kernel
+      const int live = *p.rows_dev;
       int stage = 0; uint32_t phase = 0, job_i = 0;
       bool ok = true;
       GemmWalk walk(p);
@@ -320,7 +336,11 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
         const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
         if (!mbar_wait(smem_u32(&ctrl->acc_empty[buf]), aph ^ 1u, &ctrl->abort)) break;
         tc_fence_after();
-        const uint32_t d = tmem_base + buf * (uint32_t)p.n_act;
+        // N and the operand's first row inside the box (a multiple of 8 rows = one swizzle atom)
+        const int n_rows = shifted ? 2 * gemm_tile_rows8(p, live, j.arow) : p.a_box_rows;
+        const uint32_t a_off = (uint32_t)(p.a_box_rows - n_rows) * 128;
+        const uint32_t idesc = idesc_bf16_f32(128, n_rows);
+        const uint32_t d = tmem_base + buf * (uint32_t)p.a_box_rows;
         uint32_t acc = 0;
         for (int ks = j.kb0; ks < j.kb1; ++ks) {
           if (!mbar_wait(smem_u32(&ctrl->full[stage]), phase, &ctrl->abort)) { ok = false; break; }
@@ -328,8 +348,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
           const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
 #pragma unroll
           for (int i = 0; i < KSB; ++i) {
-            // with two boxes per stage KSB is 1 and the boxes are adjacent: n_act contiguous rows
-            const uint32_t ab = sb + (uint32_t)i * p.a_box_rows * 128;
+            const uint32_t ab = sb + (uint32_t)i * p.a_box_rows * 128 + a_off;
             const uint32_t wb = sb + a_bytes + (uint32_t)i * NT * 128;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -347,8 +366,10 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
     }
   } else {
     // ---- epilogue: a thread owns one output feature of the tile (its TMEM lane) and walks the
-    // activation rows (TMEM columns): hi + lo in registers, one reduction per (row, feature)
+    // live activation rows (pairs of TMEM columns): hi + lo in registers, one reduction per
+    // (row, feature)
     pdl_wait();                                      // the result matrix may still be read by the kernel before
+    const int live = *p.rows_dev;
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
     const int feature = q * 32 + lane;
     uint32_t job_i = 0;
@@ -358,19 +379,18 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
       const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
       if (!mbar_wait(smem_u32(&ctrl->acc_full[buf]), aph, &ctrl->abort)) break;
       tc_fence_after();
-      int rows = p.valid_rows - j.arow;              // live activation rows of this row tile
-      rows = rows > p.lo_col ? p.lo_col : rows;
+      int rows = live - j.arow;                      // live activation rows of this row tile
+      rows = rows > 128 ? 128 : rows;
       float* dst = p.out + ((size_t)j.g * p.Rt + j.arow) * p.J + j.wrow + feature;
-      const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)p.n_act;
+      const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)p.a_box_rows;
 #pragma unroll 1
       for (int r0 = 0; r0 < rows; r0 += 8) {
-        uint32_t hi[8], lo[8];
-        tmem_ld8(t0 + r0, hi);
-        tmem_ld8(t0 + p.lo_col + r0, lo);
+        uint32_t v[16];
+        tmem_ld16(t0 + 2 * r0, v);
         tmem_ld_wait();
 #pragma unroll
         for (int x = 0; x < 8; ++x)
-          if (r0 + x < rows) red_add_f32(dst + (size_t)(r0 + x) * p.J, __uint_as_float(hi[x]) + __uint_as_float(lo[x]));
+          if (r0 + x < rows) red_add_f32(dst + (size_t)(r0 + x) * p.J, __uint_as_float(v[2 * x]) + __uint_as_float(v[2 * x + 1]));
       }
       tc_fence_before();
       __syncwarp();
@@ -381,7 +401,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.err, 1);
-  if (warp == 2) tmem_dealloc(tmem_base, gemm_tmem_cols(p.n_act));
+  if (warp == 2) tmem_dealloc(tmem_base, gemm_tmem_cols(p.a_box_rows));
 }
 
 // =================================================================================================
@@ -585,6 +605,29 @@ bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long 
 // Tensor map over the same matrix seen as [cols / 64 k-blocks][rows][64]: one box brings
 // `box_kb` k-blocks of `box_rows` rows, laid out k-block after k-block (each k-block is then a
 // K-major 128-byte-swizzled operand tile).
+//
+// A map is a pure function of (base, rows, cols, box): the encoded maps are kept, so that a decode
+// step, whose operands sit at the same addresses step after step, encodes none in steady state.
+namespace {
+struct TmapKey {
+  const void* base; long long rows, cols; int box_rows, box_kb;
+  bool operator==(const TmapKey& o) const {
+    return base == o.base && rows == o.rows && cols == o.cols && box_rows == o.box_rows && box_kb == o.box_kb;
+  }
+};
+struct TmapKeyHash {
+  size_t operator()(const TmapKey& k) const {
+    size_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+    h ^= (size_t)k.rows * 0xC2B2AE3D27D4EB4Full + (size_t)k.cols * 0x165667B19E3779F9ull;
+    h ^= ((size_t)k.box_rows << 20) ^ (size_t)k.box_kb;
+    return h;
+  }
+};
+constexpr size_t kTmapCacheMax = 4096;           // entries kept; the cache starts over beyond that
+std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> g_tmap_cache;
+std::mutex g_tmap_mu;
+}  // namespace
+
 bool make_tmap_bf16_kblocks(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows,
                             int box_kb) {
   EncodeTiledFn fn = encode_fn();
@@ -592,13 +635,24 @@ bool make_tmap_bf16_kblocks(CUtensorMap* m, const void* base, long long rows, lo
   if ((reinterpret_cast<uintptr_t>(base) & 15) || (cols % 64) || box_rows < 1 || box_rows > 256 || box_kb < 1 ||
       box_kb > 256 || rows < 1)
     return false;
+  const TmapKey key{base, rows, cols, box_rows, box_kb};
+  {
+    std::lock_guard<std::mutex> lock(g_tmap_mu);
+    auto it = g_tmap_cache.find(key);
+    if (it != g_tmap_cache.end()) { *m = it->second; return true; }
+  }
   cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
   cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128};
   cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_kb};
   cuuint32_t es[3] = {1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  std::lock_guard<std::mutex> lock(g_tmap_mu);
+  if (g_tmap_cache.size() >= kTmapCacheMax) g_tmap_cache.clear();
+  g_tmap_cache.emplace(key, *m);
+  return true;
 }
 
 template <int NT, int KSB>
@@ -609,16 +663,16 @@ static int pick_stages(int a_parts, int a_box_rows, int extra) {
 }
 
 // Stages of the GEMM ring that fit beside the control block (every operand row an MMA reads is
-// loaded, so no readable padding is needed behind the ring).
-int stream_gemm_stages(int ksb, int n_act) {
-  const int stage = ksb * n_act * 128 + ksb * kGemmNT * 128;
+// loaded or zero-filled, so no readable padding is needed behind the ring).
+int stream_gemm_stages(int ksb, int a_box_rows) {
+  const int stage = ksb * a_box_rows * 128 + ksb * kGemmNT * 128;
   const int s = (227 * 1024 - 2048) / stage;
   return s > kMaxStages ? kMaxStages : s;
 }
 
 template <int KSB, int STAGES>
 static cudaError_t launch_gemm_t(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
-  const size_t stage = (size_t)KSB * p.n_act * 128 + (size_t)KSB * kGemmNT * 128;
+  const size_t stage = (size_t)KSB * p.a_box_rows * 128 + (size_t)KSB * kGemmNT * 128;
   const size_t smem = 1024 + 1024 + STAGES * stage;
   auto kern = k_stream_gemm<KSB, STAGES>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -630,7 +684,7 @@ static cudaError_t launch_gemm_t(const StreamGemmParams& p, const CUtensorMap* m
 // p.ksb k-blocks per box.
 template <int KSB>
 static cudaError_t launch_stream_gemm_k(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
-  const int st = stream_gemm_stages(KSB, p.n_act);
+  const int st = stream_gemm_stages(KSB, p.a_box_rows);
   if (st >= 8) return launch_gemm_t<KSB, 8>(p, maps, grid, s);
   if (st >= 6) return launch_gemm_t<KSB, 6>(p, maps, grid, s);
   if (st >= 5) return launch_gemm_t<KSB, 5>(p, maps, grid, s);
@@ -639,8 +693,8 @@ static cudaError_t launch_stream_gemm_k(const StreamGemmParams& p, const CUtenso
   return cudaErrorInvalidConfiguration;
 }
 cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s) {
-  if (!p.out || !p.err || p.n_act != p.a_parts * p.a_box_rows || p.n_act % 16 || p.n_act < 16 || p.n_act > 256 ||
-      (p.a_parts == 2 && p.ksb != 1) || p.lo_col % 8 || p.lo_col * 2 > p.n_act)
+  if (!p.out || !p.err || !p.rows_dev || p.a_box_rows % 16 || p.a_box_rows < 16 || p.a_box_rows > 256 ||
+      (p.row_tiles > 1 && p.a_box_rows != 256))
     return cudaErrorInvalidValue;
   if (p.ksb == 2) return launch_stream_gemm_k<2>(p, maps, grid, s);
   if (p.ksb == 1) return launch_stream_gemm_k<1>(p, maps, grid, s);

@@ -51,22 +51,26 @@ cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counte
 // The unit space is (row tile, group, weight tile, k-step); CTA c of G owns units
 // [floor(cU/G), floor((c+1)U/G)).  Every maximal run of units inside one tile and one CTA is one
 // accumulator.  Operands are swapped with respect to the result's orientation: the 128 weight rows
-// of a tile are the MMA's M, the activation rows - hi parts and lo parts side by side - its N, so
-// that one MMA covers both parts whatever the number of rows, and a thread of the epilogue owns one
-// output feature: it adds hi and lo columns in registers and reduces the sums into the fp32
-// result matrix out[group][Rt][J] (lanes = consecutive features = consecutive addresses).
+// of a tile are the MMA's M, the activation rows its N, and a thread of the epilogue owns one
+// output feature.
+//
+// The activation operand holds the hi part and the lo part of PACKED row r in rows 2r and 2r + 1
+// (bf16 [2 * Rt, K]); only the first *rows_dev packed rows carry data, a count that only the device
+// knows.  One TMA box of a_box_rows (= 2 * min(Rt, 128)) operand rows is loaded per stage.  With
+// a single row tile the box starts at the NEGATIVE row 2 * P8 - a_box_rows (P8 = live rows rounded
+// up to 8): the rows before row 0 are filled with zeros without touching memory, the live rows
+// land at the end of the box, and the MMA's N is 2 * P8 - so the bytes an SM takes in per weight
+// tile follow the number of rows that exist, not the capacity of the pass.  The epilogue adds the
+// hi and lo columns of a row in registers and reduces the sums into the fp32 result matrix
+// out[group][Rt][J] (lanes = consecutive features = consecutive addresses).
 struct StreamGemmParams {
-  int row_tiles;         // 128-row tiles of the activations (outermost dimension of the unit space)
+  int row_tiles;         // 128-row tiles of the packed activation rows (outermost dimension of the unit space)
   int groups, tiles_per_group, ksteps;
   int ksb;               // 64-column k-blocks per stage and TMA box: 2 when the stages stay small, else 1
-  int a_box_rows;        // rows per TMA box of activations (multiple of 8)
-  int a_parts;           // boxes per stage: 1 (hi and lo rows are one contiguous box), or 2 (Rt > 128)
-  int a_part_row;        // first global row of part 1 (= Rt)
-  int n_act;             // the MMA's N: a_parts * a_box_rows, multiple of 16, <= 256
-  int lo_col;            // accumulator column of the lo part of row 0
+  int a_box_rows;        // operand rows per TMA box (multiple of 16, <= 256): the MMA's largest N
   float* out;            // [groups][Rt][J] fp32, zero before the first add
   int J, Rt;
-  int valid_rows;        // rows of the pass (results of rows beyond them are dropped)
+  const int* rows_dev;   // device word: packed rows that carry data (<= Rt)
   int* err;
 };
 
@@ -114,7 +118,7 @@ cudaError_t launch_pair_gemm(const PairGemmParams& p, const void* act_hl, const 
                              cudaStream_t s);
 
 bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows);
-int stream_gemm_stages(int ksb, int n_act);
+int stream_gemm_stages(int ksb, int a_box_rows);
 cudaError_t launch_stream_gemm(const StreamGemmParams& p, const CUtensorMap* maps, int grid, cudaStream_t s);
 cudaError_t launch_stream_logits(const StreamLogitsParams& p, const LogitMaps* maps, int grid, bool merge,
                                  Prof* prof, cudaStream_t s);

@@ -638,6 +638,14 @@ def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: i
     am = torch.zeros(N, dtype=torch.int32, device=dev)
     mx = torch.zeros(N, dtype=torch.float32, device=dev)
     lse_host = torch.zeros(N, dtype=torch.float32).pin_memory()
+    half_scratch = None
+    if args.prompt_encoder == "fp16":
+        # memory for fp16 copies of one encoder's weights: prompt-sized passes then take one
+        # tensor-core pass per k-step (activations rounded once to fp16) instead of two
+        nbytes = zb.encoder_half_bytes(cfg)
+        half_scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
+        half_scratch = half_scratch[(-half_scratch.data_ptr()) % 256:][:nbytes]
+        zb.z2z_set_encoder_half_scratch(cb, half_scratch)
 
     def step(tok_dev, hid_dev):
         zb.z2z_codebook_init(cb)
@@ -697,6 +705,7 @@ def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: i
         enc_rows += int(ln.numpy()[:int(n_fin[b])].sum())
     enc_flops = 2.0 * enc_rows * w.enc_layers * 2.0 * (4 * w.d * w.d + 2 * w.d * w.dff)
     enc_tfs = enc_flops * Kc / max(cls_ms["encoder_gemm"], 1e-9) / 1e9
+    passes = 1.0 if half_scratch is not None else 2.0       # tensor-core passes per k-step
     prompt_tokens = w.B * w.T * world
     bad = int(sum(1 for x in st.tolist() if x & (zb.ST_BAD_TOKEN | zb.ST_TABLE_FULL | zb.ST_WAIT_TIMEOUT)))
     es = 2
@@ -708,6 +717,7 @@ def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: i
         "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "prompt_tokens": w.T, "M": w.M, "cap": w.cap,
                    "compressed_positions": N, "hypertokens": int(n_fin.sum()), "replicas": world,
+                   "prompt_encoder": args.prompt_encoder,
                    "l2": "W_U, the caches and the hidden rows exceed the 126 MB L2"},
         "status_errors": bad,
         "per_class_ms_per_step": {k: v / Kc for k, v in cls_ms.items()},
@@ -721,13 +731,15 @@ def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: i
                      "flops_per_launch": flops * Kc / n_logit, "us_per_launch": cls_ms["logits"] / n_logit * 1e3,
                      "frac_of_burst_peak": tfs / pk["bf16_tflops"], "frac_of_nominal_2250": tfs / 2250.0,
                      "encoder_gemm": {"kernel": "k_pair_gemm", "rows": enc_rows,
-                                      "algorithmic_tflops": enc_tfs, "executed_tflops": 2.0 * enc_tfs,
+                                      "operands": "one fp16 activation operand, fp16 weight copies" if half_scratch is not None
+                                                  else "bf16 hi + lo activation parts, bf16 weights",
+                                      "algorithmic_tflops": enc_tfs, "executed_tflops": passes * enc_tfs,
                                       "ms_per_step": cls_ms["encoder_gemm"] / Kc,
-                                      "frac_executed_of_sustained_peak": 2.0 * enc_tfs / pk["bf16_tflops_sustained"],
-                                      "note": "activations enter as bf16 hi + lo parts: two MMAs per k-step, so the "
-                                              "tensor pipe executes twice the algorithmic flop"}},
+                                      "frac_executed_of_sustained_peak": passes * enc_tfs / pk["bf16_tflops_sustained"],
+                                      "note": "the two-part form issues two MMAs per k-step, so the tensor pipe "
+                                              "executes twice the algorithmic flop; the fp16 form issues one"}},
     }
-    del cb, E_h, U_h, hidden, hid_host, lse, am, mx
+    del cb, E_h, U_h, hidden, hid_host, lse, am, mx, half_scratch
     return line
 
 
@@ -875,6 +887,9 @@ def main(argv=None):
                     help="prompt-scoring workloads: use this many sequences instead of the workload's B")
     ap.add_argument("--prompt-steps", type=int, default=2,
                     help="timed steps of a prompt-scoring workload (one step is a whole prompt batch)")
+    ap.add_argument("--prompt-encoder", default="fp16", choices=["fp16", "two_part"],
+                    help="prompt-scoring workloads: hyper-encoder GEMM operands (fp16: one tensor-core pass per "
+                         "k-step on fp16 weight copies; two_part: bf16 hi + lo activation parts, two passes)")
     ap.add_argument("--stub", action="store_true", help="launcher self-test: ranks report fixed numbers, no GPU work")
     args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3)

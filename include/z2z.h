@@ -51,7 +51,8 @@ enum {
   Z2Z_ST_BAD_TOKEN = 2,      /* a code named a hypertoken that does not exist; state unchanged */
   Z2Z_ST_TABLE_FULL = 4,     /* hash probe ran through the whole table (cannot happen at load <= 1/2) */
   Z2Z_ST_WAIT_TIMEOUT = 8,   /* a bounded wait inside a kernel gave up                          */
-  Z2Z_ST_OUTPUT_TRUNCATED = 16 /* z2z_lzw_decode: the base tokens did not fit in T_out_max       */
+  Z2Z_ST_OUTPUT_TRUNCATED = 16, /* z2z_lzw_decode: the base tokens did not fit in T_out_max      */
+  Z2Z_ST_HALF_RANGE = 32     /* z2z_set_encoder_half_scratch: an encoder weight lies outside fp16's range */
 };
 
 enum { Z2Z_DTYPE_FP32 = 0, Z2Z_DTYPE_BF16 = 1 };
@@ -251,6 +252,22 @@ int32_t z2z_codebook_read(z2z_codebook* cb, int32_t b, int32_t* h_cons, int32_t*
  * column strips per row tile when 1 <= s <= 8 (s = 0: chosen by shape).  All produce results
  * within the stated tolerance.                                                                 */
 int32_t z2z_set_tensor_cores(z2z_codebook* cb, int32_t enable);
+
+/* Faster hyper-encoder for whole prompts (Section 2.2 applied to every entry of a prompt, Section
+ * 2.3 steps 3-4; the number format is this library's choice, the paper fixes none).  By default
+ * the tensor-core passes keep activations as two bf16 parts (about 16 mantissa bits), two
+ * tensor-core instructions per k-step.  When the caller lends device memory for fp16 copies of one
+ * encoder's linear-layer weights, z2z_hyper_embed calls that span at least four prompt-sized passes
+ * (bf16 sessions, passes of >= 1024 rows) remake the copies at the start of the call - a bf16
+ * value inside fp16's range converts exactly - and round each activation once to fp16 (11 mantissa
+ * bits): one instruction per k-step, half the tensor-core work.  Measured against the fp64
+ * definition with randomly drawn gains and biases, the largest error of a hyper-embedding grows
+ * from 9e-5 to 7.3e-3 at d = 4096 (tolerance 2e-2); sessions that need the wider margin leave the
+ * scratch unset.  Decode steps are not affected.
+ *   d_scratch: 256-byte aligned, bytes >= 2 * enc_layers * (4 d^2 + 2 d enc_dff) * 2, valid until
+ *   replaced; NULL or 0 bytes returns to the two-part form.  A weight beyond fp16's range
+ *   (|w| > 65504) cannot be copied exactly: Z2Z_ST_HALF_RANGE is then reported by z2z_status.   */
+int32_t z2z_set_encoder_half_scratch(z2z_codebook* cb, void* d_scratch, size_t bytes);
 
 /* Launch accounting and per-kernel-class timing (no counterpart in the paper; measurement aid).
  * The library always counts the kernels it launches, per class:

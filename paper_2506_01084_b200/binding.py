@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libz2z.so")
 
 OK = 0
-ST_CAP_FROZEN, ST_BAD_TOKEN, ST_TABLE_FULL, ST_WAIT_TIMEOUT, ST_OUTPUT_TRUNCATED = 1, 2, 4, 8, 16
+ST_CAP_FROZEN, ST_BAD_TOKEN, ST_TABLE_FULL, ST_WAIT_TIMEOUT, ST_OUTPUT_TRUNCATED, ST_HALF_RANGE = 1, 2, 4, 8, 16, 32
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 SELECT_ARGMAX, SELECT_GUMBEL = 0, 1
 CODE_NONE, CODE_SELECTED = -1, -2
@@ -27,7 +27,8 @@ EXPORTS = ["z2z_workspace_bytes", "z2z_codebook_init", "z2z_lzw_encode", "z2z_lz
            "z2z_hyper_embed", "z2z_dynamic_logits", "z2z_decode_step", "z2z_status",
            "z2z_codebook_read", "z2z_codebook_destroy", "z2z_last_error", "z2z_profile",
            "z2z_profile_read", "z2z_set_tensor_cores", "z2z_logits_static_scratch",
-           "z2z_lzw_decode", "z2z_embed_lookup", "z2z_upload_rows", "z2z_sample_filtered"]
+           "z2z_lzw_decode", "z2z_embed_lookup", "z2z_upload_rows", "z2z_sample_filtered",
+           "z2z_set_encoder_half_scratch"]
 
 
 class Config(C.Structure):
@@ -255,6 +256,20 @@ def z2z_set_tensor_cores(cb: Codebook, enable):
     2 + 16 * s: the CTA-pair logits kernel for every z2z_dynamic_logits call, with s column strips
     (0: chosen by shape)."""
     _check(lib().z2z_set_tensor_cores(cb.handle, C.c_int32(int(enable))))
+
+
+def encoder_half_bytes(cfg: Config) -> int:
+    """Bytes of scratch z2z_set_encoder_half_scratch needs for this configuration."""
+    return 2 * cfg.enc_layers * (4 * cfg.d * cfg.d + 2 * cfg.d * cfg.enc_dff)
+
+
+def z2z_set_encoder_half_scratch(cb: Codebook, scratch: Optional[torch.Tensor]):
+    """Lend device memory (a uint8 tensor, 256-byte aligned) for fp16 copies of one encoder's
+    linear-layer weights: long prompt-sized z2z_hyper_embed calls then run one tensor-core pass per
+    k-step.  None returns to the two-part form.  The handle keeps a reference to the tensor."""
+    cb._half_scratch = scratch
+    nbytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
+    _check(lib().z2z_set_encoder_half_scratch(cb.handle, _ptr(scratch), C.c_size_t(nbytes)))
 
 
 def z2z_logits_static_scratch(hidden: torch.Tensor, row_seq: Optional[torch.Tensor],

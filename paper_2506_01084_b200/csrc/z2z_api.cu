@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
@@ -19,6 +20,9 @@ struct z2z_codebook {
   int prefill_strips;        // > 0: fixed number of column strips in the prompt-scoring kernel
   int* h_frozen;             // pinned host word the decode-update kernel writes once every codebook is full
   int epoch;                 // session number: incremented by every z2z_codebook_init
+  void* half_scratch;        // caller's memory for fp16 copies of one encoder's linear-layer weights, or NULL
+  size_t half_bytes;
+  std::vector<const void*> half_ptrs;   // device addresses of the copies, ABI tensor order
   z2z::Prof prof;
 };
 
@@ -296,6 +300,17 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
   long long bound = (long long)cb->cfg.B * cb->cfg.cap;
   if (max_entries > 0 && max_entries < bound) bound = max_entries;
   const int n_chunks = (int)((bound + el.chunk - 1) / el.chunk);
+  // Single-pass fp16 form of the prompt-sized passes: when the caller has lent memory for the
+  // weight copies and the call is long enough (several passes) to repay making them.
+  a.w_half = nullptr;
+  if (tc && cb->half_scratch && cb->cfg.enc_layers > 0 && n_chunks >= 4 &&
+      z2z::encoder_pass_is_prompt_sized(a.entries, el.chunk, cb->cfg.M) &&
+      cb->half_bytes >= z2z::encoder_half_bytes(cb->cfg.d, cb->dff, cb->cfg.enc_layers)) {
+    cb->half_ptrs.assign((size_t)enc->n_tensors, nullptr);
+    Z2Z_CUDA(z2z::convert_encoder_weights_to_half(enc->tensors, cb->cfg.d, cb->dff, cb->cfg.enc_layers, cb->half_scratch,
+                                                  cb->half_ptrs.data(), a.err, &cb->prof, s), "hyper_embed (fp16 weight copies)");
+    a.w_half = cb->half_ptrs.data();
+  }
   {
     z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
     Z2Z_CUDA(z2z::launch_entry_offsets(cb->view, which, d_first, d_count, el, s), "hyper_embed");
@@ -449,7 +464,8 @@ int32_t z2z_status(z2z_codebook* cb, int32_t* h_status, int32_t* h_n, z2z_stream
   Z2Z_CUDA(cudaMemcpyAsync(&kernel_err, cb->ws + cb->plan.off_words, 4, cudaMemcpyDeviceToHost, s), "status");
   Z2Z_CUDA(cudaStreamSynchronize(s), "status");
   if (kernel_err && h_status)
-    for (int b = 0; b < cb->cfg.B; ++b) h_status[b] |= Z2Z_ST_WAIT_TIMEOUT;
+    for (int b = 0; b < cb->cfg.B; ++b)
+      h_status[b] |= ((kernel_err & 1) ? Z2Z_ST_WAIT_TIMEOUT : 0) | ((kernel_err & 2) ? Z2Z_ST_HALF_RANGE : 0);
   return Z2Z_OK;
 }
 
@@ -485,6 +501,14 @@ int32_t z2z_set_tensor_cores(z2z_codebook* cb, int32_t enable) {
   cb->use_tensor_cores = enable == 0 ? 0 : (enable % 16 == 2 ? 2 : 1);
   cb->prefill_strips = enable / 16;
   if (cb->prefill_strips > z2z::kPrefillMaxStrips) cb->prefill_strips = z2z::kPrefillMaxStrips;
+  return Z2Z_OK;
+}
+
+int32_t z2z_set_encoder_half_scratch(z2z_codebook* cb, void* d_scratch, size_t bytes) {
+  if (!cb) return fail(Z2Z_ERR_INVALID_ARG, "cb is NULL");
+  if (d_scratch && (reinterpret_cast<uintptr_t>(d_scratch) & 255) != 0) return fail(Z2Z_ERR_INVALID_ARG, "scratch must be 256-byte aligned");
+  cb->half_scratch = bytes > 0 ? d_scratch : nullptr;
+  cb->half_bytes = d_scratch ? bytes : 0;
   return Z2Z_OK;
 }
 

@@ -8,6 +8,12 @@
 // and lo*w are exact in fp32, so A.W^T = hi.W^T + lo.W^T with fp32 accumulation.  Rounding the
 // activations to a single bf16 would leave the hyper-embeddings outside the 2e-2 tolerance.
 //
+// Prompt-sized passes may instead round every activation ONCE to fp16 and multiply by fp16 copies
+// of the weights (exact for bf16 values within fp16's range), when the caller has lent memory
+// for the copies: one MMA per k-step instead of two.  The rounding error (2^-11 relative per
+// operand element) stays inside the tolerance with a margin of about 3 at d = 4096; the two-part
+// form keeps a margin of about 200 and remains the default.
+//
 // Rows are PACKED in both kinds of pass: entry e owns the rows row_off[e] .. row_off[e] + len[e],
 // there are no padding rows, and only the device knows how many rows a pass has (the word behind
 // the last entry slot of row_off).
@@ -30,6 +36,8 @@
 // what a kernel needs about an entry (its length, the base token of a row) is one load from the
 // work list, and every data load is issued before the first value is used - whether a row is valid
 // only decides what is stored.
+#include <cuda_fp16.h>
+
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
 #include "z2z_sm100.cuh"
@@ -71,6 +79,14 @@ __device__ __forceinline__ void split_store4(bf16* hi, bf16* lo, float4 x) {
   *reinterpret_cast<uint2*>(hi) = H;
   *reinterpret_cast<uint2*>(lo) = L;
 }
+// 4 values rounded once to fp16; one 8-byte store.  `dst` points into an fp16 matrix that shares
+// the bf16 operand buffer (same element size).
+__device__ __forceinline__ void half_store4(bf16* dst, float4 x) {
+  uint2 H;
+  H.x = (uint32_t)__half_as_ushort(__float2half_rn(x.x)) | ((uint32_t)__half_as_ushort(__float2half_rn(x.y)) << 16);
+  H.y = (uint32_t)__half_as_ushort(__float2half_rn(x.z)) | ((uint32_t)__half_as_ushort(__float2half_rn(x.w)) << 16);
+  *reinterpret_cast<uint2*>(dst) = H;
+}
 // Base tokens of work-list entry e (0 for an unused slot): one load, so that the kernels below can
 // issue it together with their data loads instead of ahead of them.
 __device__ __forceinline__ int entry_len_tc(const CbView& cb, const EntryList& el, int e) {
@@ -98,7 +114,7 @@ __device__ __forceinline__ float block_sum(float v, float* sm) {
 // written as hi/lo bf16.  eps 1e-5, biased variance, two-pass.
 // gw / gb: gamma and beta of the thread's columns, packed 4 bf16 per uint2 and loaded by the caller
 // together with the row, so that no load waits behind the reductions.
-template <int NV>
+template <int NV, bool HALF = false>
 __device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[NV], int nvec, const uint2 (&gw)[NV],
                                                      const uint2 (&gb)[NV], bf16* hi, bf16* lo, int d, float* sm) {
   float s = 0.f;
@@ -124,7 +140,8 @@ __device__ __forceinline__ void layernorm_split_regs(const float4 (&x)[NV], int 
       y.y = (x[v].y - mean) * rstd * gg.y + bb.y;
       y.z = (x[v].z - mean) * rstd * gg.z + bb.z;
       y.w = (x[v].w - mean) * rstd * gg.w + bb.w;
-      split_store4(hi + idx * 4, lo + idx * 4, y);
+      if (HALF) half_store4(hi + idx * 4, y);
+      else split_store4(hi + idx * 4, lo + idx * 4, y);
     }
   }
 }
@@ -425,7 +442,7 @@ __global__ void __launch_bounds__(1024) k_tc_row_map(CbView cb, EntryList el, in
 }
 
 // X = table[y] + pos for every packed row, then LN1 of layer 0 -> hi/lo.  grid (row capacity).
-template <int NV>
+template <int NV, bool HALF>
 __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln_packed(CbView cb, EntryList el, const int* total,
                                                                      const bf16* table, const bf16* pos, const bf16* ln_w,
                                                                      const bf16* ln_b, float* X, bf16* Ahl, int d, int Rt,
@@ -453,7 +470,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_gather_ln_packed(CbView cb, 
       *reinterpret_cast<float4*>(x + idx * 4) = xv[v];
     }
   }
-  if (has_ln) layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
+  if (has_ln) layernorm_split_regs<NV, HALF>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
 // Mean-pool on packed rows: cache row = mean of the entry's rows of X.  grid (entries,
@@ -484,7 +501,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_pool_packed(CbView cb, Entry
 
 // LayerNorm of the packed rows of X -> hi/lo (the GEMM epilogue has already added bias and
 // residual into X).  grid (row capacity), one encoder.
-template <int NV>
+template <int NV, bool HALF>
 __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, const float* X, const bf16* ln_w,
                                                             const bf16* ln_b, bf16* Ahl, int d, int Rt) {
   __shared__ float sm[32];
@@ -504,7 +521,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, co
     }
   }
   bf16* hi = Ahl + (size_t)r * d;
-  layernorm_split_regs<NV>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
+  layernorm_split_regs<NV, HALF>(xv, nvec, gw, gb, hi, hi + (size_t)Rt * d, d, sm);
 }
 
 // Bidirectional attention inside one entry from fp32 q, k, v of its packed rows [rows, 3d] (bias
@@ -512,7 +529,7 @@ __global__ void __launch_bounds__(kRowThreads) k_tc_ln_rows(const int* total, co
 // are loaded into registers at once (a lane holds four columns of every row), the L x L scores are
 // warp reductions, no shared memory and no block barrier.  MM = compile-time bound on the merge
 // size; dh <= 128 (larger heads take the kernel below).  grid = ceil(entries * heads / 8), block 256.
-template <int MM>
+template <int MM, bool HALF>
 __global__ void __launch_bounds__(256) k_tc_attention_rows_warp(CbView cb, EntryList el, const float* QKV, bf16* Ohl,
                                                                 int E, int d, int heads, int Rt) {
   const int lane = threadIdx.x & 31;
@@ -562,13 +579,17 @@ __global__ void __launch_bounds__(256) k_tc_attention_rows_warp(CbView cb, Entry
       const float wj = s[j] * inv;
       o.x = fmaf(wj, v[j].x, o.x); o.y = fmaf(wj, v[j].y, o.y); o.z = fmaf(wj, v[j].z, o.z); o.w = fmaf(wj, v[j].w, o.w);
     }
-    if (on) split_store4(hi + (size_t)i * d, lo + (size_t)i * d, o);
+    if (on) {
+      if (HALF) half_store4(hi + (size_t)i * d, o);
+      else split_store4(hi + (size_t)i * d, lo + (size_t)i * d, o);
+    }
   }
 }
 
 // The same for heads wider than 128 columns or merge sizes above 4: staged in shared memory.
 // grid (entries, heads), block (32, M), dynamic smem M * 3 * dh floats.
-__global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, bf16* Ohl, int d, int heads, int Rt) {
+__global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, bf16* Ohl, int d, int heads, int Rt,
+                                    int half) {
   extern __shared__ float s_qkv[];
   const int e = blockIdx.x, h = blockIdx.y, i = threadIdx.y, lane = threadIdx.x;
   const int L = entry_len_tc(cb, el, e);
@@ -611,10 +632,34 @@ __global__ void k_tc_attention_rows(CbView cb, EntryList el, const float* QKV, b
 #pragma unroll
     for (int j = 0; j < kMaxM; ++j)
       if (j < L) v = fmaf(s[j] * inv, s_qkv[(j * 3 + 2) * dh + c], v);
-    const bf16 hh = __float2bfloat16_rn(v);
-    hi[c] = hh;
-    lo[c] = __float2bfloat16_rn(v - __bfloat162float(hh));
+    if (half) {
+      reinterpret_cast<__half*>(hi)[c] = __float2half_rn(v);
+    } else {
+      const bf16 hh = __float2bfloat16_rn(v);
+      hi[c] = hh;
+      lo[c] = __float2bfloat16_rn(v - __bfloat162float(hh));
+    }
   }
+}
+
+// fp16 copy of a bf16 weight tensor (n a multiple of 8).  A bf16 value inside fp16's range converts
+// exactly; a value beyond it cannot be represented and raises bit 1 of the error word.
+__global__ void __launch_bounds__(256) k_tc_weights_to_half(const bf16* __restrict__ src, __half* __restrict__ dst,
+                                                            size_t n8, int* err) {
+  bool over = false;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+    const uint4 u = reinterpret_cast<const uint4*>(src)[i];
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float a = bf_lo(w[k]), b = bf_hi(w[k]);
+      over |= fabsf(a) > 65504.f || fabsf(b) > 65504.f;
+      o[k] = (uint32_t)__half_as_ushort(__float2half_rn(a)) | ((uint32_t)__half_as_ushort(__float2half_rn(b)) << 16);
+    }
+    reinterpret_cast<uint4*>(dst)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  if (over) atomicOr(err, 2);
 }
 
 int sm_count() {
@@ -642,22 +687,25 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
                                          Prof* prof, cudaStream_t s) {
   const int d = a.d, dff = a.dff, M = cb.M;
   const int R = E * M, Rt = (R + 7) / 8 * 8;
+  const bool half = a.w_half != nullptr;               // fp16 copies of the linear-layer weights exist
   auto Wp = [&](int i) { return reinterpret_cast<const bf16*>(a.w[i]); };
   const int* total = el.row_off + E;                   // packed rows of this pass (device word)
   const bool narrow = d <= 4 * kRowThreads * kNarrowVec4;      // a row fits four float4 per thread: fewer registers, more CTAs per SM
-  auto lnk = narrow ? k_tc_ln_rows<kNarrowVec4> : k_tc_ln_rows<kMaxVec4>;
+  auto lnk = half ? (narrow ? k_tc_ln_rows<kNarrowVec4, true> : k_tc_ln_rows<kMaxVec4, true>)
+                  : (narrow ? k_tc_ln_rows<kNarrowVec4, false> : k_tc_ln_rows<kMaxVec4, false>);
   PairGemmParams g{};
   g.cb = cb; g.el = el; g.R = R; g.Rt = Rt; g.live_rows = total; g.err = a.err;
   auto gemm = [&](const bf16* act, int K, int widx, int J, int epi, float* out, bf16* out_hl) -> cudaError_t {
     PairGemmParams p = g;
     p.J = J; p.bias = a.w[widx + 1]; p.out = out; p.out_hl = out_hl;
     ProfScope ps(prof, kProfEncGemm, 1, s);
-    return launch_pair_gemm(p, act, a.w[widx], K, epi, s);
+    return launch_pair_gemm(p, act, half ? a.w_half[widx] : a.w[widx], K, epi, half, s);
   };
   {
     ProfScope ps(prof, kProfEncOther, 2, s);
     k_tc_row_map<<<1, 1024, 0, s>>>(cb, el, E);
-    auto gk = narrow ? k_tc_gather_ln_packed<kNarrowVec4> : k_tc_gather_ln_packed<kMaxVec4>;
+    auto gk = half ? (narrow ? k_tc_gather_ln_packed<kNarrowVec4, true> : k_tc_gather_ln_packed<kMaxVec4, true>)
+                   : (narrow ? k_tc_gather_ln_packed<kNarrowVec4, false> : k_tc_gather_ln_packed<kMaxVec4, false>);
     gk<<<R, kRowThreads, 0, s>>>(cb, el, total, reinterpret_cast<const bf16*>(a.table), Wp(0), a.layers ? Wp(1) : Wp(0),
                                  a.layers ? Wp(2) : Wp(0), a.X, a.Ahl, d, Rt, a.layers > 0 ? 1 : 0);
   }
@@ -668,11 +716,13 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
     if ((e = gemm(a.Ahl, d, o + 2, 3 * d, kEpiStore, a.QKV, nullptr)) != cudaSuccess) return e;
     {
       ProfScope ps(prof, kProfEncOther, 1, s);
-      if (dh <= 128 && M <= 4)
-        k_tc_attention_rows_warp<4><<<(E * a.heads + 7) / 8, 256, 0, s>>>(cb, el, a.QKV, a.Ahl, E, d, a.heads, Rt);
-      else
+      if (dh <= 128 && M <= 4) {
+        auto ak = half ? k_tc_attention_rows_warp<4, true> : k_tc_attention_rows_warp<4, false>;
+        ak<<<(E * a.heads + 7) / 8, 256, 0, s>>>(cb, el, a.QKV, a.Ahl, E, d, a.heads, Rt);
+      } else {
         k_tc_attention_rows<<<dim3(E, a.heads), dim3(32, M), (size_t)M * 3 * dh * 4, s>>>(cb, el, a.QKV, a.Ahl, d,
-                                                                                           a.heads, Rt);
+                                                                                           a.heads, Rt, half ? 1 : 0);
+      }
     }
     if ((e = gemm(a.Ahl, d, o + 4, d, kEpiResid, a.X, nullptr)) != cudaSuccess) return e;
     if (dff > 0) {                                     // dff == 0: attention-only layer
@@ -691,6 +741,40 @@ static cudaError_t run_encoder_pass_pair(const CbView& cb, const EncoderArgs& a,
   ProfScope ps(prof, kProfEncOther, 1, s);
   k_tc_pool_packed<<<dim3(E, (d / 4 + kRowThreads - 1) / kRowThreads), kRowThreads, 0, s>>>(cb, el, a.X, a.cache,
                                                                                         a.cache_f32, d);
+  return cudaGetLastError();
+}
+
+// Bytes of fp16 copies of one encoder's linear-layer weights.
+size_t encoder_half_bytes(int d, int dff, int layers) {
+  return (size_t)layers * ((size_t)4 * d * d + (size_t)2 * d * dff) * 2;
+}
+
+// Whether a pass of `entries` work-list slots is a prompt-sized one (CTA-pair GEMMs).
+bool encoder_pass_is_prompt_sized(int entries, int chunk, int M) {
+  const int E = entries < chunk ? entries : chunk;
+  return E * M >= kPairPassMinRows;
+}
+
+// Makes fp16 copies of the linear-layer weights of one encoder in `scratch` and fills
+// half_ptrs[i] (host array, ABI tensor order) with their device addresses (nullptr elsewhere).
+cudaError_t convert_encoder_weights_to_half(const void* const* w, int d, int dff, int layers, void* scratch,
+                                            const void** half_ptrs, int* err_word, Prof* prof, cudaStream_t s) {
+  char* dst = reinterpret_cast<char*>(scratch);
+  for (int i = 0; i < 1 + 12 * layers; ++i) half_ptrs[i] = nullptr;
+  const int n_sm = sm_count();
+  for (int l = 0; l < layers; ++l) {
+    const int o = 1 + 12 * l;
+    const int idx[4] = {o + 2, o + 4, o + 8, o + 10};
+    const size_t elems[4] = {(size_t)3 * d * d, (size_t)d * d, (size_t)dff * d, (size_t)d * dff};
+    for (int k = 0; k < 4; ++k) {
+      if (elems[k] == 0) continue;
+      ProfScope ps(prof, kProfEncOther, 1, s);
+      k_tc_weights_to_half<<<n_sm * 8, 256, 0, s>>>(reinterpret_cast<const bf16*>(w[idx[k]]),
+                                                    reinterpret_cast<__half*>(dst), elems[k] / 8, err_word);
+      half_ptrs[idx[k]] = dst;
+      dst += elems[k] * 2;
+    }
+  }
   return cudaGetLastError();
 }
 

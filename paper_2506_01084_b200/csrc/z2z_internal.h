@@ -59,6 +59,7 @@ struct EncoderArgs {
   int dtype;
   const void* table;            // [V, d]
   const void* const* w;         // host array of device pointers, ABI order
+  const void* const* w_half;    // or NULL: fp16 copies of the linear-layer weights, same order (prompt-sized passes)
   void* cache;                  // [B, cap, d] dtype
   float* cache_f32;             // optional
   float *X, *A, *QKV, *H;       // fp32 scratch, rows = chunk * M
@@ -69,6 +70,10 @@ struct EncoderArgs {
   int* err;                     // device error word of the tensor-core kernels
 };
 bool encoder_tc_supported(int d, int dff, int dtype, int heads, int M);
+size_t encoder_half_bytes(int d, int dff, int layers);
+bool encoder_pass_is_prompt_sized(int entries, int chunk, int M);
+cudaError_t convert_encoder_weights_to_half(const void* const* w, int d, int dff, int layers, void* scratch,
+                                            const void** half_ptrs, int* err_word, Prof* prof, cudaStream_t s);
 bool logits_tc_supported(int d, int dtype);
 // Two encoders (embedding side, unembedding side) run through the same launches.
 // rows_mapped: the packed-row map of the work list (row_off, row_src, row_tok) is already there.

@@ -15,8 +15,15 @@
 // Rows that are padding of their entry (or lie beyond the pass) are not written (kEpiGelu writes
 // zeros there, because the next GEMM reads them).
 //
+// HALF variant: the activations are ONE fp16 matrix (rounded once, 2^-11 relative) and the weights
+// an fp16 copy of the bf16 tensor (exact within fp16's range), so a k-step is one MMA instead of
+// two and a stage holds 32 KB instead of 48: half the tensor-core work of the layer.  kEpiGelu
+// then writes one fp16 matrix.
+//
 // Roles per CTA: warp 0 lane 0 TMA producer, warp 1 lane 0 MMA issuer (leader CTA only), warps
 // 2-5 epilogue (thread = row).  Every mbarrier wait is bounded.
+#include <cuda_fp16.h>
+
 #include "z2z_common.cuh"
 #include "z2z_internal.h"
 #include "z2z_sm100.cuh"
@@ -28,18 +35,24 @@ using namespace sm100;
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kPgStages = 4;              // 48 KB per stage and CTA: A hi, A lo, W, each 128 x 64 bf16
-constexpr uint32_t kPgStageBytes = 49152;
+constexpr int kPgMaxStages = 6;
+// Two-part operands: 4 stages of 48 KB per CTA (A hi, A lo, W, each 128 x 64 bf16); one fp16 operand:
+// 6 stages of 32 KB (A, W).
+__host__ __device__ constexpr int pg_stages(bool half) { return half ? 6 : 4; }
+__host__ __device__ constexpr uint32_t pg_stage_bytes(bool half) { return half ? 32768u : 49152u; }
 
 struct PgCtrl {
-  unsigned long long full[kPgStages], empty[kPgStages], acc_full[2], acc_empty[2];
+  unsigned long long full[kPgMaxStages], empty[kPgMaxStages], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort;
 };
 
-template <int EPI>
+template <int EPI, bool HALF>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW) {
+  constexpr int kPgStages = pg_stages(HALF);
+  constexpr uint32_t kPgStageBytes = pg_stage_bytes(HALF);
+  constexpr uint32_t kWOff = HALF ? 16384u : 32768u;        // weight tile inside a stage
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   PgCtrl* ctrl = reinterpret_cast<PgCtrl*>(sm);
@@ -93,9 +106,9 @@ k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, con
           if (!mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, &ctrl->abort)) { ok = false; break; }
           if (rank == 0) mbar_expect_tx(smem_u32(&ctrl->full[stage]), 2 * kPgStageBytes);
           const uint32_t sb = stage_base + (uint32_t)stage * kPgStageBytes;
-          tma_load_2d_pair(sb, &tmA, ks * 64, arow, full_leader[stage], pol);                 // hi rows
-          tma_load_2d_pair(sb + 16384, &tmA, ks * 64, p.Rt + arow, full_leader[stage], pol);   // lo rows
-          tma_load_2d_pair(sb + 32768, &tmW, ks * 64, wrow, full_leader[stage], pol);
+          tma_load_2d_pair(sb, &tmA, ks * 64, arow, full_leader[stage], pol);                 // hi rows (HALF: the rows)
+          if (!HALF) tma_load_2d_pair(sb + 16384, &tmA, ks * 64, p.Rt + arow, full_leader[stage], pol);   // lo rows
+          tma_load_2d_pair(sb + kWOff, &tmW, ks * 64, wrow, full_leader[stage], pol);
           if (++stage == kPgStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -103,7 +116,7 @@ k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, con
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
       // ---------------- MMA issuer (leader only) ------------------------------------------------------
-      const uint32_t idesc = idesc_bf16_f32(256, 256);
+      const uint32_t idesc = HALF ? idesc_f16_f32(256, 256) : idesc_bf16_f32(256, 256);
       int stage = 0; uint32_t phase = 0, job_i = 0;
       bool ok = true;
       for (int t = cluster_id; t < n_tiles && ok; t += n_clusters) {
@@ -117,10 +130,10 @@ k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, con
           tc_fence_after();
           const uint32_t sb = stage_base + (uint32_t)stage * kPgStageBytes;
 #pragma unroll
-          for (int part = 0; part < 2; ++part)        // hi part, then lo part, into the same accumulator
+          for (int part = 0; part < (HALF ? 1 : 2); ++part)        // hi part, then lo part, into the same accumulator
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              umma_bf16_pair(d, smem_desc_sw128(sb + part * 16384 + k * 32), smem_desc_sw128(sb + 32768 + k * 32),
+              umma_bf16_pair(d, smem_desc_sw128(sb + part * 16384 + k * 32), smem_desc_sw128(sb + kWOff + k * 32),
                              idesc, acc);
               acc = 1;
             }
@@ -179,6 +192,23 @@ k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, con
               }
               *reinterpret_cast<float4*>(dst + x) = o;
             }
+          } else if (HALF) {
+            __half* ho = reinterpret_cast<__half*>(p.out_hl) + (size_t)r * p.J + col;
+#pragma unroll
+            for (int x = 0; x < 32; x += 8) {
+              uint32_t H[4];
+#pragma unroll
+              for (int y = 0; y < 8; y += 2) {
+                float g0 = 0.f, g1 = 0.f;
+                if (valid) {
+                  const float a0 = __uint_as_float(v[x + y]) + bs[x + y], a1 = __uint_as_float(v[x + y + 1]) + bs[x + y + 1];
+                  g0 = 0.5f * a0 * (1.0f + erff(a0 * 0.70710678118654752440f));
+                  g1 = 0.5f * a1 * (1.0f + erff(a1 * 0.70710678118654752440f));
+                }
+                H[y >> 1] = (uint32_t)__half_as_ushort(__float2half_rn(g0)) | ((uint32_t)__half_as_ushort(__float2half_rn(g1)) << 16);
+              }
+              *reinterpret_cast<uint4*>(ho + x) = make_uint4(H[0], H[1], H[2], H[3]);
+            }
           } else {
             __nv_bfloat16* hi = p.out_hl + (size_t)r * p.J + col;
             __nv_bfloat16* lo = hi + (size_t)p.Rt * p.J;
@@ -220,8 +250,20 @@ k_pair_gemm(const PairGemmParams p, const __grid_constant__ CUtensorMap tmA, con
 
 }  // namespace
 
-// D = (A_hi + A_lo) W^T with the epilogue `epi`, for a pass of R rows (Rt rows per hi / lo block).
-cudaError_t launch_pair_gemm(const PairGemmParams& p0, const void* act_hl, const void* W, int K, int epi,
+template <int EPI, bool HALF>
+static cudaError_t launch_pair_gemm_t(const PairGemmParams& p, const CUtensorMap& mA, const CUtensorMap& mW, int clusters,
+                                      cudaStream_t s) {
+  const size_t smem = 1024 + 1024 + (size_t)pg_stages(HALF) * pg_stage_bytes(HALF);
+  auto kern = k_pair_gemm<EPI, HALF>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<2 * clusters, kThreads, smem, s>>>(p, mA, mW);
+  return cudaGetLastError();
+}
+
+// D = A W^T with the epilogue `epi`, for a pass of R rows.  half == false: A = A_hi + A_lo, two bf16
+// blocks of Rt rows each, W bf16.  half == true: A is one fp16 matrix of Rt rows, W an fp16 copy.
+cudaError_t launch_pair_gemm(const PairGemmParams& p0, const void* act, const void* W, int K, int epi, bool half,
                              cudaStream_t s) {
   static int n_sm = 0;
   if (!n_sm) {
@@ -235,16 +277,19 @@ cudaError_t launch_pair_gemm(const PairGemmParams& p0, const void* act_hl, const
   p.row_tiles = (p.R + 255) / 256;
   p.col_tiles = (p.J + 255) / 256;
   CUtensorMap mA, mW;
-  if (!make_tmap_bf16(&mA, act_hl, 2ll * p.Rt, K, 128)) return cudaErrorInvalidValue;
+  // (the element type of a tensor map only fixes the element size and the fill value: bf16 and fp16 alike)
+  if (!make_tmap_bf16(&mA, act, (half ? 1ll : 2ll) * p.Rt, K, 128)) return cudaErrorInvalidValue;
   if (!make_tmap_bf16(&mW, W, p.J, K, 128)) return cudaErrorInvalidValue;
   const int tiles = p.row_tiles * p.col_tiles;
   const int clusters = tiles < n_sm / 2 ? tiles : n_sm / 2;
-  const size_t smem = 1024 + 1024 + (size_t)kPgStages * kPgStageBytes;
-  auto kern = epi == kEpiStore ? k_pair_gemm<kEpiStore> : (epi == kEpiResid ? k_pair_gemm<kEpiResid> : k_pair_gemm<kEpiGelu>);
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  kern<<<2 * clusters, kThreads, smem, s>>>(p, mA, mW);
-  return cudaGetLastError();
+  if (half) {
+    if (epi == kEpiStore) return launch_pair_gemm_t<kEpiStore, true>(p, mA, mW, clusters, s);
+    if (epi == kEpiResid) return launch_pair_gemm_t<kEpiResid, true>(p, mA, mW, clusters, s);
+    return launch_pair_gemm_t<kEpiGelu, true>(p, mA, mW, clusters, s);
+  }
+  if (epi == kEpiStore) return launch_pair_gemm_t<kEpiStore, false>(p, mA, mW, clusters, s);
+  if (epi == kEpiResid) return launch_pair_gemm_t<kEpiResid, false>(p, mA, mW, clusters, s);
+  return launch_pair_gemm_t<kEpiGelu, false>(p, mA, mW, clusters, s);
 }
 
 }  // namespace z2z

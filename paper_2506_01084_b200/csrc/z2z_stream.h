@@ -110,11 +110,11 @@ struct PairGemmParams {
   int J;                 // output columns (a multiple of 128)
   const void* bias;      // [J] bf16
   float* out;            // kEpiStore / kEpiResid: fp32 [R, J]
-  __nv_bfloat16* out_hl; // kEpiGelu: bf16 [2 Rt, J], hi rows then lo rows
+  __nv_bfloat16* out_hl; // kEpiGelu: bf16 [2 Rt, J], hi rows then lo rows (single fp16 operand: fp16 [Rt, J])
   int ksteps, row_tiles, col_tiles;
   int* err;
 };
-cudaError_t launch_pair_gemm(const PairGemmParams& p, const void* act_hl, const void* W, int K, int epi,
+cudaError_t launch_pair_gemm(const PairGemmParams& p, const void* act, const void* W, int K, int epi, bool half,
                              cudaStream_t s);
 
 bool make_tmap_bf16(CUtensorMap* m, const void* base, long long rows, long long cols, int box_rows);

@@ -252,5 +252,26 @@ def test_full_size_prompt_scoring_sampled():
             worst_e = max(worst_e, err)
             assert err <= TOL, (side, b, k, err)
             assert torch.equal(cache[b, k].cpu(), E32[b, k].cpu().to(w.torch_dtype))
+        if side == "E":
+            # the same entries once more with a single fp16 operand per GEMM (weights copied to fp16,
+            # activations rounded once): same oracle rows, same tolerance
+            nbytes = zb.encoder_half_bytes(s.cfg)
+            scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device=DEV)
+            scratch = scratch[(-scratch.data_ptr()) % 256:][:nbytes]
+            zb.z2z_set_encoder_half_scratch(s.cb, scratch)
+            E32.zero_()
+            zb.z2z_hyper_embed(s.cb, zb.CACHE_EMBED, s.g_WE, s.g_encE, first, count, 8 * 1024, s.E_h, E32)
+            worst_h = 0.0
+            for b, k in picks:
+                want = _oracle_embed(s.book(b).entries[k], table, enc64, w.heads)
+                err = np.abs(E32[b, k].cpu().double().numpy() - want).max()
+                worst_h = max(worst_h, err)
+                assert err <= TOL, ("E, single fp16 operand", b, k, err)
+                assert torch.equal(cache[b, k].cpu(), E32[b, k].cpu().to(w.torch_dtype))
+            st, _ = zb.z2z_status(s.cb)
+            assert int(st.max()) & zb.ST_HALF_RANGE == 0
+            zb.z2z_set_encoder_half_scratch(s.cb, None)
+            del scratch
+            print(f"prefill_heavy: single fp16 operand, worst |hyper-embedding error| {worst_h:.2e}")
         del enc64
     print(f"prefill_heavy: {len(picks)} entries per side, worst |hyper-embedding error| {worst_e:.2e}")

@@ -604,7 +604,7 @@ ROWS_BF16 = si.Workload("rows_bf16", V=3000, d=256, dtype="bf16", B=2, T=220, M=
                          ids=lambda w: w.name)
 def test_weight_streaming_gemm_with_several_row_tiles(w):
     # passes of 480 / 675 rows: below the size of the CTA-pair GEMM and above one 128-row tile, so
-    # the hi rows and the lo rows of a row tile are two operand boxes and the last tile is ragged
+    # the packed rows span several row tiles (one 256-row operand box each) and the last is ragged
     assert 128 < w.B * w.cap * w.M < 1024
     p = Pair(w, seed=35)
     _, worst = _prefill_both(p)
@@ -624,6 +624,77 @@ def test_prompt_sized_pass_with_long_entries_and_wide_heads(w):
     _, worst = _prefill_both(p)
     assert worst <= TOL
     print(f"{w.name}: max |hyper-embedding error| = {worst:.3e}")
+
+
+def _embed_all_both_sides(p, max_entries):
+    w = p.w
+    p.E_f32.zero_(); p.U_f32.zero_()
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, max_entries, p.E_h, p.E_f32)
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_UNEMBED, p.g_WU, p.g_encU, None, None, max_entries, p.U_h, p.U_f32)
+    worst = max(p.check_cache_rows(b, 0, p.oracle.books[b].n()) for b in range(w.B))
+    return worst, p.E_f32.clone(), p.U_f32.clone()
+
+
+@pytest.mark.parametrize("w", [SMALL_BF16.scaled(name="half_m4", B=5, cap=1000, T=1300),
+                               SMALL_BF16.scaled(name="half_m5_dh256", M=5, d=512, enc_heads=2, enc_dff=1024, B=5,
+                                                 cap=1000, T=1000),
+                               SMALL_BF16.scaled(name="half_attn_only", enc_layers=2, enc_ffn=0, B=5, cap=1000, T=1100)],
+                         ids=lambda w: w.name)
+def test_prompt_sized_passes_with_a_single_fp16_operand(w):
+    # z2z_set_encoder_half_scratch: calls that span several prompt-sized passes copy the encoder's
+    # linear-layer weights to fp16 and round each activation once to fp16 (one MMA per k-step).  Held
+    # to the same tolerance as the two-part form, against the same oracle rows.
+    p = Pair(w, seed=48)
+    codes, clen, after = p.gpu_encode()
+    ocodes, _ = p.oracle.prefill([p.tokens[b].tolist() for b in range(w.B)])
+    for b in range(w.B):
+        assert codes[b, :clen[b]].tolist() == ocodes[b]
+    bound = w.B * w.cap                                        # 5 passes of 1024 entries each
+    worst2, E2, U2 = _embed_all_both_sides(p, bound)
+    zb.z2z_profile_read(p.cb)
+    scratch = torch.empty(zb.encoder_half_bytes(p.cfg) + 256, dtype=torch.uint8, device=DEV)
+    scratch = scratch[(-scratch.data_ptr()) % 256:][:zb.encoder_half_bytes(p.cfg)]
+    zb.z2z_set_encoder_half_scratch(p.cb, scratch)
+    zb.z2z_codebook_init(p.cb)                                 # same handle, new session: embed everything again
+    p.gpu_encode()
+    p.E_h.zero_(); p.U_h.zero_()
+    worst1, E1, U1 = _embed_all_both_sides(p, bound)
+    assert worst1 <= TOL and worst2 <= TOL
+    assert not torch.equal(E1, E2) and not torch.equal(U1, U2)            # the other arithmetic really ran
+    assert worst1 >= worst2                                     # 11 mantissa bits against about 16
+    print(f"{w.name}: max |hyper-embedding error| two-part {worst2:.3e}, single fp16 operand {worst1:.3e}")
+    st, _ = zb.z2z_status(p.cb)
+    assert int(st.max()) & zb.ST_HALF_RANGE == 0
+    # short calls (fewer than four passes) keep the two-part form: bit-identical to the first run
+    zb.z2z_codebook_init(p.cb)
+    p.gpu_encode()
+    assert sum(bk.n() for bk in p.oracle.books) <= 3 * 1024
+    worst3, E3, U3 = _embed_all_both_sides(p, 3 * 1024)
+    assert torch.equal(E3, E2) and torch.equal(U3, U2)
+    # ... and without the scratch everything is as before
+    zb.z2z_set_encoder_half_scratch(p.cb, None)
+    zb.z2z_codebook_init(p.cb)
+    p.gpu_encode()
+    worst4, E4, U4 = _embed_all_both_sides(p, bound)
+    assert worst4 == worst2
+
+
+def test_half_scratch_reports_weights_beyond_fp16_range():
+    w = SMALL_BF16.scaled(name="half_range", B=5, cap=1000, T=600)
+    p = Pair(w, seed=49)
+    p.gpu_encode()
+    scratch = torch.empty(zb.encoder_half_bytes(p.cfg) + 256, dtype=torch.uint8, device=DEV)
+    scratch = scratch[(-scratch.data_ptr()) % 256:][:zb.encoder_half_bytes(p.cfg)]
+    zb.z2z_set_encoder_half_scratch(p.cb, scratch)
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, w.B * w.cap, p.E_h, None)
+    st, _ = zb.z2z_status(p.cb)
+    assert int(st.max()) & zb.ST_HALF_RANGE == 0
+    p.g_encE_t[1 + 8][3, 5] = 1.0e6                             # W1 of layer 0: not representable in fp16
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, w.B * w.cap, p.E_h, None)
+    st, _ = zb.z2z_status(p.cb)
+    assert all(int(x) & zb.ST_HALF_RANGE for x in st)
+    with pytest.raises(zb.Z2ZError, match="aligned"):
+        zb.z2z_set_encoder_half_scratch(p.cb, scratch[8:])
 
 
 def test_attention_only_layers_on_every_encoder_path():

@@ -319,9 +319,11 @@ def run_decode(args, w: si.Workload, inputs: Inputs, rank: int, world: int):
     ev[0].record()
     zb.z2z_lzw_encode(cb, g_tok, None, codes, clen, None)
     ev[1].record()
-    zb.z2z_hyper_embed(cb, zb.CACHE_EMBED, g_WE, encE, None, None, w.B * w.T, E_h, None)
+    n_codes = int(clen.sum().item())           # a prompt creates fewer entries than it has codes
+    ev[3].record()
+    zb.z2z_hyper_embed(cb, zb.CACHE_EMBED, g_WE, encE, None, None, n_codes, E_h, None)
     if not w.tied:
-        zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, w.B * w.T, U_h, None)
+        zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, n_codes, U_h, None)
     ev[2].record()
     torch.cuda.synchronize()
     forced_dev = None
@@ -335,9 +337,13 @@ def run_decode(args, w: si.Workload, inputs: Inputs, rank: int, world: int):
             zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, w.B * w.T, U_h, None)
         torch.cuda.synchronize()
     st, n0 = zb.z2z_status(cb)
-    prefill = {"lzw_encode_ms": ev[0].elapsed_time(ev[1]), "hyper_embed_all_ms": ev[1].elapsed_time(ev[2]),
+    _, setup_launches = zb.z2z_profile_read(cb)
+    prefill = {"lzw_encode_ms": ev[0].elapsed_time(ev[1]), "hyper_embed_all_ms": ev[3].elapsed_time(ev[2]),
                "prompt_tokens": int(w.B * w.T), "compressed_tokens": int(clen.sum().item()),
-               "hypertokens": int(n0.sum().item())}
+               "hypertokens": int(n0.sum().item()),
+               "launches": setup_launches,
+               "note": "session set-up, not part of the timed steps; z2z_hyper_embed is given max_entries = "
+                       "the prompts' code count, which bounds its passes of 1024 entries"}
 
     nxt_all = torch.zeros(max_steps, w.B, dtype=torch.int32, device=dev)
     lse = torch.zeros(w.B, dtype=torch.float32, device=dev)
@@ -372,7 +378,7 @@ def run_decode(args, w: si.Workload, inputs: Inputs, rank: int, world: int):
     _, n_now = zb.z2z_status(cb)
     room_steps = int(w.cap - int(n_now.max().item())) - 3 * Ka - 1
     room_steps = min(room_steps, max_steps - cursor[0] - 3 * Ka)
-    R = plan_regions(K, est_ms, room_steps)
+    R = plan_regions(K, est_ms, room_steps, args.min_timed_s)
     if world > 1:                              # every rank runs the same number of regions
         rr = torch.tensor([R], device=dev, dtype=torch.int64)
         torch.distributed.all_reduce(rr, op=torch.distributed.ReduceOp.MIN)
@@ -890,6 +896,9 @@ def main(argv=None):
     ap.add_argument("--prompt-encoder", default="fp16", choices=["fp16", "two_part"],
                     help="prompt-scoring workloads: hyper-encoder GEMM operands (fp16: one tensor-core pass per "
                          "k-step on fp16 weight copies; two_part: bf16 hi + lo activation parts, two passes)")
+    ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S,
+                    help="device time the repeated K-step regions of a decode workload must cover (0: one region, "
+                         "for runs under a profiler)")
     ap.add_argument("--stub", action="store_true", help="launcher self-test: ranks report fixed numbers, no GPU work")
     args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3)

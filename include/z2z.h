@@ -130,7 +130,12 @@ int32_t z2z_lzw_step(z2z_codebook* cb, const int32_t* d_new_codes, const uint8_t
  *            only selects which "embedded so far" counter is used when d_first/d_count are NULL.
  *   d_table  [V, d]; enc: that side's encoder.
  *   d_first / d_count [B] or both NULL = every entry created since the last such call.
- *   max_entries  host upper bound on sum_b count_b (<= 0: B * cap); bounds the launch count.
+ *   max_entries  host upper bound on sum_b count_b (<= 0: B * cap).  It bounds the launch count:
+ *            entries are processed in passes of 1024, and a pass is about ten launches per layer
+ *            whether or not it finds entries (the counts are device state).  After z2z_lzw_encode
+ *            pass the number of prompt tokens (or the sum of the code lengths, if known on the
+ *            host): a prompt of T tokens creates fewer than T entries.  With 0 a large session
+ *            (B * cap = 524288) would enqueue 512 passes.
  *   d_cache  [B, cap, d] in the configured dtype (row k of sequence b = hypertoken V + k).
  *   d_cache_f32 [B, cap, d] fp32 or NULL: the same rows before rounding to the cache dtype.    */
 int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,

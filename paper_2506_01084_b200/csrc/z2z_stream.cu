@@ -267,7 +267,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t a_bytes = (uint32_t)KSB * p.a_box_rows * 128;
   const uint32_t stage_bytes = a_bytes + (uint32_t)KSB * NT * 128;
-  const bool shifted = p.row_tiles == 1;           // one row tile: the box is shifted so that only live rows are read
+  const bool narrow_n = p.row_tiles == 1;          // one row tile: the MMA's N follows the live rows
   pdl_trigger();                                   // the next kernel may get resident behind this one
   setup_barriers<STAGES>(ctrl);
   if (warp == 0 && lane == 0) { prefetch_tmap(&tmA0); prefetch_tmap(&tmW0); if (p.groups > 1) { prefetch_tmap(&tmA1); prefetch_tmap(&tmW1); } }
@@ -283,25 +283,19 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
       // ---- TMA producer.  The weight tiles depend on no earlier kernel, the activation tiles do:
       // during the first pass over the ring only the weight boxes are issued and the activation
       // boxes are noted; once the ring is full (or the work ends) the producer waits for the
-      // preceding kernel, learns how many rows are live and issues them.  With an ordinary launch
-      // the wait returns at once.
+      // preceding kernel and issues them.  With an ordinary launch the wait returns at once.
       const CUtensorMap* amaps[2] = {&tmA0, &tmA1};
       const CUtensorMap* wmaps[2] = {&tmW0, &tmW1};
       const uint64_t pol_w = policy_evict_first(), pol_a = policy_evict_last();
       struct Deferred { uint32_t dst, bar; int map, arow, kb; };
       Deferred def[kMaxStages];
-      int n_def = 0, issued = 0, live = 0;
+      int n_def = 0, issued = 0;
       bool deps = false, ok = true;
-      // first operand row of the box of the row tile that starts at packed row `arow`
-      auto box_row = [&](int arow) {
-        return shifted ? 2 * gemm_tile_rows8(p, live, arow) - p.a_box_rows : 2 * arow;
-      };
       auto need_deps = [&]() {
         if (deps) return;
         pdl_wait();
-        live = *p.rows_dev;
         for (int i = 0; i < n_def; ++i)
-          tma_load_3d(def[i].dst, amaps[def[i].map], 0, box_row(def[i].arow), def[i].kb, def[i].bar, pol_a);
+          tma_load_3d(def[i].dst, amaps[def[i].map], 0, 2 * def[i].arow, def[i].kb, def[i].bar, pol_a);
         deps = true;
       };
       int stage = 0; uint32_t phase = 0;
@@ -315,7 +309,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
           mbar_expect_tx(full, stage_bytes);        // rows of a box outside the tensor are zero-filled and counted
           const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
           tma_load_3d(sb + a_bytes, wmaps[j.g], 0, j.wrow, ks * KSB, full, pol_w);
-          if (deps) tma_load_3d(sb, amaps[j.g], 0, box_row(j.arow), ks * KSB, full, pol_a);
+          if (deps) tma_load_3d(sb, amaps[j.g], 0, 2 * j.arow, ks * KSB, full, pol_a);
           else { def[n_def].dst = sb; def[n_def].bar = full; def[n_def].map = j.g; def[n_def].arow = j.arow; def[n_def].kb = ks * KSB; ++n_def; }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -336,9 +330,8 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
         const uint32_t buf = job_i & 1u, aph = (job_i >> 1) & 1u;
         if (!mbar_wait(smem_u32(&ctrl->acc_empty[buf]), aph ^ 1u, &ctrl->abort)) break;
         tc_fence_after();
-        // N and the operand's first row inside the box (a multiple of 8 rows = one swizzle atom)
-        const int n_rows = shifted ? 2 * gemm_tile_rows8(p, live, j.arow) : p.a_box_rows;
-        const uint32_t a_off = (uint32_t)(p.a_box_rows - n_rows) * 128;
+        // N covers the live operand rows, which sit at the start of the box (a multiple of 16)
+        const int n_rows = narrow_n ? 2 * gemm_tile_rows8(p, live, j.arow) : p.a_box_rows;
         const uint32_t idesc = idesc_bf16_f32(128, n_rows);
         const uint32_t d = tmem_base + buf * (uint32_t)p.a_box_rows;
         uint32_t acc = 0;
@@ -348,7 +341,7 @@ k_stream_gemm(const StreamGemmParams p, const __grid_constant__ CUtensorMap tmA0
           const uint32_t sb = stage_base + (uint32_t)stage * stage_bytes;
 #pragma unroll
           for (int i = 0; i < KSB; ++i) {
-            const uint32_t ab = sb + (uint32_t)i * p.a_box_rows * 128 + a_off;
+            const uint32_t ab = sb + (uint32_t)i * p.a_box_rows * 128;
             const uint32_t wb = sb + a_bytes + (uint32_t)i * NT * 128;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {

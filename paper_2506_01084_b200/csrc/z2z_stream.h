@@ -56,13 +56,11 @@ cudaError_t run_logits_decode(const CbView& cb, const LogitsArgs& a, int* counte
 //
 // The activation operand holds the hi part and the lo part of PACKED row r in rows 2r and 2r + 1
 // (bf16 [2 * Rt, K]); only the first *rows_dev packed rows carry data, a count that only the device
-// knows.  One TMA box of a_box_rows (= 2 * min(Rt, 128)) operand rows is loaded per stage.  With
-// a single row tile the box starts at the NEGATIVE row 2 * P8 - a_box_rows (P8 = live rows rounded
-// up to 8): the rows before row 0 are filled with zeros without touching memory, the live rows
-// land at the end of the box, and the MMA's N is 2 * P8 - so the bytes an SM takes in per weight
-// tile follow the number of rows that exist, not the capacity of the pass.  The epilogue adds the
-// hi and lo columns of a row in registers and reduces the sums into the fp32 result matrix
-// out[group][Rt][J] (lanes = consecutive features = consecutive addresses).
+// knows.  One TMA box of a_box_rows (= 2 * min(Rt, 128)) operand rows is loaded per stage; with a
+// single row tile the MMA's N is 2 * P8 (P8 = live rows rounded up to 8): the tensor-core work
+// and the epilogue's reductions follow the number of rows that exist, not the capacity of the
+// pass.  The epilogue adds the hi and lo columns of a row in registers and reduces the sums into
+// the fp32 result matrix out[group][Rt][J] (lanes = consecutive features = consecutive addresses).
 struct StreamGemmParams {
   int row_tiles;         // 128-row tiles of the packed activation rows (outermost dimension of the unit space)
   int groups, tiles_per_group, ksteps;

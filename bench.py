@@ -656,8 +656,10 @@ def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: i
     def step(tok_dev, hid_dev):
         zb.z2z_codebook_init(cb)
         zb.z2z_lzw_encode(cb, tok_dev, None, codes, clen, None)
-        zb.z2z_hyper_embed(cb, zb.CACHE_EMBED, g_WE, encE, None, None, w.B * w.T, E_h, None)
-        zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, w.B * w.T, U_h, None)
+        # max_entries = -1: the call reads the entry count back (one wait on the stream) instead of
+        # enqueueing a pass for every 1024 entries the prompts could have created at most
+        zb.z2z_hyper_embed(cb, zb.CACHE_EMBED, g_WE, encE, None, None, -1, E_h, None)
+        zb.z2z_hyper_embed(cb, zb.CACHE_UNEMBED, g_WU, encU, None, None, -1, U_h, None)
         zb.z2z_dynamic_logits(cb, hid_dev, row_seq, None, g_WU, U_h, zb.SELECT_ARGMAX, 1.0, 0, 0, None,
                               lse, am, mx)
 

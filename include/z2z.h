@@ -16,7 +16,8 @@
  *     buffer; the library allocates no device memory.  The opaque handle is host memory that
  *     stores the configuration and offsets into the caller's workspace.
  *   - All work is enqueued on the given stream and returns without synchronising (except
- *     z2z_status, which waits for the stream).  The enqueueing calls may therefore be captured
+ *     z2z_status, z2z_codebook_read, z2z_profile_read and z2z_hyper_embed with max_entries < 0,
+ *     which wait for the stream).  The enqueueing calls may therefore be captured
  *     into a CUDA graph (arguments passed by value, the sampling step among them, are then fixed
  *     for every replay); capture again after z2z_codebook_init starts a new session, because
  *     z2z_decode_step decides on the host whether the session still needs its hyper-encoder pass.
@@ -136,6 +137,10 @@ int32_t z2z_lzw_step(z2z_codebook* cb, const int32_t* d_new_codes, const uint8_t
  *            pass the number of prompt tokens (or the sum of the code lengths, if known on the
  *            host): a prompt of T tokens creates fewer than T entries.  With 0 a large session
  *            (B * cap = 524288) would enqueue 512 passes.
+ *            max_entries < 0: exact.  The call reads the number of entries it has to embed back
+ *            from the device - it waits for the stream once, the only enqueueing call that does,
+ *            and therefore cannot be captured into a graph - and launches no pass without work.
+ *            Meant for whole prompts, where hundreds of empty passes would cost more than the wait.
  *   d_cache  [B, cap, d] in the configured dtype (row k of sequence b = hypertoken V + k).
  *   d_cache_f32 [B, cap, d] fp32 or NULL: the same rows before rounding to the cache dtype.    */
 int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,

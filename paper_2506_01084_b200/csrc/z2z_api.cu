@@ -297,8 +297,22 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
   z2z::EncoderArgs a = encoder_args(cb, d_table, enc, d_cache, d_cache_f32, el.chunk);
   const bool tc = cb->use_tensor_cores && cb->cfg.enc_layers >= 0 &&
                   z2z::encoder_tc_supported(cb->cfg.d, cb->dff, cb->cfg.dtype, cb->heads, cb->cfg.M);
+  {
+    z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
+    Z2Z_CUDA(z2z::launch_entry_offsets(cb->view, which, d_first, d_count, el, s), "hyper_embed");
+  }
   long long bound = (long long)cb->cfg.B * cb->cfg.cap;
   if (max_entries > 0 && max_entries < bound) bound = max_entries;
+  if (max_entries < 0) {
+    // exact: read the number of entries this call has to embed back from the device (the one
+    // place where an enqueueing call waits for the stream), so that no pass is launched for nothing
+    int32_t total = 0;
+    int32_t* land = cb->h_frozen ? cb->h_frozen + 8 : &total;      // pinned host word when there is one
+    Z2Z_CUDA(cudaMemcpyAsync(land, el.off + cb->cfg.B, 4, cudaMemcpyDeviceToHost, s), "hyper_embed (entry count)");
+    Z2Z_CUDA(cudaStreamSynchronize(s), "hyper_embed (entry count)");
+    total = *reinterpret_cast<volatile int32_t*>(land);
+    if (total >= 0 && total < bound) bound = total;
+  }
   const int n_chunks = (int)((bound + el.chunk - 1) / el.chunk);
   // Single-pass fp16 form of the prompt-sized passes: when the caller has lent memory for the
   // weight copies and the call is long enough (several passes) to repay making them.
@@ -310,10 +324,6 @@ int32_t z2z_hyper_embed(z2z_codebook* cb, int32_t which, const void* d_table,
     Z2Z_CUDA(z2z::convert_encoder_weights_to_half(enc->tensors, cb->cfg.d, cb->dff, cb->cfg.enc_layers, cb->half_scratch,
                                                   cb->half_ptrs.data(), a.err, &cb->prof, s), "hyper_embed (fp16 weight copies)");
     a.w_half = cb->half_ptrs.data();
-  }
-  {
-    z2z::ProfScope ps(&cb->prof, z2z::kProfEncOther, 1, s);
-    Z2Z_CUDA(z2z::launch_entry_offsets(cb->view, which, d_first, d_count, el, s), "hyper_embed");
   }
   for (int c = 0; c < n_chunks; ++c) {
     {

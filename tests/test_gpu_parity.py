@@ -227,6 +227,21 @@ def test_hyper_embed_explicit_ranges_and_incremental():
     got = p.E_f32.cpu().double().numpy()
     for b in range(w.B):
         assert np.abs(got[b, :n[b]] - p.oracle.E_exact[b]).max() <= TOL
+    # max_entries < 0: the call reads the entry count back and launches only passes with work;
+    # the same rows come out, and a call with nothing to do launches no encoder kernel at all
+    first_run = p.E_f32.clone()
+    zb.z2z_codebook_init(p.cb)
+    p.gpu_encode()
+    p.E_f32.zero_()
+    zb.z2z_profile_read(p.cb)
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, -1, p.E_h, p.E_f32)
+    assert float((p.E_f32 - first_run).abs().max()) <= 1e-5
+    _, launches = zb.z2z_profile_read(p.cb)
+    assert launches["encoder_gemm"] > 0
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, -1, p.E_h, p.E_f32)   # nothing new
+    _, launches = zb.z2z_profile_read(p.cb)
+    assert launches["encoder_gemm"] == 0
+    assert float((p.E_f32 - first_run).abs().max()) <= 1e-5
 
 
 # ------------------------------------------------------------------------------------------------

@@ -13,6 +13,9 @@ namespace z2z {
 
 __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateArgs a, EntryList el) {
   __shared__ int s_cnt[1024];
+  __shared__ int s_n[1024];                 // hypertokens of the sequence after this step
+  __shared__ signed char s_len[1024];       // base tokens of the entry it created
+  __shared__ int s_tok[1024][kMaxM];        // ... and the tokens themselves: the work list needs no reload
   __shared__ int s_warp[32];
   sm100::pdl_trigger();
   sm100::pdl_wait();               // the logits partials and the codebook state come from earlier kernels
@@ -50,10 +53,14 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
       a.next_codes[b] = code;
     }
     // ---- online LZW update with the applied code
-    const int created = sits_out ? -1 : warp_lzw_step(cb, b, code, state);
+    int new_tok = -1;
+    const int created = sits_out ? -1 : warp_lzw_step(cb, b, code, state, &new_tok);
+    if (lane < cb.M) s_tok[b][lane] = new_tok;
     if (lane == 0) {
       if (a.new_entry) a.new_entry[b] = created;
       s_cnt[b] = created >= 0 ? created + 1 : 0;         // 0: none, else entry number + 1
+      s_len[b] = (signed char)(created >= 0 ? state.plen + 1 : 0);
+      s_n[b] = state.n + (created >= 0 ? 1 : 0);
     }
   }
   __syncthreads();
@@ -63,7 +70,7 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
   // half, rows in the high half (at most 1024 entries of at most 8 rows).
   const int mine = tid < cb.B ? s_cnt[tid] : 0;
   const int flag = mine > 0 ? 1 : 0;
-  const int my_len = flag ? (int)cb.len[(size_t)tid * cb.cap + (mine - 1)] : 0;     // written above by this block
+  const int my_len = flag ? (int)s_len[tid] : 0;
   const int val = flag | (my_len << 16);
   int incl = val;
 #pragma unroll
@@ -96,7 +103,7 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
     el.len[excl] = my_len;
     el.row_off[excl] = row0;
     for (int i = 0; i < cb.M; ++i) {
-      const int tok = cb.cons[((size_t)tid * cb.cap + (mine - 1)) * cb.M + i];
+      const int tok = s_tok[tid][i];
       el.tok[(size_t)excl * cb.M + i] = tok;
       if (i < my_len) { el.row_src[row0 + i] = excl * cb.M + i; el.row_tok[row0 + i] = tok; }
     }
@@ -108,7 +115,7 @@ __global__ void __launch_bounds__(1024) k_decode_update(CbView cb, DecodeUpdateA
   // both caches will hold every entry once the encoder pass that follows has run
   int full = 1;
   if (tid < cb.B) {
-    const int n = cb.n[tid];
+    const int n = s_n[tid];
     cb.n_emb[tid] = n; cb.n_emb[cb.B + tid] = n;
     full = n >= cb.cap && mine == 0;             // full already when this step began: it created nothing
   }

@@ -57,22 +57,50 @@ __device__ __forceinline__ void warp_write_entry(const CbView& cb, int b, int k,
 }
 
 // The part of a sequence's state that the update needs and that does not depend on the new code;
-// a caller that still has to compute the code can load it ahead.
-struct LzwPrev { int n, prev, plen; };
+// a caller that still has to compute the code can load it ahead.  ptok: base token `lane` of the
+// previous phrase (-1 beyond its length), so that writing a new entry needs no further load.
+struct LzwPrev { int n, prev, plen, ptok; };
 __device__ __forceinline__ LzwPrev warp_lzw_load(const CbView& cb, int b) {
+  const int lane = threadIdx.x & 31;
   LzwPrev s;
   s.n = cb.n[b];
   s.prev = cb.prev[b];
   s.plen = 0;
-  if (s.prev >= 0) s.plen = s.prev < cb.V ? 1 : (int)cb.len[(size_t)b * cb.cap + (s.prev - cb.V)];
+  s.ptok = -1;
+  if (s.prev >= 0) {
+    if (s.prev < cb.V) {
+      s.plen = 1;
+      if (lane == 0) s.ptok = s.prev;
+    } else {
+      const size_t e = (size_t)b * cb.cap + (s.prev - cb.V);
+      if (lane < cb.M) s.ptok = cb.cons[e * cb.M + lane];      // -1 padded behind the phrase
+      s.plen = (int)cb.len[e];
+    }
+  }
   return s;
+}
+// Write entry k = phrase(prev) ++ c from the previous phrase's tokens held by the lanes; returns the
+// token this lane wrote (-1: padding, or a lane beyond M).
+__device__ __forceinline__ int warp_write_entry_from(const CbView& cb, int b, int k, const LzwPrev& s, int c) {
+  const int lane = threadIdx.x & 31;
+  int v = -1;
+  if (lane < cb.M) {
+    if (lane < s.plen) v = s.ptok;
+    else if (lane == s.plen) v = c;
+    cb.cons[((size_t)b * cb.cap + k) * cb.M + lane] = v;
+  }
+  if (lane == 0) cb.len[(size_t)b * cb.cap + k] = (uint8_t)(s.plen + 1);
+  return v;
 }
 // Online update of sequence b with the newly selected code z (Figure 1; Section 2.3 step 10).
 // Candidate entry = phrase(prev) ++ first(phrase(z)); returns the entry created, or -1.
 // A code that names no existing (or about-to-exist) hypertoken raises BAD_TOKEN and leaves the
 // sequence untouched.
-__device__ __forceinline__ int warp_lzw_step(const CbView& cb, int b, int z, const LzwPrev& s) {
+// new_tok (optional): base token `lane` of the entry created (-1 if none / padding).
+__device__ __forceinline__ int warp_lzw_step(const CbView& cb, int b, int z, const LzwPrev& s,
+                                             int* new_tok = nullptr) {
   const int lane = threadIdx.x & 31;
+  if (new_tok) *new_tok = -1;
   unsigned long long* table = cb.hash + (size_t)b * cb.n_slots;
   const int n = s.n;
   const int prev = s.prev;
@@ -91,7 +119,8 @@ __device__ __forceinline__ int warp_lzw_step(const CbView& cb, int b, int z, con
       if (p.found < 0) {
         if (p.slot >= 0) {
           if (lane == 0) table[p.slot] = pack_slot((uint32_t)prev, (uint32_t)first, (uint32_t)n);
-          warp_write_entry(cb, b, n, prev, plen, first);
+          const int wrote = warp_write_entry_from(cb, b, n, s, first);
+          if (new_tok) *new_tok = wrote;
           created = n;
           if (n + 1 >= cb.cap) st |= Z2Z_ST_CAP_FROZEN;
         } else {

@@ -579,9 +579,9 @@ def oracle_sample(w: si.Workload, n_steps: int, seed: int = 1000, prompt_tokens:
     return {"value": base / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
             "threads": torch.get_num_threads(),
             "sample": f"{n_steps} decode steps of the full-shape workload {w.name} (V, d, B, M, encoder as "
-                      f"configured) after prompts CUT to {T} of {w.T} tokens (a smaller codebook state than the "
-                      f"GPU arm's); oracle prefill took {t_prefill:.1f} s; numpy fp64, "
-                      f"{torch.get_num_threads()} threads",
+                      f"configured) after " + (f"prompts CUT to {T} of {w.T} tokens (a smaller codebook state than "
+                      f"the GPU arm's)" if T < w.T else f"the full prompts of {T} tokens") +
+                      f"; oracle prefill took {t_prefill:.1f} s; numpy fp64, {torch.get_num_threads()} threads",
             "seconds": dt, "ms_per_step": dt / n_steps * 1e3}
 
 

@@ -161,7 +161,7 @@ def reduce_over_ranks(times_ms, counts, world: int, device):
 def plan_regions(K: int, est_ms_per_step: float, steps_available: int, min_s: float = MIN_TIMED_S) -> int:
     """Number of K-step regions: enough to cover `min_s` of device time at the estimated step
     time, at most what the session's remaining codebook room (in steps) allows, at least one."""
-    want = int(math.ceil(min_s * 1e3 / max(K * est_ms_per_step, 1e-6)))
+    want = int(math.ceil(1.1 * min_s * 1e3 / max(K * est_ms_per_step, 1e-6)))    # 10 % over: the estimate is a probe
     room = max(1, steps_available // max(K, 1))
     return max(1, min(want, room, MAX_REGIONS))
 

@@ -71,7 +71,32 @@ def test_gpus_flag_starts_the_ranks_itself():
 
 def test_region_planning():
     import bench
-    assert bench.plan_regions(20, 0.25, 10 ** 6) == 60       # 0.3 s / (20 x 0.25 ms)
+    assert bench.plan_regions(20, 0.25, 10 ** 6) == 66       # 1.1 x 0.3 s / (20 x 0.25 ms)
     assert bench.plan_regions(20, 0.25, 100) == 5            # bounded by the codebook room in steps
     assert bench.plan_regions(256, 2.0, 10 ** 6) == 1        # one region already covers 0.3 s
     assert bench.plan_regions(20, 0.25, -5) == 1
+
+
+def test_inputs_shared_between_workloads_equal_fresh_draws():
+    # bench.Inputs keeps generated tensors per (shape, seed) and, for a workload that differs from a
+    # cached one only in the merge size, draws the position table alone: the result must be what
+    # synth_inputs.make_encoder draws for that workload from scratch
+    import bench
+    from paper_2506_01084_b200 import synth_inputs as si
+    base = si.Workload("w3", V=300, d=64, dtype="bf16", B=2, T=32, M=3, cap=16, zipf_s=1.1, copy_p=0.3,
+                       seg_min=2, seg_max=5, steps=1, enc_layers=2, enc_heads=2, enc_dff=128)
+    other = base.scaled(name="w5", M=5)
+    inp = bench.Inputs(torch.device("cpu"))
+    first = inp.encoder(base, 77)
+    again = inp.encoder(other, 77)
+    fresh = si.make_encoder(other, 77)
+    assert len(again) == len(fresh) and again[0].shape == (5, 64)
+    for a, b in zip(again, fresh):
+        assert torch.equal(a, b)
+    for a, b in zip(first, si.make_encoder(base, 77)):
+        assert torch.equal(a, b)
+    assert inp.encoder(base, 77)[3] is first[3]                # cached, not drawn again
+    te, tu = inp.tables(base, 5)
+    fe, fu = si.make_tables(base, 5)
+    assert torch.equal(te, fe) and torch.equal(tu, fu)
+    assert inp.to_dev(te) is inp.to_dev(te)

@@ -124,11 +124,19 @@ int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s, z2z::Logits
   const bool prefill = tc && info == nullptr && z2z::prefill_logits_supported(cb->cfg.d, cb->cfg.dtype) &&
                        (cb->use_tensor_cores == 2 || N >= kPrefillMinRows);
   long long chunk = z2z::kLogitRowChunk;
+  int prefill_strips = cb->prefill_strips;
   if (prefill) {
-    const int strips = cb->prefill_strips > 0 ? cb->prefill_strips : z2z::prefill_logits_strips(N);
-    chunk = z2z::prefill_logits_max_rows(cb->plan.lpart_bytes, cb->plan.plan_bytes, strips);
-    if (chunk < N)      // several launches: size them for the worst split
-      chunk = z2z::prefill_logits_max_rows(cb->plan.lpart_bytes, cb->plan.plan_bytes, z2z::kPrefillMaxStrips);
+    // the number of column strips is fixed for the whole call; when the partial-reduction scratch
+    // cannot take all rows at that split, the rows go out in launches of equal size
+    if (prefill_strips <= 0) prefill_strips = z2z::prefill_logits_strips(N, cb->cfg.d);
+    const long long cap_rows = z2z::prefill_logits_max_rows(cb->plan.lpart_bytes, cb->plan.plan_bytes, prefill_strips);
+    if (cap_rows < 256) return fail(Z2Z_ERR_WORKSPACE_TOO_SMALL, "logits scratch too small for one row tile");
+    chunk = cap_rows;
+    if (chunk < N) {
+      const long long launches = (N + cap_rows - 1) / cap_rows;
+      chunk = ((N + launches - 1) / launches + 255) / 256 * 256;
+      if (chunk > cap_rows) chunk = cap_rows;
+    }
   }
   for (long long r0 = 0; r0 < N; r0 += chunk) {
     z2z::LogitsArgs c = a;
@@ -148,7 +156,7 @@ int logits_call(z2z_codebook* cb, z2z::LogitsArgs a, cudaStream_t s, z2z::Logits
     int* words = reinterpret_cast<int*>(cb->ws + cb->plan.off_words);
     if (prefill) {
       Z2Z_CUDA(z2z::run_logits_prefill(cb->view, c, reinterpret_cast<int32_t*>(cb->ws + cb->plan.off_plan), words,
-                                       cb->prefill_strips, &cb->prof, s), "logits (prompt scoring)");
+                                       prefill_strips, &cb->prof, s), "logits (prompt scoring)");
     } else if (tc) {
       Z2Z_CUDA(z2z::run_logits_tc(cb->view, c, words + 1, words, info, &cb->prof, s), "logits (tensor cores)");
     } else {

@@ -81,7 +81,7 @@ struct WsPlan {
 };
 
 constexpr int kLogitRowChunk = 8192;              // rows per logits launch (larger N loops)
-constexpr int kLogitPartRows = 1 << 19;           // partial-reduction slots (rows x groups)
+constexpr int kLogitPartRows = 1 << 20;           // partial-reduction slots (rows x groups), 32 bytes each
 constexpr int kPrefillPlanTiles = 1 << 14;        // 256-row tiles one prompt-scoring launch may have
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -124,7 +124,7 @@ cudaError_t run_logits_tc(const CbView& cb, const LogitsArgs& a, int* vt_word, i
 bool prefill_logits_supported(int d, int dtype);
 // Rows one launch can take with the given scratch when `strips` partials per row are needed.
 long long prefill_logits_max_rows(size_t lpart_bytes, size_t plan_bytes, int strips);
-int prefill_logits_strips(int N);
+int prefill_logits_strips(int N, int d);
 cudaError_t run_logits_prefill(const CbView& cb, const LogitsArgs& a, int32_t* plan, int* err_word,
                                int strips_override, Prof* prof, cudaStream_t s);
 

@@ -363,11 +363,33 @@ static int sm_count_prefill() {
   return n_sm;
 }
 
-// Number of column strips per row tile: the smallest split that keeps the clusters busy in the
-// last round too (at least 90 %), at most kPrefillMaxStrips.
-static int pick_strips(int row_tiles, int n_clusters) {
-  int best = 1; double best_eff = 0.0;
-  for (int s = 1; s <= kPrefillMaxStrips; ++s) {
+static size_t l2_bytes_prefill() {
+  static size_t l2 = 0;
+  if (!l2) {
+    int dev = 0, v = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, dev);
+    l2 = v > 0 ? (size_t)v : ((size_t)64 << 20);
+  }
+  return l2;
+}
+
+// Number of column strips per row tile.  Two conditions:
+//   * the hidden-row tiles that are in work at the same time must stay in the L2 cache, because a
+//     pair re-reads its 256 x d tile for every column tile of its strip: n_clusters / strips tiles
+//     of 512 d bytes within a third of the cache (with one strip at d = 4096 the 74 pairs keep
+//     148 MB of tiles in work, more than the cache holds, and every column tile fetches its
+//     hidden rows from HBM again: 0.92 instead of 1.15 PFLOP/s at 1.8e5 rows);
+//   * the clusters should be busy in the last round too (at least 90 %).
+// The smallest split that meets both, at most kPrefillMaxStrips.
+static int pick_strips(int row_tiles, int n_clusters, int d) {
+  const size_t tile_bytes = (size_t)kTileRows * d * 2;
+  const size_t budget = l2_bytes_prefill() / 3;
+  int s_min = (int)(((size_t)n_clusters * tile_bytes + budget - 1) / budget);
+  if (row_tiles < n_clusters) s_min = (int)(((size_t)row_tiles * tile_bytes + budget - 1) / budget);
+  s_min = s_min < 1 ? 1 : (s_min > kPrefillMaxStrips ? kPrefillMaxStrips : s_min);
+  int best = s_min; double best_eff = 0.0;
+  for (int s = s_min; s <= kPrefillMaxStrips; ++s) {
     const long long units = (long long)row_tiles * s;
     const long long rounds = (units + n_clusters - 1) / n_clusters;
     const double eff = (double)units / (double)(rounds * n_clusters);
@@ -377,8 +399,8 @@ static int pick_strips(int row_tiles, int n_clusters) {
   return best;
 }
 
-int prefill_logits_strips(int N) {
-  return pick_strips((N + kTileRows - 1) / kTileRows, sm_count_prefill() / 2);
+int prefill_logits_strips(int N, int d) {
+  return pick_strips((N + kTileRows - 1) / kTileRows, sm_count_prefill() / 2, d);
 }
 
 cudaError_t run_logits_prefill(const CbView& cb, const LogitsArgs& a, int32_t* plan, int* err_word, int strips_override,
@@ -390,7 +412,7 @@ cudaError_t run_logits_prefill(const CbView& cb, const LogitsArgs& a, int32_t* p
   p.row_tiles = (a.N + kTileRows - 1) / kTileRows;
   p.n_static = (cb.V + kTileCols - 1) / kTileCols;
   const int max_clusters = n_sm / 2;
-  p.strips = strips_override > 0 ? strips_override : pick_strips(p.row_tiles, max_clusters);
+  p.strips = strips_override > 0 ? strips_override : pick_strips(p.row_tiles, max_clusters, a.d);
   if (p.strips > kPrefillMaxStrips) p.strips = kPrefillMaxStrips;
   if (p.strips > p.n_static) p.strips = p.n_static;          // every strip gets at least one tile
   p.tile_lo = plan; p.tile_hi = plan + p.row_tiles; p.tile_nh = plan + 2 * p.row_tiles;

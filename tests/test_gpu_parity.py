@@ -222,6 +222,13 @@ def test_hyper_embed_explicit_ranges_and_incremental():
         if hi > lo:
             assert np.abs(got[b, lo:hi] - p.oracle.E_exact[b][lo:hi]).max() <= TOL
         assert np.all(got[b, :lo] == 0) and np.all(got[b, hi:] == 0)
+    # the same ranges with the exact pass count (max_entries < 0): the same rows, nothing else touched
+    ranges_run = p.E_f32.clone()
+    p.E_f32.zero_()
+    zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE,
+                       torch.tensor(first, dtype=torch.int32, device=DEV),
+                       torch.tensor(count, dtype=torch.int32, device=DEV), -1, p.E_h, p.E_f32)
+    assert float((p.E_f32 - ranges_run).abs().max()) <= 1e-5
     # NULL ranges after that: "everything since the last NULL call" = all entries
     zb.z2z_hyper_embed(p.cb, zb.CACHE_EMBED, p.g_WE, p.g_encE, None, None, 0, p.E_h, p.E_f32)
     got = p.E_f32.cpu().double().numpy()

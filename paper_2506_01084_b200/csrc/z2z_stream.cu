@@ -7,10 +7,10 @@
 // issues tcgen05.mma (fp32 accumulators in tensor memory, double buffered), warps 2-5 drain
 // accumulators.  Two kernels share the ring and its barriers:
 //   * hyper-encoder linear layers (k_stream_gemm): a tile of 128 weight rows is the MMA's M
-//     operand, the activation rows (hi parts | lo parts) its N operand; work is cut stream-K
-//     style, every CTA gets the same number of (tile, k-step) units and adds its accumulators
-//     into one fp32 result matrix with reductions in global memory (sums of two or three partial
-//     tiles in arrival order);
+//     operand, the packed activation rows (hi and lo part of a row in adjacent operand rows) its
+//     N operand, as wide as the rows that exist; work is cut stream-K style, every CTA gets the
+//     same number of (tile, k-step) units and adds its accumulators into one fp32 result matrix
+//     with reductions in global memory (sums of two or three partial tiles in arrival order);
 //   * joint logits for 33 .. 2047 hidden rows (k_stream_logits; paper Section 2.3 steps 7-9):
 //     the hidden rows are the 128-row M operand, tiles run over W_U and then over the visible
 //     rows of each sequence's U_h; the epilogue keeps max / sum-exp / argmax / best perturbed

@@ -937,17 +937,24 @@ def main(argv=None):
                 gc.collect()
                 torch.cuda.empty_cache()
                 sw = si.WORKLOADS[name]
-                if sw.steps == 0:
-                    per[name] = run_prompt_scoring(args, sw, inputs, rank, world, max(1, args.prompt_steps), 3)
-                else:
-                    per[name] = run_decode(args, sw, inputs, rank, world)
+                try:
+                    if sw.steps == 0:
+                        per[name] = run_prompt_scoring(args, sw, inputs, rank, world, max(1, args.prompt_steps), 3)
+                    else:
+                        per[name] = run_decode(args, sw, inputs, rank, world)
+                except Exception as e:           # a sub-record must not cost the headline line
+                    per[name] = {"error": f"{type(e).__name__}: {e}"[:300]}
+                    continue
                 for k in ("metric", "unit", "higher_is_better", "scaling", "vs_baseline", "data", "n_gpus"):
                     if k != "metric" or sw.steps > 0:
                         per[name].pop(k, None)
             line["per_workload"] = per
         if rank == 0 and world == 1 and not args.no_cpu_baseline and not prompt_mode:
-            res = oracle_sample(w, n_steps=2 if w.d >= 2048 else 16, inputs=inputs)
-            line["cpu_baseline"] = {k: res[k] for k in ("value", "unit", "cores", "threads", "kind", "sample")}
+            try:
+                res = oracle_sample(w, n_steps=2 if w.d >= 2048 else 16, inputs=inputs)
+                line["cpu_baseline"] = {k: res[k] for k in ("value", "unit", "cores", "threads", "kind", "sample")}
+            except Exception as e:
+                line["cpu_baseline"] = {"error": f"{type(e).__name__}: {e}"[:300], "kind": "oracle"}
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

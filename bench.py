@@ -686,6 +686,22 @@ def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: i
         step(g_tok, hidden)
     zb.z2z_profile(cb, False)
     cls_ms, cls_launches = zb.z2z_profile_read(cb)
+    # the causal variant of the scoring call (Section 2.4: entries are created in order, so what a
+    # position sees is a per-row column limit; z2z_lzw_encode's entries_after supplies it), timed alone
+    after = torch.zeros(w.B, w.T, dtype=torch.int32, device=dev)
+    zb.z2z_codebook_init(cb)
+    zb.z2z_lzw_encode(cb, g_tok, None, codes, clen, after)
+    row_nvis = after[torch.arange(w.T, device=dev)[None, :] < clen[:, None]].contiguous()
+    causal_ms = []
+    for _ in range(3):
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        zb.z2z_dynamic_logits(cb, hidden, row_seq, row_nvis, g_WU, U_h, zb.SELECT_ARGMAX, 1.0, 0, 0, None,
+                              lse, am, mx)
+        c1.record()
+        torch.cuda.synchronize()
+        causal_ms.append(c0.elapsed_time(c1))
+    causal_flops = 2.0 * w.d * (float(N) * w.V + float(row_nvis.to(torch.int64).sum().item()))
     # end to end: prompts and hidden rows from pinned host memory, LSE back to the host
     Ke = 1
     tok_dev = torch.empty_like(g_tok)
@@ -738,6 +754,10 @@ def run_prompt_scoring(args, w: si.Workload, inputs: Inputs, rank: int, world: i
                      "traffic": None, "peak_source": pk["source"] + " (cuBLAS bf16, sustained)",
                      "flops_per_launch": flops * Kc / n_logit, "us_per_launch": cls_ms["logits"] / n_logit * 1e3,
                      "frac_of_burst_peak": tfs / pk["bf16_tflops"], "frac_of_nominal_2250": tfs / 2250.0,
+                     "causal": {"ms": min(causal_ms), "tflops": causal_flops / min(causal_ms) / 1e9,
+                                "frac": causal_flops / min(causal_ms) / 1e9 / pk["bf16_tflops_sustained"],
+                                "note": "the same call with per-row visibility limits (d_row_nvis = entries that exist "
+                                        "once the position's code is out), best of 3, whole call with its plan kernel"},
                      "encoder_gemm": {"kernel": "k_pair_gemm", "rows": enc_rows,
                                       "operands": "one fp16 activation operand, fp16 weight copies" if half_scratch is not None
                                                   else "bf16 hi + lo activation parts, bf16 weights",

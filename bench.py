@@ -510,7 +510,7 @@ def run_decode(args, w: si.Workload, inputs: Inputs, rank: int, world: int):
         "steps": K, "warmup": Wm, "ms_per_step": dev_ms / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "V": w.V, "d": w.d, "B": w.B, "prompt_tokens": w.T,
-                   "M": w.M, "cap": w.cap, "enc_layers": w.enc_layers, "enc_dff": w.dff,
+                   "M": w.M, "cap": w.cap, "enc_layers": w.enc_layers, "enc_dff": w.dff, "tied": int(w.tied),
                    "select": ("argmax computed, the update is fed the LZW codes of a generator continuation "
                               "(teacher forcing)" if forced_mode else "argmax, free-running"),
                    "replicas": world,
@@ -921,6 +921,9 @@ def main(argv=None):
     ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S,
                     help="device time the repeated K-step regions of a decode workload must cover (0: one region, "
                          "for runs under a profiler)")
+    ap.add_argument("--tied", action="store_true",
+                    help="decode workloads: tied embedding / unembedding tables, one hyper-encoder and one cache "
+                         "for both sides (Section 2.2)")
     ap.add_argument("--stub", action="store_true", help="launcher self-test: ranks report fixed numbers, no GPU work")
     args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3)
@@ -943,6 +946,8 @@ def main(argv=None):
     else:
         inputs = Inputs(_local_device())
         w = si.WORKLOADS[args.workload or DEFAULT_WORKLOAD]
+        if args.tied:
+            w = w.scaled(tied=1)
         prompt_mode = w.steps == 0
         if prompt_mode:
             line = run_prompt_scoring(args, w, inputs, rank, world, max(1, args.prompt_steps), 3)
